@@ -1,0 +1,338 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests retypes the oracle's formulas: each compares the oracle with
+a closed form, a hand-computable case, an invariant, a library routine
+(torch SDPA, scikit-learn's cosine similarity), exhaustive search on tiny
+inputs, or a value the paper prints (Tables 1-2).
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from adsa_workloads import bf16_bits_to_f32, f32_to_bf16_bits, structured_values
+from oracle import adsa_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "tables_1_2_cache_rows.txt")
+
+
+def _bf16(x):
+    return bf16_bits_to_f32(f32_to_bf16_bits(np.asarray(x, dtype=np.float32)))
+
+
+def _randn(rng, *shape):
+    return _bf16(rng.standard_normal(shape))
+
+
+# --------------------------------------------------------------------------
+# Section 4.1 partition: local window against brute-force grid enumeration
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("H,W", [(1, 1), (1, 5), (5, 1), (3, 4), (4, 4), (16, 16)])
+@pytest.mark.parametrize("R", [1, 2])
+def test_local_window_matches_grid_neighbour_enumeration(H, W, R):
+    T0 = 7
+    for r in range(H):
+        for c in range(W):
+            cur = T0 + r * W + c
+            # brute force over every cell (r2, c2): earlier in raster order, at most R rows up
+            want = set()
+            for r2 in range(H):
+                for c2 in range(W):
+                    earlier = (r2 < r) or (r2 == r and c2 < c)
+                    if earlier and (r - r2) <= R:
+                        want.add(T0 + r2 * W + c2)
+            got = {p for p in range(cur) if orc.region(p, cur, T0, W, T0, R) == orc.REGION_LOCAL}
+            assert got == want
+            assert len(got) == min(r, R) * W + c
+            # the two attention peaks of Fig. 2: previous token and same column one row up
+            if c > 0 or r > 0:
+                assert (cur - 1) in got or cur - 1 < T0
+            if r > 0:
+                assert (cur - W) in got
+            # text rows are never local; with n_prefix = T0 they are all prefix
+            assert all(orc.region(p, cur, T0, W, T0, R) == orc.REGION_PREFIX for p in range(T0))
+
+
+def test_partition_is_exhaustive_and_prefix_threshold_moves():
+    T0, W = 5, 4
+    cur = T0 + 11
+    for n_prefix in (0, 3, T0, T0 + 2):
+        regions = [orc.region(p, cur, T0, W, n_prefix, 1) for p in range(cur)]
+        assert all(r in (0, 1, 2) for r in regions)
+        assert [r == orc.REGION_PREFIX for r in regions] == [p < n_prefix for p in range(cur)]
+    # rows at or beyond the current position cannot be cached
+    assert orc.region(cur, cur, T0, W, T0, 1) == orc.REGION_INVALID
+    assert orc.region(-1, cur, T0, W, T0, 1) == orc.REGION_INVALID
+    # while decoding the text condition itself nothing is local
+    assert orc.region(2, 4, T0, W, 0, 1) == orc.REGION_PREVIOUS
+
+
+# --------------------------------------------------------------------------
+# Eq. 1-2: hand cases, closed forms, invariants, library routine
+# --------------------------------------------------------------------------
+def test_score_identical_rows_is_one_and_orthogonal_rows_is_zero():
+    v = np.tile(_bf16([[0.5, -2.0, 3.0, 1.0]]), (6, 1))
+    np.testing.assert_allclose(orc.score_definition(v), 1.0, atol=1e-6)
+    np.testing.assert_allclose(orc.score_definition(np.eye(5, 8, dtype=np.float32) * 3.0), 0.0, atol=1e-7)
+
+
+def test_score_two_orthogonal_clusters_closed_form():
+    a, b = 3, 5
+    e0, e1 = np.zeros(6, np.float32), np.zeros(6, np.float32)
+    e0[1], e1[4] = 2.0, 0.25
+    v = np.stack([e0] * a + [e1] * b)
+    s = orc.score_definition(v)
+    p = a + b
+    np.testing.assert_allclose(s[:a], (a - 1) / (p - 1), atol=1e-6)
+    np.testing.assert_allclose(s[a:], (b - 1) / (p - 1), atol=1e-6)
+
+
+def test_score_antipodal_pair_and_known_angle():
+    # rows: x, -x, y with y orthogonal to x  ->  S = (-1+0)/2, (-1+0)/2, 0
+    v = np.array([[1, 0, 0], [-4, 0, 0], [0, 2, 0]], dtype=np.float32)
+    np.testing.assert_allclose(orc.score_definition(v), [-0.5, -0.5, 0.0], atol=1e-7)
+    # 60 degrees apart: cos = 1/2, p = 2 so S_i = S_ij
+    v = np.array([[1, 0], [0.5, np.sqrt(3) / 2]], dtype=np.float32)
+    np.testing.assert_allclose(orc.score_definition(v), [0.5, 0.5], atol=1e-6)
+
+
+def test_score_zero_row_and_degenerate_sizes():
+    v = np.array([[0, 0, 0], [1, 1, 0], [1, 1, 0]], dtype=np.float32)
+    np.testing.assert_allclose(orc.score_definition(v), [0.0, 0.5, 0.5], atol=1e-6)
+    assert orc.score_definition(np.ones((1, 4), np.float32)).tolist() == [0.0]
+    assert orc.score_definition(np.zeros((0, 4), np.float32)).shape == (0,)
+
+
+def test_score_matches_sklearn_cosine_similarity_offdiagonal_mean():
+    from sklearn.metrics.pairwise import cosine_similarity
+    rng = np.random.default_rng(3)
+    for p, d in [(2, 4), (17, 64), (50, 100)]:
+        v = _randn(rng, p, d)
+        c = cosine_similarity(v.astype(np.float64))
+        want = (c.sum(axis=1) - np.diag(c)) / (p - 1)
+        np.testing.assert_allclose(orc.score_definition(v), want, atol=2e-7)
+
+
+def test_score_scale_invariance_permutation_equivariance():
+    rng = np.random.default_rng(4)
+    v = _randn(rng, 23, 16)
+    s = orc.score_definition(v)
+    scales = (2.0 ** rng.integers(-3, 4, size=(23, 1))).astype(np.float32)  # exact in bf16
+    np.testing.assert_allclose(orc.score_definition(v * scales), s, atol=1e-7)
+    perm = rng.permutation(23)
+    np.testing.assert_allclose(orc.score_definition(v[perm]), s[perm], atol=1e-7)
+    # sum over i of (p-1) S_i counts every unordered pair twice
+    from sklearn.metrics.pairwise import cosine_similarity
+    c = cosine_similarity(v.astype(np.float64))
+    np.testing.assert_allclose(s.astype(np.float64).sum() * 22, c.sum() - np.trace(c), rtol=1e-5)
+
+
+@pytest.mark.parametrize("kind", ["iid", "clusters", "duplicates", "equal", "zeros"])
+def test_rowsum_variant_agrees_with_definition(kind):
+    v = bf16_bits_to_f32(structured_values(kind, 97, 64, seed=11))
+    np.testing.assert_allclose(orc.score_rowsum(v), orc.score_definition(v), atol=1e-6)
+
+
+# --------------------------------------------------------------------------
+# Eq. 3: exhaustive subset search, ties, the eviction special case
+# --------------------------------------------------------------------------
+def _brute_force_subset(score, pos, K):
+    best = None
+    for sub in itertools.combinations(range(len(score)), K):
+        key = (sum(float(score[i]) for i in sub), tuple(sorted(int(pos[i]) for i in sub)))
+        if best is None or key < best[0]:
+            best = (key, sub)
+    return set(best[1]) if best else set()
+
+
+def test_select_equals_argmin_over_all_subsets():
+    rng = np.random.default_rng(5)
+    for trial in range(30):
+        p = int(rng.integers(1, 11))
+        # dyadic scores: subset sums are exact, ties are frequent
+        score = (rng.integers(-4, 5, size=p) / 8.0).astype(np.float32)
+        pos = rng.permutation(40)[:p].astype(np.int32)
+        for K in range(p + 1):
+            keep = orc.select_lowest(score, pos, K)
+            assert set(np.flatnonzero(keep).tolist()) == _brute_force_subset(score, pos, K)
+
+
+def test_select_all_equal_scores_keeps_lowest_positions_and_clamps():
+    pos = np.array([9, 2, 7, 4, 30, 1], dtype=np.int32)
+    score = np.full(6, 0.25, dtype=np.float32)
+    keep = orc.select_lowest(score, pos, 3)
+    assert sorted(pos[keep == 1].tolist()) == [1, 2, 4]
+    assert orc.select_lowest(score, pos, 0).sum() == 0
+    assert orc.select_lowest(score, pos, 99).sum() == 6
+
+
+def test_select_k_equals_p_minus_one_evicts_the_most_similar_token():
+    # Section 4.2: when the cache is full the token most similar to the others goes
+    v = np.eye(12, 16, dtype=np.float32) * 2.0   # mutually orthogonal rows: S = 0
+    v[7] = v[3]                                  # rows 3 and 7 are duplicates: S = 1/(p-1) for both
+    s = orc.score_definition(v)
+    pos = np.arange(100, 112, dtype=np.int32)
+    keep = orc.select_lowest(s, pos, 11)
+    evicted = int(np.flatnonzero(keep == 0)[0])
+    assert s[evicted] == s.max()
+    assert evicted == 7  # equal scores: the lower position (row 3) is kept
+
+
+# --------------------------------------------------------------------------
+# Attention: closed forms, invariants, library routine
+# --------------------------------------------------------------------------
+def test_attention_closed_forms():
+    d = 4
+    v = np.array([[1, 2, 3, 4], [5, 6, 7, 8], [-1, 0, 1, 0]], dtype=np.float32)
+    # equal keys -> uniform weights -> mean of V
+    out, w = orc.attend(np.ones(d, np.float32), np.ones((3, d), np.float32), v)
+    np.testing.assert_allclose(w, 1 / 3, atol=1e-12)
+    np.testing.assert_allclose(out, v.mean(axis=0), atol=1e-12)
+    # q = 0 -> the same
+    out, _ = orc.attend(np.zeros(d, np.float32), np.arange(12, dtype=np.float32).reshape(3, d), v)
+    np.testing.assert_allclose(out, v.mean(axis=0), atol=1e-12)
+    # two keys whose logits differ by ln 3 -> weights 3/4 and 1/4 (scale given explicitly)
+    q = np.array([1, 0, 0, 0], np.float32)
+    k = np.array([[2, 9, 9, 9], [1, -5, 0, 3]], np.float32)
+    out, w = orc.attend(q, k, v[:2], scale=np.log(3.0))
+    np.testing.assert_allclose(w, [0.75, 0.25], atol=1e-12)
+    np.testing.assert_allclose(out, 0.75 * v[0] + 0.25 * v[1], atol=1e-12)
+    # default scale is 1/sqrt(d): d = 4 halves the logits, so a gap of 2 ln 3 gives 3:1 again
+    k2 = np.array([[2 * np.log(3.0), 0, 0, 0], [0, 0, 0, 0]], np.float32)
+    _, w = orc.attend(q, k2, v[:2])
+    np.testing.assert_allclose(w, [0.75, 0.25], atol=1e-6)
+    # one dominant key -> its value row
+    out, _ = orc.attend(q * 100, np.array([[5, 0, 0, 0], [0, 0, 0, 0], [-5, 0, 0, 0]], np.float32), v)
+    np.testing.assert_allclose(out, v[0], atol=1e-9)
+
+
+def test_attention_invariants_and_sdpa():
+    rng = np.random.default_rng(7)
+    for n, d in [(1, 8), (37, 64), (200, 100)]:
+        q, k, v = _randn(rng, d), _randn(rng, n, d), _randn(rng, n, d)
+        out, w = orc.attend(q, k, v)
+        assert abs(w.sum() - 1.0) < 1e-12 and (w >= 0).all()
+        assert (out <= v.max(axis=0) + 1e-9).all() and (out >= v.min(axis=0) - 1e-9).all()
+        # shifting every key by the same vector moves all logits equally
+        out2, _ = orc.attend(q, k + _bf16(np.ones(d)), v)
+        np.testing.assert_allclose(out2, out, atol=1e-9)
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q.astype(np.float64))[None, None, None, :],
+            torch.from_numpy(k.astype(np.float64))[None, None],
+            torch.from_numpy(v.astype(np.float64))[None, None])[0, 0, 0].numpy()
+        np.testing.assert_allclose(out, ref, atol=1e-10)
+
+
+# --------------------------------------------------------------------------
+# The layer-step: dense equivalence, set invariants, Tables 1-2
+# --------------------------------------------------------------------------
+def _run_steps(T0, H, W, d, budget_fn, n_prefix, seed, score_variant=0, n_streams=2):
+    rng = np.random.default_rng(seed)
+    L = T0 + H * W
+    st = orc.OracleStreams(n_streams, d, L, T0, W, n_prefix, score_variant=score_variant)
+    hist_k = np.zeros((n_streams, L, d), np.float32)
+    hist_v = np.zeros((n_streams, L, d), np.float32)
+    if T0:
+        hist_k[:, :T0], hist_v[:, :T0] = _randn(rng, n_streams, T0, d), _randn(rng, n_streams, T0, d)
+        st.append_rows(hist_k[:, :T0], hist_v[:, :T0], 0)
+    log = []
+    for g in range(H * W):
+        cur = T0 + g
+        q, kn, vn = _randn(rng, n_streams, d), _randn(rng, n_streams, d), _randn(rng, n_streams, d)
+        hist_k[:, cur], hist_v[:, cur] = kn, vn
+        before = [set(st.rows(s)[0].tolist()) for s in range(n_streams)]
+        res = st.step(q, kn, vn, cur, budget_fn(cur))
+        log.append((cur, q, before, res, st.n_live.copy()))
+    return st, hist_k, hist_v, log
+
+
+def test_budget_covering_the_context_is_dense_attention():
+    # "behaves identically to the baseline when the cache is not full" (Section 4.2)
+    T0, H, W, d = 6, 4, 5, 16
+    st, hk, hv, log = _run_steps(T0, H, W, d, lambda cur: 10_000, T0, seed=8)
+    for cur, q, before, res, n_live in log:
+        assert (n_live == cur + 1).all()
+        for s in range(2):
+            assert len(res.evict_pos[s]) == 0
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                torch.from_numpy(q[s].astype(np.float64))[None, None, None, :],
+                torch.from_numpy(hk[s, :cur + 1].astype(np.float64))[None, None],
+                torch.from_numpy(hv[s, :cur + 1].astype(np.float64))[None, None])[0, 0, 0].numpy()
+            np.testing.assert_allclose(res.out[s], ref, atol=1e-10)
+
+
+def test_sparse_step_attends_exactly_the_retained_rows():
+    # the output must equal library attention restricted to kept_pos + the new row
+    T0, H, W, d = 5, 6, 6, 8
+    C = (T0 + H * W) // 2
+    st, hk, hv, log = _run_steps(T0, H, W, d, lambda cur: C, T0, seed=9)
+    for cur, q, before, res, n_live in log:
+        for s in range(2):
+            idx = np.array(sorted(res.kept_pos[s].tolist()) + [cur])
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                torch.from_numpy(q[s].astype(np.float64))[None, None, None, :],
+                torch.from_numpy(hk[s, idx].astype(np.float64))[None, None],
+                torch.from_numpy(hv[s, idx].astype(np.float64))[None, None])[0, 0, 0].numpy()
+            np.testing.assert_allclose(res.out[s], ref, atol=1e-10)
+
+
+@pytest.mark.parametrize("n_prefix_kind", ["text", "none", "text+5%"])
+def test_update_invariants(n_prefix_kind):
+    T0, H, W, d = 6, 6, 5, 8
+    L = T0 + H * W
+    C = L // 2
+    n_prefix = {"text": T0, "none": 0, "text+5%": T0 + int(np.ceil(0.05 * H * W))}[n_prefix_kind]
+    st, hk, hv, log = _run_steps(T0, H, W, d, lambda cur: C, n_prefix, seed=10)
+    gone = [set(), set()]
+    for cur, q, before, res, n_live in log:
+        g = cur - T0
+        r, c = divmod(g, W)
+        for s in range(2):
+            kept, ev = set(res.kept_pos[s].tolist()), set(res.evict_pos[s].tolist())
+            assert kept | ev == before[s] and not (kept & ev)
+            assert not (ev & {p for p in before[s] if p < n_prefix})            # prefix never leaves
+            local = {T0 + g2 for g2 in range(g) if r - g2 // W <= 1}
+            assert local <= kept or local <= kept | {p for p in local if p < n_prefix}
+            assert set(res.cand_pos[s].tolist()) == before[s] - local - set(range(n_prefix))
+            mandatory = len(before[s] & (local | set(range(n_prefix))))
+            assert n_live[s] == max(min(len(before[s]) + 1, C), mandatory + 1)
+            assert not (before[s] & gone[s])                                     # evicted rows never return
+            gone[s] |= ev
+            # the evicted rows are the highest-scoring candidates
+            if len(ev):
+                sc = dict(zip(res.cand_pos[s].tolist(), res.cand_score[s].tolist()))
+                assert min(sc[p] for p in ev) >= max([sc[p] for p in kept if p in sc] or [-np.inf])
+    for s in range(2):
+        pos, k, v = st.rows(s)
+        assert len(set(pos.tolist())) == len(pos)
+        np.testing.assert_array_equal(k, hk[s, pos])                             # payload bit-identical
+        np.testing.assert_array_equal(v, hv[s, pos])
+
+
+def _golden_rows():
+    rows = []
+    with open(GOLDEN) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                t, h, w, dense, cache, red = line.split()
+                rows.append((int(t), int(h), int(w), int(dense), int(cache), float(red)))
+    return rows
+
+
+@pytest.mark.parametrize("table,H,W,dense,cache,printed", _golden_rows())
+def test_cache_sizes_of_tables_1_and_2(table, H, W, dense, cache, printed):
+    assert H * W == dense
+    # the reduction the paper prints next to each cache size
+    assert abs((1 - cache / dense) * 100 - printed) < 0.06
+    # image tokens only (T0 = 0, no text condition), fixed capacity = the printed cache size
+    st, hk, hv, log = _run_steps(0, H, W, 4, lambda cur: cache, 0, seed=12, n_streams=1)
+    peak = 0
+    for cur, q, before, res, n_live in log:
+        peak = max(peak, int(n_live[0]))
+        if cur + 1 <= cache:
+            assert len(res.evict_pos[0]) == 0 and n_live[0] == cur + 1           # dense until full
+        else:
+            assert len(res.evict_pos[0]) == 1 and n_live[0] == cache             # then one eviction per step
+    assert peak == cache
