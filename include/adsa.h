@@ -1,0 +1,206 @@
+/*
+ * libadsa: decode attention with Adaptive Dynamic Sparse Attention (ADSA) on a
+ * paged bf16 KV pool, for one NVIDIA B200 (sm_100a).
+ *
+ * The library implements one layer-step of the method of "Make It Efficient:
+ * Dynamic Sparse Attention for Autoregressive Image Generation" (Section 4):
+ *
+ *   adsa_score               Eq. 1-2   mean pairwise cosine similarity of the cached V rows
+ *   adsa_select              Eq. 3     keep prefix + 2D-local window + the K lowest-scoring rows
+ *   adsa_sparse_decode_attn  Eq. 4     softmax(q.K^T).V over the retained rows and the new row
+ *   adsa_kv_update           Sec. 4.2  evict what was not retained, insert the new row, compact
+ *
+ * Vocabulary.  A *stream* is one (layer, batch row, head); it owns a private
+ * cache of rows (pos, k[d], v[d]).  Stream index = (layer*batch + b)*n_heads + h.
+ * Context position `pos` counts the text condition first (0 .. n_text-1) and
+ * then the image grid in raster order: cell g = pos - n_text, row g / grid_w,
+ * column g % grid_w.  Live rows of a stream occupy slots 0 .. n_live-1; slot s
+ * lives in page page_table[stream][s / page_rows] at row s % page_rows.  The
+ * order of rows inside a stream is not part of the contract (compaction moves
+ * rows); a stream is the *set* of its (pos, k, v) rows.
+ *
+ * General rules.
+ *   - Every function returns 0 (ADSA_OK) or a negative adsa_status.  Nothing
+ *     throws or aborts.  A CUDA error is sticky: later calls return ADSA_ECUDA.
+ *   - Pointers marked [device] must be device memory of the current device,
+ *     owned by the caller and alive for as long as the context uses them;
+ *     pointers marked [host] are ordinary host memory.  The library allocates
+ *     no device memory; it owns only the host-side adsa_ctx.
+ *   - Calls taking a cudaStream_t only enqueue work on that stream; they do not
+ *     synchronise (the *_host variants and adsa_get_status say so where they do).
+ *   - Inconsistencies that only the device can see (pool exhausted, a cached
+ *     position at or after cur_pos) set bits of a status word, skip the
+ *     offending access and never trap; read it with adsa_get_status.
+ *   - A context is not thread-safe: use it from one host thread at a time.
+ *   - bf16 tensors are dense, row-major, innermost dimension head_dim
+ *     ([batch][n_heads][head_dim] unless stated); all arithmetic is fp32.
+ */
+#ifndef ADSA_H_
+#define ADSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define ADSA_API __attribute__((visibility("default")))
+#else
+#define ADSA_API
+#endif
+
+typedef struct CUstream_st *adsa_stream_t; /* a cudaStream_t; 0 = the default stream */
+typedef struct adsa_ctx adsa_ctx;          /* opaque, host side only */
+
+typedef enum {
+    ADSA_OK = 0,
+    ADSA_EINVAL = -1, /* bad argument or configuration */
+    ADSA_ESTATE = -2, /* calls out of order, or cur_pos differs between the calls of one layer-step */
+    ADSA_ENOMEM = -3, /* pool, workspace or row capacity too small (found on the host, nothing launched) */
+    ADSA_ECUDA = -4   /* a CUDA call failed; sticky */
+} adsa_status;
+
+/* bits of the device status word (adsa_get_status) */
+#define ADSA_DEV_POOL_EXHAUSTED 1u /* a page was needed and the free ring was empty */
+#define ADSA_DEV_BAD_POSITION 2u   /* a cached row had pos < 0 or pos >= cur_pos */
+#define ADSA_DEV_ROW_OVERFLOW 4u   /* a stream would exceed max_rows_per_stream */
+#define ADSA_DEV_RING_TIMEOUT 8u   /* bounded wait on a free-ring entry ran out */
+#define ADSA_DEV_BAD_EVICT 16u     /* hole/survivor pairing of the compaction did not balance */
+#define ADSA_DEV_COPY_TIMEOUT 32u  /* bounded wait on a bulk copy into shared memory ran out */
+
+typedef struct {
+    int32_t n_layers, batch, n_heads; /* multi-head attention: one KV head per query head */
+    int32_t head_dim;                 /* d, 8 .. 256 */
+    int32_t row_stride;               /* elements per pool row: >= head_dim, a multiple of 8 (16 bytes), <= 256 */
+    int32_t page_rows;                /* rows per page, 2 .. 4096 */
+    int32_t n_pages;                  /* pages in k_pool (and in v_pool) */
+    int32_t max_rows_per_stream;      /* largest n_live any stream may reach */
+    int32_t n_text, grid_h, grid_w;   /* position -> grid cell mapping */
+    int32_t n_prefix;                 /* rows with pos < n_prefix are always kept (Section 4.1 "prefix") */
+    int32_t local_rows_back;          /* R: the local window holds the current grid row and R rows above it */
+    int32_t score_mode;               /* 0 = mean V-cosine similarity, keep the lowest (Eq. 1-3) */
+    float softmax_scale;              /* 0 => 1/sqrt(head_dim) */
+} adsa_config;
+
+typedef struct {
+    void *k_pool, *v_pool;   /* [device] bf16 [n_pages][page_rows][row_stride], 16-byte aligned */
+    int32_t *page_table;     /* [device] [n_streams][ceil(max_rows_per_stream / page_rows)] */
+    int32_t *pos;            /* [device] [n_streams][max_rows_per_stream] context position per slot */
+    float *inv_norm;         /* [device] [n_streams][max_rows_per_stream] 1 / max(|v|, 1e-8) per slot */
+    int32_t *n_live;         /* [device] [n_streams] */
+    int32_t *free_ring;      /* [device] [n_pages] ring of free page ids */
+    int32_t *free_state;     /* [device] [4]: head, tail, free count, low-water mark of the free count */
+    void *workspace;         /* [device] scratch of adsa_workspace_bytes() bytes, 256-byte aligned */
+    size_t workspace_bytes;
+} adsa_buffers;
+/* n_streams = n_layers * batch * n_heads.  All buffers are initialised by adsa_reset. */
+
+/* Scratch size the configuration needs (scores, keep masks, evict lists, split
+ * partials, staging for the *_host call).  No CUDA call is made. */
+ADSA_API int adsa_workspace_bytes(const adsa_config *cfg, size_t *out_bytes);
+
+/* Validate cfg and buffers and build the host-side context.  Queries the
+ * current device's SM count; launches nothing.  ADSA_EINVAL / ADSA_ENOMEM
+ * (workspace too small) on failure, *out untouched. */
+ADSA_API int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out);
+ADSA_API int adsa_destroy(adsa_ctx *ctx);
+
+/* Empty every stream, put all pages on the free ring, clear the status word. */
+ADSA_API int adsa_reset(adsa_ctx *ctx, adsa_stream_t stream);
+
+/* Append n_rows rows to every stream of `layer` (how the text condition, or a
+ * saved cache, enters the pool).  k, v: [device] bf16
+ * [batch][n_heads][n_rows][head_dim].  Positions are first_pos ..
+ * first_pos+n_rows-1 when pos is NULL, else pos: [device] int32
+ * [batch][n_heads][n_rows] gives each row's position (distinct per stream, and
+ * distinct from the rows already cached).  Pages are taken from the free ring
+ * as needed.  ADSA_ENOMEM if rows or pages cannot fit. */
+ADSA_API int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, const int32_t *pos, int n_rows,
+                               int first_pos, adsa_stream_t stream);
+
+/* Replace the cache of one stream by the given rows (tests, resynchronisation,
+ * restoring a snapshot).  k, v: [device] bf16 [n_rows][head_dim]; pos: [device]
+ * int32 [n_rows], distinct.  Pages are freed or taken as needed. */
+ADSA_API int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, const void *v, const int32_t *pos,
+                         int n_rows, adsa_stream_t stream);
+
+/* ---- the four calls of one layer-step, in this order, with the same cur_pos ----
+ * cur_pos is the context position of the token being decoded (its row is "the
+ * new row").  Section 4.1 partitions each stream's live rows by position into
+ * prefix (pos < n_prefix), local (image cells before the current one, in the
+ * current grid row or the R rows above) and previous (the rest). */
+
+/* Eq. 1-2.  For every row i of the previous region of every stream of `layer`:
+ * S_i = (1/(p-1)) sum_{j != i} cos(v_i, v_j), j over the same region (p rows);
+ * p <= 1 gives 0.  Computed through the identity sum_j cos = u_i.(sum_j u_j) - u_i.u_i
+ * with u = v * inv_norm.  Scores stay in the workspace for adsa_select.
+ * scores_out: [device] float [batch*n_heads][max_rows_per_stream] indexed by
+ * slot, NaN for rows outside the previous region; may be NULL. */
+ADSA_API int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_stream_t stream);
+
+/* Eq. 3 plus the always-kept regions.  budget_rows counts the new row:
+ * K = min(p, max(0, budget_rows - |prefix| - |local| - 1)) previous rows are
+ * kept, the K lowest in the order (score ascending, position ascending).
+ * Outputs (each [device], each may be NULL), stream-major with stride
+ * max_rows_per_stream, entries in ascending slot order:
+ *   sel_slots / sel_pos     retained cached rows (the new row is not listed)
+ *   evict_pos               rows that adsa_kv_update will drop
+ *   counts                  int32 [batch*n_heads][4]: previous rows p, evicted, retained, K */
+ADSA_API int adsa_select(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, int32_t *sel_slots, int32_t *sel_pos,
+                int32_t *evict_pos, int32_t *counts, adsa_stream_t stream);
+
+/* Eq. 4 and the attention of Fig. 3: out = softmax_j(q.k_j * scale) . v_j over
+ * the retained rows and the new row (k_new, v_new), maximum subtracted, fp32.
+ * q, k_new, v_new: [device] bf16 [batch][n_heads][head_dim].
+ * out_bf16: [device] bf16 same shape (round to nearest even); out_f32: [device]
+ * float same shape.  Either output may be NULL, not both. */
+ADSA_API int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q, const void *k_new,
+                            const void *v_new, void *out_bf16, float *out_f32, adsa_stream_t stream);
+
+/* Section 4.2.  Drops the rows adsa_select marked, writes the new row
+ * (k_new, v_new, cur_pos, its inverse norm) and compacts so that live rows are
+ * slots 0 .. n_live-1: holes are filled by the new row and by survivors from
+ * the tail.  Pages that became empty return to the free ring; a page is taken
+ * when the stream grows into one.  Evict-before-insert: a stream never holds
+ * more than max(budget_rows, |prefix|+|local|+1) rows. */
+ADSA_API int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, const void *v_new,
+                   adsa_stream_t stream);
+
+/* The four calls above in one: score, select, attend, update for `layer`. */
+ADSA_API int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                    const void *v_new, void *out_bf16, adsa_stream_t stream);
+
+/* adsa_layer_step with HOST tensors: q, k_new, v_new [host] bf16
+ * [batch][n_heads][head_dim] are copied to staging space in the workspace,
+ * the step runs, out [host] bf16 is copied back, and the call returns after
+ * the stream has drained (it synchronises `stream`).  Pinned host memory makes
+ * the copies asynchronous up to that point. */
+ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q_host,
+                         const void *k_new_host, const void *v_new_host, void *out_host, adsa_stream_t stream);
+
+/* How adsa_sparse_decode_attn would split a stream of n_rows cached rows:
+ * number of chunks per stream and rows per chunk.  Pure host arithmetic. */
+ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);
+
+/* Override the rows per attention chunk (0 = choose automatically). */
+ADSA_API int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows);
+
+/* Upper bound, tracked on the host, of n_live over the streams of `layer`. */
+ADSA_API int adsa_layer_rows_bound(const adsa_ctx *ctx, int layer, int *n_rows);
+
+/* Synchronises the device, then copies out the device status word (OR of
+ * ADSA_DEV_* bits since the last reset) and the free-ring state
+ * {head, tail, free pages, fewest free pages seen}.  Either pointer may be NULL. */
+ADSA_API int adsa_get_status(adsa_ctx *ctx, uint32_t *dev_status, int32_t free_state[4]);
+
+/* Number of kernels this context has launched so far (host counter). */
+ADSA_API int64_t adsa_launch_count(const adsa_ctx *ctx);
+
+ADSA_API const char *adsa_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADSA_H_ */

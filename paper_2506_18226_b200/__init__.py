@@ -1,0 +1,12 @@
+"""B200-native ADSA decode attention: CUDA kernels behind a C-ABI (libadsa.so) plus a thin binding."""
+from .binding import (  # noqa: F401
+    AdsaBuffers,
+    AdsaConfig,
+    AdsaEngine,
+    AdsaError,
+    EXPORTS,
+    load,
+    strerror,
+    workspace_bytes,
+)
+from .build import build_lib  # noqa: F401

@@ -1,0 +1,446 @@
+// C-ABI of libadsa: argument checking, the host-side state machine of a
+// layer-step (score -> select -> attend -> update), launch planning, and the
+// host-buffer variant.  Row counts are functions of positions and budgets only,
+// never of data, so every launch is sized on the host without reading back.
+#include <math.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+#include <vector>
+
+#include "adsa_dev.cuh"
+#include "adsa_launch.h"
+
+using namespace adsa;
+
+namespace {
+
+enum Phase { kIdle = 0, kScored = 1, kSelected = 2, kAttended = 3 };
+
+struct LayerState {
+    int phase = kIdle;
+    int cur_pos = -1;
+    int budget = 0;
+    int rows_hi = 0;   // upper bound of n_live over the layer's streams
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+    size_t scores, keep_mask, evict_slots, counts, partials, tickets, status, staging, total;
+};
+
+int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
+
+WorkspaceLayout layout_of(const adsa_config &cfg)
+{
+    const size_t S = (size_t)cfg.batch * cfg.n_heads, R = (size_t)cfg.max_rows_per_stream;
+    WorkspaceLayout w;
+    size_t off = 0;
+    w.scores = off;      off = align_up(off + S * R * sizeof(float), 256);
+    w.keep_mask = off;   off = align_up(off + S * mask_words_of(cfg) * sizeof(uint32_t), 256);
+    w.evict_slots = off; off = align_up(off + S * R * sizeof(int32_t), 256);
+    w.counts = off;      off = align_up(off + S * 4 * sizeof(int32_t), 256);
+    w.partials = off;    off = align_up(off + S * kMaxSplits * (size_t)(cfg.row_stride + 2) * sizeof(float), 256);
+    w.tickets = off;     off = align_up(off + S * sizeof(int32_t), 256);
+    w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
+    w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.head_dim * sizeof(__nv_bfloat16), 256);
+    w.total = off;
+    return w;
+}
+
+int check_config(const adsa_config *c)
+{
+    if (!c) return ADSA_EINVAL;
+    if (c->n_layers < 1 || c->batch < 1 || c->n_heads < 1) return ADSA_EINVAL;
+    if (c->head_dim < 8 || c->head_dim > 256) return ADSA_EINVAL;
+    if (c->row_stride < c->head_dim || c->row_stride % 8 != 0 || c->row_stride > 256) return ADSA_EINVAL;
+    if (c->page_rows < 2 || c->page_rows > 4096) return ADSA_EINVAL;
+    if (c->n_pages < 1) return ADSA_EINVAL;
+    if (c->max_rows_per_stream < 1 || c->max_rows_per_stream > 16384) return ADSA_EINVAL;
+    if (c->n_text < 0 || c->grid_h < 1 || c->grid_w < 1) return ADSA_EINVAL;
+    if (c->n_prefix < 0 || c->local_rows_back < 0) return ADSA_EINVAL;
+    if (c->score_mode != 0) return ADSA_EINVAL;
+    if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return ADSA_EINVAL;
+    if ((long long)c->n_layers * c->batch * c->n_heads > (1ll << 24)) return ADSA_EINVAL;
+    if ((long long)c->n_pages * c->page_rows * c->row_stride > (1ll << 40)) return ADSA_EINVAL;
+    return ADSA_OK;
+}
+
+// slot / page_rows == umulhi(slot, magic) for every slot the pool can hold
+bool magic_divides(uint32_t magic, int page_rows, int max_rows)
+{
+    for (int s = 0; s <= max_rows; ++s)
+        if ((uint32_t)(((uint64_t)s * magic) >> 32) != (uint32_t)(s / page_rows)) return false;
+    return true;
+}
+
+}  // namespace
+
+struct adsa_ctx {
+    adsa_config cfg;
+    adsa_buffers buf;
+    DevCtx dev;
+    WorkspaceLayout ws;
+    std::vector<LayerState> layers;
+    int sm_count = 148;
+    int chunk_override = 0;
+    int cuda_error = 0;  // sticky
+    int64_t launches = 0;
+    __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
+};
+
+namespace {
+
+int cuda_fail(adsa_ctx *ctx, cudaError_t e)
+{
+    if (e == cudaSuccess) return ADSA_OK;
+    ctx->cuda_error = (int)e;
+    return ADSA_ECUDA;
+}
+
+int pages_for(const adsa_ctx *ctx, int rows) { return (rows + ctx->cfg.page_rows - 1) / ctx->cfg.page_rows; }
+
+// pages the whole pool may need if `layer` grows to `rows` rows per stream
+bool pool_can_hold(const adsa_ctx *ctx, int layer, int rows)
+{
+    long long need = 0;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l)
+        need += (long long)ctx->dev.S * pages_for(ctx, l == layer ? rows : ctx->layers[l].rows_hi);
+    return need <= ctx->cfg.n_pages;
+}
+
+// largest number of rows the prefix and local regions can hold at cur_pos
+int mandatory_rows_bound(const adsa_ctx *ctx, int cur_pos)
+{
+    const adsa_config &c = ctx->cfg;
+    int pre = c.n_prefix < cur_pos ? c.n_prefix : cur_pos;
+    int loc = 0;
+    if (cur_pos >= c.n_text) {
+        int g = cur_pos - c.n_text, r = g / c.grid_w, col = g % c.grid_w;
+        int back = r < c.local_rows_back ? r : c.local_rows_back;
+        loc = back * c.grid_w + col;
+    }
+    return pre + loc;
+}
+
+AttnPlan plan_attn(const adsa_ctx *ctx, int n_rows)
+{
+    AttnPlan p;
+    int rows = n_rows < 1 ? 1 : n_rows;
+    int chunk = ctx->chunk_override;
+    if (chunk <= 0) {
+        // enough blocks to fill every SM several times over, but no chunk below 64 rows
+        long long target_blocks = (long long)ctx->sm_count * 8;
+        int splits = (int)((target_blocks + ctx->dev.S - 1) / ctx->dev.S);
+        if (splits < 1) splits = 1;
+        chunk = (rows + splits - 1) / splits;
+        if (chunk < 64) chunk = 64;
+    }
+    chunk = (chunk + 31) / 32 * 32;
+    int splits = (rows + chunk - 1) / chunk;
+    if (splits > kMaxSplits) {
+        splits = kMaxSplits;
+        chunk = ((rows + splits - 1) / splits + 31) / 32 * 32;
+        splits = (rows + chunk - 1) / chunk;
+    }
+    p.n_splits = splits;
+    p.chunk_rows = chunk;
+    return p;
+}
+
+int check_layer(const adsa_ctx *ctx, int layer)
+{
+    if (!ctx) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return ADSA_EINVAL;
+    return ADSA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adsa_workspace_bytes(const adsa_config *cfg, size_t *out_bytes)
+{
+    int rc = check_config(cfg);
+    if (rc != ADSA_OK || !out_bytes) return ADSA_EINVAL;
+    *out_bytes = layout_of(*cfg).total;
+    return ADSA_OK;
+}
+
+int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
+{
+    int rc = check_config(cfg);
+    if (rc != ADSA_OK || !buf || !out) return ADSA_EINVAL;
+    if (!buf->k_pool || !buf->v_pool || !buf->page_table || !buf->pos || !buf->inv_norm || !buf->n_live ||
+        !buf->free_ring || !buf->free_state || !buf->workspace)
+        return ADSA_EINVAL;
+    if (((uintptr_t)buf->k_pool | (uintptr_t)buf->v_pool) & 15u) return ADSA_EINVAL;
+    if ((uintptr_t)buf->workspace & 255u) return ADSA_EINVAL;
+    WorkspaceLayout ws = layout_of(*cfg);
+    if (buf->workspace_bytes < ws.total) return ADSA_ENOMEM;
+    if ((size_t)cfg->max_rows_per_stream * 9 + 16 > 200 * 1024) return ADSA_EINVAL;
+
+    uint32_t magic = (uint32_t)((1ull << 32) / (uint32_t)cfg->page_rows) + 1u;
+    if (!magic_divides(magic, cfg->page_rows, cfg->max_rows_per_stream)) return ADSA_EINVAL;
+
+    adsa_ctx *ctx = new (std::nothrow) adsa_ctx();
+    if (!ctx) return ADSA_ENOMEM;
+    ctx->cfg = *cfg;
+    ctx->buf = *buf;
+    ctx->ws = ws;
+    ctx->layers.resize(cfg->n_layers);
+    char *w = (char *)buf->workspace;
+    DevCtx &d = ctx->dev;
+    d.k_pool = (__nv_bfloat16 *)buf->k_pool;
+    d.v_pool = (__nv_bfloat16 *)buf->v_pool;
+    d.page_table = buf->page_table;
+    d.pos = buf->pos;
+    d.n_live = buf->n_live;
+    d.inv_norm = buf->inv_norm;
+    d.free_ring = buf->free_ring;
+    d.free_state = buf->free_state;
+    d.scores = (float *)(w + ws.scores);
+    d.keep_mask = (uint32_t *)(w + ws.keep_mask);
+    d.evict_slots = (int32_t *)(w + ws.evict_slots);
+    d.counts = (int32_t *)(w + ws.counts);
+    d.partials = (float *)(w + ws.partials);
+    d.tickets = (int32_t *)(w + ws.tickets);
+    d.status = (uint32_t *)(w + ws.status);
+    d.d = cfg->head_dim;
+    d.row_stride = cfg->row_stride;
+    d.page_rows = cfg->page_rows;
+    d.n_pages = cfg->n_pages;
+    d.max_rows = cfg->max_rows_per_stream;
+    d.max_pages = (cfg->max_rows_per_stream + cfg->page_rows - 1) / cfg->page_rows;
+    d.mask_words = mask_words_of(*cfg);
+    d.S = cfg->batch * cfg->n_heads;
+    d.partial_stride = cfg->row_stride + 2;
+    d.pr_magic = magic;
+    d.n_text = cfg->n_text;
+    d.grid_w = cfg->grid_w;
+    d.n_prefix = cfg->n_prefix;
+    d.rows_back = cfg->local_rows_back;
+    float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+    d.scale_log2e = scale * 1.4426950408889634f;
+    size_t stage = (size_t)d.S * cfg->head_dim;
+    ctx->stage_q = (__nv_bfloat16 *)(w + ws.staging);
+    ctx->stage_k = ctx->stage_q + stage;
+    ctx->stage_v = ctx->stage_k + stage;
+    ctx->stage_o = ctx->stage_v + stage;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+        ctx->sm_count = sms;
+        cudaError_t e = configure_kernels(d);
+        if (e != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
+    } else {
+        cudaGetLastError();  // no usable device: host-side planning still works, launches will fail
+    }
+    *out = ctx;
+    return ADSA_OK;
+}
+
+int adsa_destroy(adsa_ctx *ctx)
+{
+    delete ctx;
+    return ADSA_OK;
+}
+
+int adsa_reset(adsa_ctx *ctx, adsa_stream_t stream)
+{
+    if (!ctx) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    for (auto &l : ctx->layers) l = LayerState();
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_reset(ctx->dev, ctx->cfg.n_layers * ctx->dev.S, (cudaStream_t)stream));
+}
+
+int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, const int32_t *pos, int n_rows,
+                      int first_pos, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (!k || !v || n_rows < 1 || first_pos < 0) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kIdle) return ADSA_ESTATE;
+    if (L.rows_hi + n_rows > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+    if (!pool_can_hold(ctx, layer, L.rows_hi + n_rows)) return ADSA_ENOMEM;
+    L.rows_hi += n_rows;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
+}
+
+int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, const void *v, const int32_t *pos,
+                         int n_rows, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (b < 0 || b >= ctx->cfg.batch || h < 0 || h >= ctx->cfg.n_heads || n_rows < 0) return ADSA_EINVAL;
+    if (n_rows > 0 && (!k || !v || !pos)) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kIdle) return ADSA_ESTATE;
+    if (n_rows > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+    int hi = n_rows > L.rows_hi ? n_rows : L.rows_hi;
+    if (!pool_can_hold(ctx, layer, hi)) return ADSA_ENOMEM;
+    L.rows_hi = hi;
+    int sid = (layer * ctx->cfg.batch + b) * ctx->cfg.n_heads + h;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_set_rows(ctx->dev, sid, k, v, pos, n_rows, (cudaStream_t)stream));
+}
+
+int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (cur_pos < 0) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kIdle) return ADSA_ESTATE;
+    L.phase = kScored;
+    L.cur_pos = cur_pos;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
+}
+
+int adsa_select(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, int32_t *sel_slots, int32_t *sel_pos,
+                int32_t *evict_pos, int32_t *counts, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (budget_rows < 1) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kScored || L.cur_pos != cur_pos) return ADSA_ESTATE;
+    // rows after the update: min(rows + 1, budget), but never below prefix + local + 1
+    int mand = mandatory_rows_bound(ctx, cur_pos) + 1;
+    int cap = budget_rows > mand ? budget_rows : mand;
+    int after = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
+    if (after > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+    if (!pool_can_hold(ctx, layer, after > L.rows_hi ? after : L.rows_hi)) return ADSA_ENOMEM;
+    L.phase = kSelected;
+    L.budget = budget_rows;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_select(ctx->dev, layer, cur_pos, budget_rows, sel_slots, sel_pos, evict_pos, counts,
+                                        (cudaStream_t)stream));
+}
+
+int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q, const void *k_new,
+                            const void *v_new, void *out_bf16, float *out_f32, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (!q || !k_new || !v_new || (!out_bf16 && !out_f32)) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
+    L.phase = kAttended;
+    AttnPlan plan = plan_attn(ctx, L.rows_hi);
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32,
+                                      (cudaStream_t)stream));
+}
+
+int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, const void *v_new, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (!k_new || !v_new) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
+    int mand = mandatory_rows_bound(ctx, cur_pos) + 1;
+    int cap = L.budget > mand ? L.budget : mand;
+    L.rows_hi = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
+    L.phase = kIdle;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_kv_update(ctx->dev, layer, cur_pos, k_new, v_new, (cudaStream_t)stream));
+}
+
+int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                    const void *v_new, void *out_bf16, adsa_stream_t stream)
+{
+    int rc = adsa_score(ctx, layer, cur_pos, nullptr, stream);
+    if (rc) return rc;
+    rc = adsa_select(ctx, layer, cur_pos, budget_rows, nullptr, nullptr, nullptr, nullptr, stream);
+    if (rc) return rc;
+    rc = adsa_sparse_decode_attn(ctx, layer, cur_pos, q, k_new, v_new, out_bf16, nullptr, stream);
+    if (rc) return rc;
+    return adsa_kv_update(ctx, layer, cur_pos, k_new, v_new, stream);
+}
+
+int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q_host,
+                         const void *k_new_host, const void *v_new_host, void *out_host, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return ADSA_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t bytes = (size_t)ctx->dev.S * ctx->cfg.head_dim * sizeof(__nv_bfloat16);
+    cudaError_t e = cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_k, k_new_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_v, v_new_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    rc = adsa_layer_step(ctx, layer, cur_pos, budget_rows, ctx->stage_q, ctx->stage_k, ctx->stage_v, ctx->stage_o, stream);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(out_host, ctx->stage_o, bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return cuda_fail(ctx, e);
+}
+
+int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows)
+{
+    if (!ctx || n_rows < 0) return ADSA_EINVAL;
+    AttnPlan p = plan_attn(ctx, n_rows);
+    if (n_splits) *n_splits = p.n_splits;
+    if (chunk_rows) *chunk_rows = p.chunk_rows;
+    return ADSA_OK;
+}
+
+int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows)
+{
+    if (!ctx || chunk_rows < 0) return ADSA_EINVAL;
+    ctx->chunk_override = chunk_rows;
+    return ADSA_OK;
+}
+
+int adsa_layer_rows_bound(const adsa_ctx *ctx, int layer, int *n_rows)
+{
+    if (!ctx || !n_rows || layer < 0 || layer >= ctx->cfg.n_layers) return ADSA_EINVAL;
+    *n_rows = ctx->layers[layer].rows_hi;
+    return ADSA_OK;
+}
+
+int adsa_get_status(adsa_ctx *ctx, uint32_t *dev_status, int32_t free_state[4])
+{
+    if (!ctx) return ADSA_EINVAL;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess && dev_status) e = cudaMemcpy(dev_status, ctx->dev.status, sizeof(uint32_t), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && free_state) e = cudaMemcpy(free_state, ctx->dev.free_state, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    return cuda_fail(ctx, e);
+}
+
+int64_t adsa_launch_count(const adsa_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *adsa_strerror(int status)
+{
+    switch (status) {
+    case ADSA_OK: return "ok";
+    case ADSA_EINVAL: return "invalid argument or configuration";
+    case ADSA_ESTATE: return "call out of order for this layer-step";
+    case ADSA_ENOMEM: return "pool, workspace or row capacity too small";
+    case ADSA_ECUDA: return "a CUDA call failed";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"
+
+namespace adsa {
+
+// Opt in to large dynamic shared memory where a configuration needs it.
+cudaError_t configure_kernels(const DevCtx &c)
+{
+    cudaError_t e = configure_select_kernel(c);
+    return e != cudaSuccess ? e : configure_update_kernel(c);
+}
+
+}  // namespace adsa

@@ -1,0 +1,315 @@
+// adsa_score (Eq. 1-2 through the row-sum identity) and adsa_select (Eq. 3 plus
+// the always-kept prefix and local window).  One block per stream: a stream's
+// candidate set is at most a few thousand rows, so its scores, keys and the
+// selection state fit in one SM's shared memory and no inter-block step exists.
+#include <math_constants.h>
+
+#include "adsa_dev.cuh"
+#include "adsa_launch.h"
+
+namespace adsa {
+
+constexpr int kSSThreads = 256;
+constexpr int kSSWarps = kSSThreads / 32;
+
+// ---------------------------------------------------------------------------
+// Eq. 1-2.  With u_j = v_j / max(|v_j|, eps) and s = sum_{j in P} u_j,
+//   sum_{j != i} cos(v_i, v_j) = u_i . s - u_i . u_i,
+// so S_i = (u_i . s - u_i . u_i) / (p - 1): two sweeps over the V rows of the
+// previous region P (the second one normally served by L2) instead of the
+// p^2 pairs of the definition.  u_i . u_i is computed, not assumed to be 1, so
+// that a zero row scores 0 as the clamped definition says.
+//
+// LPR lanes share a row, 8 elements (16 bytes) each.  Summation order is fixed
+// by the thread layout (strided slots per lane group, xor tree across groups,
+// warps in index order), so scores are reproducible run to run.
+// ---------------------------------------------------------------------------
+template <int LPR>
+__global__ void __launch_bounds__(kSSThreads)
+score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
+{
+    constexpr int RPW = 32 / LPR;
+    __shared__ float s_part[kSSWarps][256];
+    __shared__ float s_vec[256];
+    __shared__ int s_p;
+    const int local = blockIdx.x, sid = layer * c.S + local;
+    const int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
+    const int32_t *pos = c.pos + (size_t)sid * c.max_rows;
+    const float *inv_norm = c.inv_norm + (size_t)sid * c.max_rows;
+    float *scores = c.scores + (size_t)local * c.max_rows;
+    if (scores_out) scores_out += (size_t)local * c.max_rows;
+    const int n = c.n_live[sid];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane % LPR, grp = lane / LPR;
+    const bool piece_ok = sub * 8 < c.row_stride;
+    if (threadIdx.x == 0) s_p = 0;
+    __syncthreads();
+
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    int cnt = 0;
+    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {
+        int reg = region_of(c, pos[slot], cur_pos);
+        if (reg == kRegionInvalid && sub == 0) set_status(c, ADSA_DEV_BAD_POSITION);
+        if (reg != kRegionPrevious) continue;
+        if (sub == 0) ++cnt;
+        if (piece_ok) {
+            float f[8];
+            unpack8(ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8), f);
+            float inv = inv_norm[slot];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(inv, f[e], acc[e]);
+        }
+    }
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    }
+    if (grp == 0 && piece_ok) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s_part[warp][sub * 8 + e] = acc[e];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0 && cnt) atomicAdd(&s_p, cnt);
+    __syncthreads();
+    if (threadIdx.x < c.row_stride) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kSSWarps; ++w) t += s_part[w][threadIdx.x];
+        s_vec[threadIdx.x] = t;
+    }
+    __syncthreads();
+    const int p = s_p;
+    float sv[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sv[e] = piece_ok ? s_vec[sub * 8 + e] : 0.f;
+
+    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {
+        int reg = region_of(c, pos[slot], cur_pos);
+        float dot = 0.f, self = 0.f;
+        if (reg == kRegionPrevious && piece_ok) {
+            float f[8];
+            unpack8(ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], sv[e], dot); self = fmaf(f[e], f[e], self); }
+        }
+#pragma unroll
+        for (int o = 1; o < LPR; o <<= 1) {
+            dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            self += __shfl_xor_sync(0xffffffffu, self, o);
+        }
+        if (sub == 0) {
+            float S = CUDART_NAN_F;
+            if (reg == kRegionPrevious) {
+                float inv = inv_norm[slot];
+                // (p-1) S_i = u_i.s - u_i.u_i; dividing (not multiplying by a reciprocal) keeps the
+                // last bit where the definition puts it; "+ 0" folds -0 into +0 for the integer ordering
+                S = p > 1 ? (inv * dot - inv * inv * self) / (float)(p - 1) + 0.0f : 0.0f;
+            }
+            scores[slot] = S;
+            if (scores_out) scores_out[slot] = S;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 3.  Each row of the previous region gets the 64-bit key
+//   (order-preserving image of the float score) << 32 | position,
+// so "score ascending, then position ascending" is plain unsigned order and all
+// keys are distinct.  The K lowest keys are found without sorting:
+//   K >= p      keep all;   K == 0  drop all;
+//   K == p - 1  (steady state of Section 4.2, one eviction per step) drop the maximum key;
+//   otherwise   most-significant-digit-first radix select, 8 bits per pass,
+//               stopping as soon as the bin of the K-th key is taken whole.
+// The result is a threshold on a masked key: keep iff (key & mask) <= thr.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t orderable(float s)
+{
+    uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kSSThreads)
+select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_slots, int32_t *sel_pos,
+              int32_t *evict_pos, int32_t *counts_out)
+{
+    extern __shared__ unsigned long long sm_keys[];  // [max_rows], then uint8 region[max_rows]
+    __shared__ int s_cnt[3];                          // prefix, local, previous
+    __shared__ int s_hist[256];
+    __shared__ unsigned long long s_max;
+    __shared__ int s_digit, s_krem, s_bin;
+    __shared__ int s_wk[kSSWarps], s_we[kSSWarps], s_bk, s_be;
+    const int local = blockIdx.x, sid = layer * c.S + local;
+    const int32_t *pos = c.pos + (size_t)sid * c.max_rows;
+    const float *scores = c.scores + (size_t)local * c.max_rows;
+    uint8_t *region = reinterpret_cast<uint8_t *>(sm_keys + c.max_rows);
+    const int n = c.n_live[sid];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { s_max = 0ull; s_bk = 0; s_be = 0; }
+    __syncthreads();
+
+    // keys and region sizes
+    unsigned long long my_max = 0ull;
+    for (int base = 0; base < n; base += kSSThreads) {
+        int slot = base + threadIdx.x;
+        int reg = kRegionInvalid;
+        if (slot < n) {
+            int ps = pos[slot];
+            reg = region_of(c, ps, cur_pos);
+            region[slot] = (uint8_t)reg;
+            unsigned long long key = ~0ull;
+            if (reg == kRegionPrevious) {
+                key = ((unsigned long long)orderable(scores[slot]) << 32) | (uint32_t)ps;
+                my_max = key > my_max ? key : my_max;
+            }
+            sm_keys[slot] = key;
+        }
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            unsigned b = __ballot_sync(0xffffffffu, reg == r);
+            if (lane == 0 && b) atomicAdd(&s_cnt[r], __popc(b));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, my_max, o);
+        my_max = other > my_max ? other : my_max;
+    }
+    if (lane == 0) atomicMax(&s_max, my_max);
+    __syncthreads();
+    const int n_pre = s_cnt[kRegionPrefix], n_loc = s_cnt[kRegionLocal], p = s_cnt[kRegionPrevious];
+    int K = budget_rows - n_pre - n_loc - 1;
+    K = K < 0 ? 0 : (K > p ? p : K);
+
+    unsigned long long mask = 0ull, thr = 0ull;  // keep iff (key & mask) <= thr
+    bool drop_all = false;
+    if (K >= p) {
+        mask = 0ull; thr = 0ull;                 // every key passes
+    } else if (K == 0) {
+        drop_all = true;
+    } else if (K == p - 1) {
+        mask = ~0ull; thr = s_max - 1ull;        // keys are distinct: everything below the maximum
+    } else {
+        int k_rem = K;
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            s_hist[threadIdx.x] = 0;             // kSSThreads == 256 bins
+            __syncthreads();
+            for (int slot = threadIdx.x; slot < n; slot += kSSThreads) {
+                unsigned long long key = sm_keys[slot];
+                if (region[slot] == kRegionPrevious && (key & mask) == thr)
+                    atomicAdd(&s_hist[(int)((key >> shift) & 255ull)], 1);
+            }
+            __syncthreads();
+            if (warp == 0) {                     // find the bin holding the k_rem-th key of the current prefix
+                int h[8], tot = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { h[i] = s_hist[lane * 8 + i]; tot += h[i]; }
+                int incl = tot;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                int excl = incl - tot;
+                if (excl < k_rem && k_rem <= incl) {
+                    int cum = excl;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (cum < k_rem && k_rem <= cum + h[i]) { s_digit = lane * 8 + i; s_krem = k_rem - cum; s_bin = h[i]; }
+                        cum += h[i];
+                    }
+                }
+            }
+            __syncthreads();
+            thr |= (unsigned long long)s_digit << shift;
+            mask |= 255ull << shift;
+            k_rem = s_krem;
+            int bin = s_bin;
+            __syncthreads();
+            if (k_rem == bin) break;             // the whole bin is kept: masked compare decides
+        }
+    }
+
+    // retained / evicted lists in ascending slot order, keep mask, counts
+    uint32_t *keep_mask = c.keep_mask + (size_t)local * c.mask_words;
+    int32_t *ev_slots = c.evict_slots + (size_t)local * c.max_rows;
+    const size_t ob = (size_t)local * c.max_rows;
+    for (int base = 0; base < n; base += kSSThreads) {
+        int slot = base + threadIdx.x;
+        bool live = slot < n, kept = false;
+        if (live) {
+            kept = region[slot] != kRegionPrevious || (!drop_all && (sm_keys[slot] & mask) <= thr);
+            if (region[slot] == kRegionInvalid) kept = true;  // flagged by adsa_score; never silently dropped
+        }
+        unsigned bk = __ballot_sync(0xffffffffu, kept), be = __ballot_sync(0xffffffffu, live && !kept);
+        if (lane == 0) {
+            s_wk[warp] = __popc(bk); s_we[warp] = __popc(be);
+            if (base + warp * 32 < n) keep_mask[(base >> 5) + warp] = bk;
+        }
+        __syncthreads();
+        int ok_ = s_bk, oe = s_be;
+        for (int w = 0; w < warp; ++w) { ok_ += s_wk[w]; oe += s_we[w]; }
+        unsigned below = (1u << lane) - 1u;
+        if (kept) {
+            int i = ok_ + __popc(bk & below);
+            if (sel_slots) sel_slots[ob + i] = slot;
+            if (sel_pos) sel_pos[ob + i] = pos[slot];
+        } else if (live) {
+            int i = oe + __popc(be & below);
+            ev_slots[i] = slot;
+            if (evict_pos) evict_pos[ob + i] = pos[slot];
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 0; w < kSSWarps; ++w) { s_bk += s_wk[w]; s_be += s_we[w]; }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int32_t *cn = c.counts + local * 4;
+        cn[0] = p; cn[1] = s_be; cn[2] = s_bk; cn[3] = K;
+        if (counts_out) { counts_out[local * 4 + 0] = p; counts_out[local * 4 + 1] = s_be;
+                          counts_out[local * 4 + 2] = s_bk; counts_out[local * 4 + 3] = K; }
+    }
+}
+
+// ---- host launchers -------------------------------------------------------
+static int lanes_per_row(int row_stride)
+{
+    int pieces = row_stride / 8;
+    return pieces <= 4 ? 4 : pieces <= 8 ? 8 : pieces <= 16 ? 16 : 32;
+}
+
+cudaError_t launch_score(const DevCtx &c, int layer, int cur_pos, float *scores_out, cudaStream_t st)
+{
+    switch (lanes_per_row(c.row_stride)) {
+    case 4: score_kernel<4><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;
+    case 8: score_kernel<8><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;
+    case 16: score_kernel<16><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;
+    default: score_kernel<32><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;
+    }
+    return cudaGetLastError();
+}
+
+size_t select_smem_bytes(const DevCtx &c) { return (size_t)c.max_rows * 9 + 16; }
+
+cudaError_t configure_select_kernel(const DevCtx &c)
+{
+    size_t b = select_smem_bytes(c);
+    if (b <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)b);
+}
+
+cudaError_t launch_select(const DevCtx &c, int layer, int cur_pos, int budget_rows, int32_t *sel_slots,
+                          int32_t *sel_pos, int32_t *evict_pos, int32_t *counts_out, cudaStream_t st)
+{
+    select_kernel<<<c.S, kSSThreads, select_smem_bytes(c), st>>>(c, layer, cur_pos, budget_rows, sel_slots, sel_pos,
+                                                                 evict_pos, counts_out);
+    return cudaGetLastError();
+}
+
+}  // namespace adsa

@@ -1,0 +1,244 @@
+"""GPU parity: the CUDA path through the C-ABI against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from adsa_workloads import (bf16_bits_to_f32, f32_to_bf16_bits, get_workload, layer_step_qkv, pick_page_rows,
+                            prefix_kv, structured_values)
+from adsa_workloads.configs import Workload
+
+pytestmark = pytest.mark.gpu
+
+
+def _harness():
+    import harness
+    return harness
+
+
+def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=None, steps=None, n_prefix=None,
+                    rows_back=1, sample=None, chunk_rows=0, score_variant=0):
+    H = _harness()
+    cap = max(budget_fn(w.n_text + g) for g in range(w.n_cells))
+    eng = H.engine_for(w, n_layers=n_layers_engine, page_rows=page_rows, capacity=cap, n_prefix=n_prefix,
+                       local_rows_back=rows_back)
+    if chunk_rows:
+        eng.set_attn_chunk_rows(chunk_rows)
+    lh = H.LayerHarness(eng, 0, oracle_cap=w.l_max + 1, sample=sample, score_variant=score_variant)
+    if w.n_text:
+        k, v = prefix_kv(w, seed, layer)
+        lh.prefill(k, v, 0)
+    for g in range(w.n_cells if steps is None else steps):
+        q, k, v = layer_step_qkv(w, seed, layer, g)
+        lh.step(q, k, v, w.n_text + g, budget_fn(w.n_text + g))
+    status, free_state = eng.get_status()
+    assert status == 0
+    return lh, eng
+
+
+# ---------------------------------------------------------------------------
+# small shapes: several tiles, ragged tails, odd page sizes, all head-dim paths
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("d,page_rows,T0,gh,gw,beta,chunk", [
+    (64, 7, 5, 6, 5, 0.5, 0),      # pages smaller than a warp tile, ragged everywhere
+    (64, 16, 0, 5, 4, 0.5, 0),     # no text condition: the first step sees an empty cache
+    (32, 3, 4, 4, 6, 0.6, 32),     # 4 lanes per row
+    (100, 5, 9, 5, 7, 0.5, 0),     # non-power-of-two head_dim, padded row stride 104
+    (128, 11, 6, 4, 4, 0.7, 0),    # 16 lanes per row
+    (256, 4, 3, 3, 5, 0.5, 0),     # 32 lanes per row
+    (8, 2, 2, 7, 3, 0.4, 0),       # smallest head_dim
+])
+def test_small_shapes_full_trajectory(d, page_rows, T0, gh, gw, beta, chunk):
+    w = Workload(f"tiny-d{d}", 90 + d % 7, 1, 2, 3, d, T0, gh, gw, beta, 1.0)
+    C = max(2, w.capacity())
+    lh, eng = _run_trajectory(w, 0, 1, lambda cur: C, page_rows=page_rows, chunk_rows=chunk)
+    assert lh.stats.steps == gh * gw and lh.stats.max_score_err <= 1e-6
+
+
+@pytest.mark.parametrize("n_prefix_kind,rows_back", [("none", 1), ("text+5%", 1), ("text", 2), ("text", 0)])
+def test_prefix_and_window_variants(n_prefix_kind, rows_back):
+    w = Workload("tiny-variants", 97, 1, 1, 4, 64, 10, 8, 8, 0.5, 1.0)
+    n_prefix = {"none": 0, "text": w.n_text, "text+5%": w.n_text + 4}[n_prefix_kind]
+    C = w.capacity()
+    lh, eng = _run_trajectory(w, 0, 2, lambda cur: C, n_prefix=n_prefix, rows_back=rows_back, page_rows=8)
+    assert lh.stats.steps == 64
+
+
+def test_budget_covering_context_is_dense_attention():
+    # no eviction ever: every step must equal dense causal attention (the oracle's own pin)
+    w = Workload("tiny-dense", 98, 1, 1, 4, 64, 12, 10, 10, 1.0, 1.0)
+    lh, eng = _run_trajectory(w, 0, 3, lambda cur: w.l_max, page_rows=16, chunk_rows=32)
+    assert int(eng._t["n_live"].max().item()) == w.l_max
+
+
+# ---------------------------------------------------------------------------
+# the benchmark configurations
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_config1_full_trajectory(seed):
+    w = get_workload(1)
+    C = w.capacity()
+    lh, eng = _run_trajectory(w, 0, seed, lambda cur: C)
+    assert lh.stats.steps == 256
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+    # pool never exceeds the budget's share: capacity rows per stream, in whole pages
+    pr = eng.cfg.page_rows
+    assert eng.pool_bytes_peak() <= w.streams_per_layer * -(-C // pr) * pr * w.row_stride * 4
+
+
+def test_config1_budget_as_fraction_of_current_context():
+    # the literal "50 % of the current context" schedule: budget grows with the context
+    w = get_workload(1)
+    lh, eng = _run_trajectory(w, 0, 0, lambda cur: max(1, -(-(cur + 1) // 2)))
+    assert lh.stats.steps == 256
+
+
+@pytest.mark.parametrize("layer", [0, 11])
+def test_config2_full_trajectory(layer):
+    w = get_workload(2)
+    C = w.capacity()
+    lh, eng = _run_trajectory(w, layer, 0, lambda cur: C)
+    assert lh.stats.steps == 256
+
+
+def _late_state(w, C, seed, n_rows, cur_pos, rng):
+    """A seeded cache state as it could look late in a generation: the text prefix, the local
+    window of cur_pos, and a random subset of the earlier image cells, n_rows rows in all."""
+    S, d = w.streams_per_layer, w.head_dim
+    g = cur_pos - w.n_text
+    r = g // w.grid_w
+    local = np.arange(w.n_text + max(0, r - 1) * w.grid_w, cur_pos)
+    older = np.arange(w.n_text, local[0]) if len(local) else np.arange(w.n_text, cur_pos)
+    n_old = n_rows - w.n_text - len(local)
+    assert 0 <= n_old <= len(older)
+    pos = np.empty((S, n_rows), dtype=np.int32)
+    for s in range(S):
+        pick = np.sort(rng.choice(older, size=n_old, replace=False))
+        row = np.concatenate([np.arange(w.n_text), pick, local])
+        pos[s] = row[rng.permutation(n_rows)]      # physical order is free: shuffle it
+    gen = np.random.Generator(np.random.Philox(key=[seed, 0xADA5]))
+    k = f32_to_bf16_bits(gen.standard_normal((w.batch, w.n_heads, n_rows, d), dtype=np.float32) * np.float32(w.sigma))
+    v = f32_to_bf16_bits(gen.standard_normal((w.batch, w.n_heads, n_rows, d), dtype=np.float32) * np.float32(w.sigma))
+    return pos, k, v
+
+
+@pytest.mark.parametrize("cfg,beta,n_sample,steps", [
+    (3, 0.5, 32, 3),
+    (4, 0.5, 32, 3),
+    (5, 0.25, 12, 2),
+    (5, 0.5, 8, 2),
+    (5, 0.75, 6, 2),
+])
+def test_full_size_layer_steps(cfg, beta, n_sample, steps):
+    """One layer at the full size of configs 3-5, in the launch configuration the benchmark
+    times, from a seeded late-generation state (cache full); the oracle follows a sample of streams."""
+    H = _harness()
+    w = get_workload(cfg, beta)
+    C = w.capacity()
+    rng = np.random.default_rng(cfg * 100 + int(beta * 100))
+    eng = H.engine_for(w, n_layers=1, capacity=C, page_rows=pick_page_rows(C, hi=128))
+    sample = sorted(rng.choice(w.streams_per_layer, size=n_sample, replace=False).tolist())
+    lh = H.LayerHarness(eng, 0, oracle_cap=C + 4, sample=sample)
+    g0 = w.n_cells - steps - w.grid_w // 2          # mid-row, near the end of the grid
+    cur0 = w.n_text + g0
+    pos, k, v = _late_state(w, C, seed=cfg, n_rows=C - 1, cur_pos=cur0, rng=rng)
+    lh.prefill(k, v, 0, pos)
+    lh.check_state()
+    for t in range(steps):
+        q, kn, vn = layer_step_qkv(w, 0, 0, g0 + t)
+        lh.step(q, kn, vn, cur0 + t, C)
+    st, fs = eng.get_status()
+    assert st == 0
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+    n_live = eng._t["n_live"].cpu().numpy()
+    assert (n_live == C).all()
+    # every page in use is accounted for, none leaked
+    pr = eng.cfg.page_rows
+    assert eng.cfg.n_pages - fs[2] == w.streams_per_layer * -(-C // pr)
+
+
+# ---------------------------------------------------------------------------
+# selection under structure: clusters, exact ties, equal and zero rows, any K
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("kind", ["clusters", "duplicates", "equal", "zeros", "iid"])
+def test_selection_on_structured_values(kind):
+    H = _harness()
+    T0, gh, gw, d = 4, 20, 16, 64
+    w = Workload("struct", 99, 1, 1, 6, d, T0, gh, gw, 0.5, 1.0)
+    n_rows = T0 + 250
+    cur = T0 + 18 * gw + 5                      # local window = 21 rows, the rest are candidates
+    for budget in (n_rows + 1, n_rows, n_rows - 1, 200, 120, T0 + 21 + 2, T0 + 21 + 1, 3):
+        eng = H.engine_for(w, capacity=n_rows + 1, page_rows=32)
+        lh = H.LayerHarness(eng, 0, oracle_cap=n_rows + 2)
+        rng = np.random.default_rng(5)
+        pos = np.stack([rng.permutation(np.concatenate([np.arange(T0), T0 + np.sort(rng.choice(cur - T0, n_rows - T0, replace=False))]))
+                        for _ in range(6)]).astype(np.int32)
+        v = np.stack([structured_values(kind, n_rows, d, seed=10 + s) for s in range(6)]).reshape(1, 6, n_rows, d)
+        k = np.stack([structured_values("iid", n_rows, d, seed=20 + s) for s in range(6)]).reshape(1, 6, n_rows, d)
+        lh.prefill(k, v, 0, pos)
+        q, kn, vn = layer_step_qkv(w, 0, 0, cur - T0)
+        lh.step(q, kn, vn, cur, budget)
+
+
+def test_repeat_runs_are_bit_identical():
+    outs = []
+    for _ in range(3):
+        w = get_workload(1)
+        lh, eng = _run_trajectory(w, 0, 0, lambda cur: w.capacity(), steps=160)
+        outs.append((lh.out_f32.cpu().numpy().copy(), np.sort(eng._t["pos"][:, :w.capacity()].cpu().numpy(), axis=1)))
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0]) and np.array_equal(o[1], outs[0][1])
+
+
+# ---------------------------------------------------------------------------
+# the one-call and host-buffer entry points agree with the four separate calls
+# ---------------------------------------------------------------------------
+def test_layer_step_and_host_variant_match_separate_calls():
+    H = _harness()
+    w = get_workload(1)
+    C = w.capacity()
+    engs = [H.engine_for(w, capacity=C) for _ in range(3)]
+    k, v = prefix_kv(w, 0, 0)
+    for e in engs:
+        e.prefill_rows(0, H.dev_bf16(k), H.dev_bf16(v), 0)
+    outs = [torch.zeros((w.streams_per_layer, w.head_dim), dtype=torch.bfloat16, device="cuda:0") for _ in range(2)]
+    out_h = torch.zeros((w.streams_per_layer, w.head_dim), dtype=torch.bfloat16).pin_memory()
+    for g in range(100):
+        qb, kb, vb = layer_step_qkv(w, 0, 0, g)
+        q, kn, vn = H.dev_bf16(qb), H.dev_bf16(kb), H.dev_bf16(vb)
+        cur = w.n_text + g
+        engs[0].score(0, cur)
+        engs[0].select(0, cur, C)
+        engs[0].sparse_decode_attn(0, cur, q, kn, vn, outs[0])
+        engs[0].kv_update(0, cur, kn, vn)
+        engs[1].layer_step(0, cur, C, q, kn, vn, outs[1])
+        hq, hk, hv = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in (qb, kb, vb))
+        engs[2].layer_step_host(0, cur, C, hq, hk, hv, out_h)
+        assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0].cpu(), out_h)
+    assert engs[0].launch_count() == engs[1].launch_count()
+
+
+def test_error_paths_return_status_and_launch_nothing():
+    import paper_2506_18226_b200 as A
+    H = _harness()
+    w = get_workload(1)
+    eng = H.engine_for(w, capacity=w.capacity())
+    before = eng.launch_count()
+    with pytest.raises(A.AdsaError) as e:
+        eng.select(0, 120, 50)                  # select before score
+    assert e.value.status == A.binding.ESTATE
+    eng.score(0, 120)
+    with pytest.raises(A.AdsaError) as e:
+        eng.select(0, 121, 50)                  # cur_pos changed inside a layer-step
+    assert e.value.status == A.binding.ESTATE
+    with pytest.raises(A.AdsaError) as e:
+        eng.score(7, 120)                       # no such layer
+    assert e.value.status == A.binding.EINVAL
+    assert eng.launch_count() == before + 1
+    # a pool that cannot hold the text condition is refused on the host
+    small = A.AdsaEngine(n_layers=1, batch=1, n_heads=12, head_dim=64, n_text=120, grid_h=16, grid_w=16,
+                         max_rows_per_stream=188, page_rows=47, n_pages=12 * 2)
+    k, v = prefix_kv(w, 0, 0)
+    with pytest.raises(A.AdsaError) as e:
+        small.prefill_rows(0, H.dev_bf16(k), H.dev_bf16(v), 0)
+    assert e.value.status == A.binding.ENOMEM
+    assert small.get_status()[0] == 0
