@@ -11,6 +11,7 @@ from .configs import CONFIGS, Workload, get_workload, pick_page_rows
 from .gen import (
     bf16_bits_to_f32,
     f32_to_bf16_bits,
+    late_state,
     layer_step_qkv,
     prefix_kv,
     structured_values,
@@ -23,6 +24,7 @@ __all__ = [
     "pick_page_rows",
     "bf16_bits_to_f32",
     "f32_to_bf16_bits",
+    "late_state",
     "layer_step_qkv",
     "prefix_kv",
     "structured_values",

@@ -104,3 +104,33 @@ def structured_values(kind: str, n_rows: int, head_dim: int, seed: int) -> np.nd
     else:
         raise ValueError(f"unknown kind {kind!r}")
     return f32_to_bf16_bits(x)
+
+
+def late_state(w: Workload, seed: int, n_rows: int, cur_pos: int, streams=None):
+    """A seeded cache state as it could look late in a generation, for every stream of one layer.
+
+    Each stream holds `n_rows` rows: the whole text condition, the 2*grid_w image cells just
+    before `cur_pos`, and a per-stream random subset of the older image cells; the physical row
+    order is shuffled (it is not part of the cache's meaning).  `streams` restricts the draw to
+    some stream indices (each stream's state depends only on (seed, stream)).
+    Returns pos int32 [S, n_rows], k and v uint16 [S, n_rows, head_dim].
+    """
+    d = w.head_dim
+    recent = np.arange(max(w.n_text, cur_pos - 2 * w.grid_w), cur_pos)
+    older = np.arange(w.n_text, recent[0]) if recent.size else np.arange(w.n_text, cur_pos)
+    n_old = n_rows - w.n_text - recent.size
+    if not 0 <= n_old <= older.size:
+        raise ValueError("n_rows does not fit between the mandatory rows and the context")
+    ids = list(range(w.streams_per_layer)) if streams is None else list(streams)
+    pos = np.empty((len(ids), n_rows), dtype=np.int32)
+    k = np.empty((len(ids), n_rows, d), dtype=np.uint16)
+    v = np.empty((len(ids), n_rows, d), dtype=np.uint16)
+    for i, s in enumerate(ids):
+        rng = np.random.Generator(np.random.Philox(key=[seed & 0xFFFFFFFFFFFFFFFF,
+                                                        (w.cfg_id << 56) | (_T_STRUCT << 48) | (1 << 40) | s]))
+        pick = rng.choice(older, size=n_old, replace=False)
+        row = np.concatenate([np.arange(w.n_text), pick, recent])
+        pos[i] = row[rng.permutation(n_rows)]
+        k[i] = _normal_bf16(rng, (n_rows, d), w.sigma)
+        v[i] = _normal_bf16(rng, (n_rows, d), w.sigma)
+    return pos, k, v

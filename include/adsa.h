@@ -180,6 +180,19 @@ ADSA_API int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_r
 ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q_host,
                          const void *k_new_host, const void *v_new_host, void *out_host, adsa_stream_t stream);
 
+/* One decoded token through every layer of an attention stack: adsa_layer_step
+ * for layer 0 .. n_layers-1 with the same cur_pos and budget.  q, k_new, v_new,
+ * out_bf16: [device] bf16 [n_layers][batch][n_heads][head_dim]. */
+ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                             const void *v_new, void *out_bf16, adsa_stream_t stream);
+
+/* adsa_token_step with HOST tensors of the same shapes: one host-to-device copy
+ * per input, all layers, one device-to-host copy of the outputs, then the
+ * stream is synchronised.  Uses the staging part of the workspace. */
+ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host,
+                                  const void *k_new_host, const void *v_new_host, void *out_host,
+                                  adsa_stream_t stream);
+
 /* How adsa_sparse_decode_attn would split a stream of n_rows cached rows:
  * number of chunks per stream and rows per chunk.  Pure host arithmetic. */
 ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);

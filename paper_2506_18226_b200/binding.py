@@ -21,7 +21,7 @@ DEV_POOL_EXHAUSTED, DEV_BAD_POSITION, DEV_ROW_OVERFLOW, DEV_RING_TIMEOUT, DEV_BA
 EXPORTS = [
     "adsa_workspace_bytes", "adsa_create", "adsa_destroy", "adsa_reset", "adsa_prefill_rows",
     "adsa_set_stream_rows", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
-    "adsa_layer_step", "adsa_layer_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows",
+    "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows",
     "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror",
 ]
 
@@ -67,6 +67,8 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_kv_update": [vp, i32, i32, vp, vp, vp],
             "adsa_layer_step": [vp, i32, i32, i32, vp, vp, vp, vp, vp],
             "adsa_layer_step_host": [vp, i32, i32, i32, vp, vp, vp, vp, vp],
+            "adsa_token_step": [vp, i32, i32, vp, vp, vp, vp, vp],
+            "adsa_token_step_host": [vp, i32, i32, vp, vp, vp, vp, vp],
             "adsa_plan_attn": [vp, i32, C.POINTER(i32), C.POINTER(i32)],
             "adsa_set_attn_chunk_rows": [vp, i32],
             "adsa_layer_rows_bound": [vp, i32, C.POINTER(i32)],
@@ -207,6 +209,19 @@ class AdsaEngine:
             if t.is_cuda:
                 raise ValueError("layer_step_host takes host tensors")
         self._call("adsa_layer_step_host", layer, cur_pos, budget_rows, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
+                   _stream())
+
+    def token_step(self, cur_pos, budget_rows, q, k_new, v_new, out_bf16):
+        """All layers of one token; tensors are [n_layers, batch, heads, head_dim] bf16 on the device."""
+        self._call("adsa_token_step", cur_pos, budget_rows, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out_bf16),
+                   _stream())
+
+    def token_step_host(self, cur_pos, budget_rows, q, k_new, v_new, out):
+        """token_step with HOST tensors (pinned for asynchronous copies).  Synchronises the stream."""
+        for t in (q, k_new, v_new, out):
+            if t.is_cuda:
+                raise ValueError("token_step_host takes host tensors")
+        self._call("adsa_token_step_host", cur_pos, budget_rows, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                    _stream())
 
     def plan_attn(self, n_rows):

@@ -44,7 +44,7 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.partials = off;    off = align_up(off + S * kMaxSplits * (size_t)(cfg.row_stride + 2) * sizeof(float), 256);
     w.tickets = off;     off = align_up(off + S * sizeof(int32_t), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
-    w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.head_dim * sizeof(__nv_bfloat16), 256);
+    w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
     return w;
 }
@@ -224,7 +224,7 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.rows_back = cfg->local_rows_back;
     float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
     d.scale_log2e = scale * 1.4426950408889634f;
-    size_t stage = (size_t)d.S * cfg->head_dim;
+    size_t stage = (size_t)d.S * cfg->n_layers * cfg->head_dim;
     ctx->stage_q = (__nv_bfloat16 *)(w + ws.staging);
     ctx->stage_k = ctx->stage_q + stage;
     ctx->stage_v = ctx->stage_k + stage;
@@ -380,6 +380,41 @@ int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows,
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_v, v_new_host, bytes, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     rc = adsa_layer_step(ctx, layer, cur_pos, budget_rows, ctx->stage_q, ctx->stage_k, ctx->stage_v, ctx->stage_o, stream);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(out_host, ctx->stage_o, bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return cuda_fail(ctx, e);
+}
+
+int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                    const void *v_new, void *out_bf16, adsa_stream_t stream)
+{
+    if (!ctx || !q || !k_new || !v_new || !out_bf16) return ADSA_EINVAL;
+    size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;
+    const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k_new,
+                        *vb = (const __nv_bfloat16 *)v_new;
+    __nv_bfloat16 *ob = (__nv_bfloat16 *)out_bf16;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+        int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
+                                 vb + l * per_layer, ob + l * per_layer, stream);
+        if (rc) return rc;
+    }
+    return ADSA_OK;
+}
+
+int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host, const void *k_new_host,
+                         const void *v_new_host, void *out_host, adsa_stream_t stream)
+{
+    if (!ctx) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return ADSA_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t bytes = (size_t)ctx->dev.S * ctx->cfg.n_layers * ctx->cfg.head_dim * sizeof(__nv_bfloat16);
+    cudaError_t e = cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_k, k_new_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_v, v_new_host, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    int rc = adsa_token_step(ctx, cur_pos, budget_rows, ctx->stage_q, ctx->stage_k, ctx->stage_v, ctx->stage_o, stream);
     if (rc) return rc;
     e = cudaMemcpyAsync(out_host, ctx->stage_o, bytes, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);

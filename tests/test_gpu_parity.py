@@ -3,8 +3,8 @@ import numpy as np
 import pytest
 import torch
 
-from adsa_workloads import (bf16_bits_to_f32, f32_to_bf16_bits, get_workload, layer_step_qkv, pick_page_rows,
-                            prefix_kv, structured_values)
+from adsa_workloads import (get_workload, late_state, layer_step_qkv, pick_page_rows, prefix_kv,
+                            structured_values)
 from adsa_workloads.configs import Workload
 
 pytestmark = pytest.mark.gpu
@@ -100,27 +100,6 @@ def test_config2_full_trajectory(layer):
     assert lh.stats.steps == 256
 
 
-def _late_state(w, C, seed, n_rows, cur_pos, rng):
-    """A seeded cache state as it could look late in a generation: the text prefix, the local
-    window of cur_pos, and a random subset of the earlier image cells, n_rows rows in all."""
-    S, d = w.streams_per_layer, w.head_dim
-    g = cur_pos - w.n_text
-    r = g // w.grid_w
-    local = np.arange(w.n_text + max(0, r - 1) * w.grid_w, cur_pos)
-    older = np.arange(w.n_text, local[0]) if len(local) else np.arange(w.n_text, cur_pos)
-    n_old = n_rows - w.n_text - len(local)
-    assert 0 <= n_old <= len(older)
-    pos = np.empty((S, n_rows), dtype=np.int32)
-    for s in range(S):
-        pick = np.sort(rng.choice(older, size=n_old, replace=False))
-        row = np.concatenate([np.arange(w.n_text), pick, local])
-        pos[s] = row[rng.permutation(n_rows)]      # physical order is free: shuffle it
-    gen = np.random.Generator(np.random.Philox(key=[seed, 0xADA5]))
-    k = f32_to_bf16_bits(gen.standard_normal((w.batch, w.n_heads, n_rows, d), dtype=np.float32) * np.float32(w.sigma))
-    v = f32_to_bf16_bits(gen.standard_normal((w.batch, w.n_heads, n_rows, d), dtype=np.float32) * np.float32(w.sigma))
-    return pos, k, v
-
-
 @pytest.mark.parametrize("cfg,beta,n_sample,steps", [
     (3, 0.5, 32, 3),
     (4, 0.5, 32, 3),
@@ -140,8 +119,8 @@ def test_full_size_layer_steps(cfg, beta, n_sample, steps):
     lh = H.LayerHarness(eng, 0, oracle_cap=C + 4, sample=sample)
     g0 = w.n_cells - steps - w.grid_w // 2          # mid-row, near the end of the grid
     cur0 = w.n_text + g0
-    pos, k, v = _late_state(w, C, seed=cfg, n_rows=C - 1, cur_pos=cur0, rng=rng)
-    lh.prefill(k, v, 0, pos)
+    pos, k, v = late_state(w, seed=cfg, n_rows=C - 1, cur_pos=cur0)
+    lh.prefill(k.reshape(w.batch, w.n_heads, C - 1, w.head_dim), v.reshape(w.batch, w.n_heads, C - 1, w.head_dim), 0, pos)
     lh.check_state()
     for t in range(steps):
         q, kn, vn = layer_step_qkv(w, 0, 0, g0 + t)
