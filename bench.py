@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--chunk-rows", type=int, default=0, help="override rows per attention chunk (0 = automatic)")
+    ap.add_argument("--profiler-range", action="store_true",
+                    help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
     return ap.parse_args()
 
 
@@ -216,6 +218,8 @@ def run_ours(args, rank, world, local_rank):
     sampler.start()
     launches0 = eng.launch_count()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.profiler_range:
+        torch.cuda.profiler.start()
     t0.record()
     g = first
     for _ in range(K):
@@ -226,6 +230,8 @@ def run_ours(args, rank, world, local_rank):
         g += 1
     t1.record()
     torch.cuda.synchronize(dev)
+    if args.profiler_range:
+        torch.cuda.profiler.stop()
     if world > 1:
         torch.distributed.barrier()
     ms_local = t0.elapsed_time(t1)
