@@ -211,6 +211,34 @@ ADSA_API int adsa_get_status(adsa_ctx *ctx, uint32_t *dev_status, int32_t free_s
 /* Number of kernels this context has launched so far (host counter). */
 ADSA_API int64_t adsa_launch_count(const adsa_ctx *ctx);
 
+/* Decode attention without a context, a workspace or any allocation (the paper has no counterpart:
+ * this exists for the integration, not for the method).  For callers that cannot allocate device
+ * memory where they need attention - a serving loop whose memory plan was frozen at start-up, a
+ * plugin interface that forbids the allocation calls, a process whose device memory belongs wholly
+ * to a framework's pool - and therefore cannot provide the workspace a context needs.
+ *
+ * out[s] = softmax_j(q[s].k_j * scale) . v_j over rows j = 0 .. n_rows[s]-1 of stream s and the new
+ * row (k_new[s], v_new[s]), fp32 arithmetic, the split reduction of adsa_sparse_decode_attn.
+ *   q, k_new, v_new   [device] bf16 [n_streams][head_dim]
+ *   k, v              [device] bf16 [n_streams][max_rows][row_stride], 16-byte aligned; row_stride >=
+ *                     head_dim, a multiple of 8, <= 256; elements past head_dim are ignored
+ *   n_rows            [device] int32 [n_streams], each clamped to 0 .. max_rows
+ *   out_bf16/out_f32  [device] [n_streams][head_dim]; either may be NULL, not both
+ *   softmax_scale     0 => 1/sqrt(head_dim)
+ * The scratch of the split reduction is a fixed 4 MiB array inside the library image: every GPU that
+ * loads the library holds it until the process exits.  Limits: n_streams <= 4096, max_rows <= 2^20
+ * (ADSA_ENOMEM beyond them; fewer chunks per stream are used when the partial states of more would
+ * not fit).  No cudaMalloc, cudaFree or allocating routine is called; the call only enqueues a
+ * counter clear and one kernel on `stream`.
+ * The first call on each device looks up the array's device address (that device must be current);
+ * make that first call before any stream capture begins.  All calls share the array and it keeps
+ * the previous call's contents, so calls whose kernels may overlap on the GPU (other streams, other
+ * host threads) race: serialise them. */
+ADSA_API int adsa_decode_attn_static(const void *q, const void *k, const void *v, const int32_t *n_rows,
+                                     const void *k_new, const void *v_new, int n_streams, int max_rows, int head_dim,
+                                     int row_stride, float softmax_scale, void *out_bf16, float *out_f32,
+                                     adsa_stream_t stream);
+
 ADSA_API const char *adsa_strerror(int status);
 
 #ifdef __cplusplus

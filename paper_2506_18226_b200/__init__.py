@@ -5,6 +5,7 @@ from .binding import (  # noqa: F401
     AdsaEngine,
     AdsaError,
     EXPORTS,
+    decode_attn_static,
     load,
     strerror,
     workspace_bytes,

@@ -22,7 +22,7 @@ EXPORTS = [
     "adsa_workspace_bytes", "adsa_create", "adsa_destroy", "adsa_reset", "adsa_prefill_rows",
     "adsa_set_stream_rows", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
     "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows",
-    "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror",
+    "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror", "adsa_decode_attn_static",
 ]
 
 
@@ -73,6 +73,7 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_set_attn_chunk_rows": [vp, i32],
             "adsa_layer_rows_bound": [vp, i32, C.POINTER(i32)],
             "adsa_get_status": [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_int32 * 4)],
+            "adsa_decode_attn_static": [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp],
         }
         for name, args in sig.items():
             fn = getattr(lib, name)
@@ -101,6 +102,23 @@ def _ptr(t):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def decode_attn_static(q, k, v, n_rows, k_new, v_new, out_bf16=None, out_f32=None, head_dim=None,
+                       softmax_scale=0.0):
+    """adsa_decode_attn_static: attention over dense rows with the library's built-in scratch.
+
+    For hosts that cannot allocate device memory when they need attention (frozen memory plan,
+    allocation calls forbidden, memory wholly owned by a pool): no context, no workspace, nothing
+    allocated.  k, v: [n_streams, max_rows, row_stride] bf16; q, k_new, v_new: [n_streams, head_dim];
+    n_rows: int32 [n_streams].  Calls must not overlap on the GPU (they share the scratch)."""
+    n_streams, max_rows, row_stride = k.shape
+    d = q.shape[-1] if head_dim is None else head_dim
+    rc = load().adsa_decode_attn_static(_ptr(q), _ptr(k), _ptr(v), _ptr(n_rows), _ptr(k_new), _ptr(v_new),
+                                        n_streams, max_rows, d, row_stride, softmax_scale, _ptr(out_bf16),
+                                        _ptr(out_f32), _stream())
+    if rc:
+        raise AdsaError(rc, "adsa_decode_attn_static")
 
 
 class AdsaEngine:
