@@ -197,6 +197,10 @@ ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, c
  * number of chunks per stream and rows per chunk.  Pure host arithmetic. */
 ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);
 
+/* 1 (default): attention and the layer-step use the staged cluster kernels whenever a stream fits a
+ * cluster's shared memory; 0: always the streaming kernels (four per layer-step).  Same results. */
+ADSA_API int adsa_set_staged(adsa_ctx *ctx, int enabled);
+
 /* Override the rows per attention chunk (0 = choose automatically). */
 ADSA_API int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows);
 

@@ -22,6 +22,7 @@ struct LayerState {
     int cur_pos = -1;
     int budget = 0;
     int rows_hi = 0;   // upper bound of n_live over the layer's streams
+    int scores_pos = -1;  // the carried scores (DevCtx::scores) are Eq. 2 for a step at this position; -1 = stale
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -37,7 +38,7 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     const size_t S = (size_t)cfg.batch * cfg.n_heads, R = (size_t)cfg.max_rows_per_stream;
     WorkspaceLayout w;
     size_t off = 0;
-    w.scores = off;      off = align_up(off + S * R * sizeof(float), 256);
+    w.scores = off;      off = align_up(off + S * (size_t)cfg.n_layers * R * sizeof(float), 256);
     w.keep_mask = off;   off = align_up(off + S * mask_words_of(cfg) * sizeof(uint32_t), 256);
     w.evict_slots = off; off = align_up(off + S * R * sizeof(int32_t), 256);
     w.counts = off;      off = align_up(off + S * 4 * sizeof(int32_t), 256);
@@ -85,6 +86,7 @@ struct adsa_ctx {
     std::vector<LayerState> layers;
     int sm_count = 148;
     int chunk_override = 0;
+    int no_staged = 0;   // 1: always use the streaming kernels (tests, comparisons)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -147,6 +149,13 @@ AttnPlan plan_attn(const adsa_ctx *ctx, int n_rows)
     p.n_splits = splits;
     p.chunk_rows = chunk;
     return p;
+}
+
+// The staged cluster kernel's plan for streams of up to n_rows rows (cluster_size 0: does not fit).
+StepPlan plan_staged(const adsa_ctx *ctx, int n_rows, bool fused)
+{
+    if (ctx->no_staged) { StepPlan none = {}; return none; }
+    return plan_step(ctx->dev, n_rows, fused, ctx->sm_count, ctx->chunk_override);
 }
 
 int check_layer(const adsa_ctx *ctx, int layer)
@@ -269,6 +278,7 @@ int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, co
     if (L.rows_hi + n_rows > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
     if (!pool_can_hold(ctx, layer, L.rows_hi + n_rows)) return ADSA_ENOMEM;
     L.rows_hi += n_rows;
+    L.scores_pos = -1;
     ++ctx->launches;
     return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
 }
@@ -286,6 +296,7 @@ int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, 
     int hi = n_rows > L.rows_hi ? n_rows : L.rows_hi;
     if (!pool_can_hold(ctx, layer, hi)) return ADSA_ENOMEM;
     L.rows_hi = hi;
+    L.scores_pos = -1;
     int sid = (layer * ctx->cfg.batch + b) * ctx->cfg.n_heads + h;
     ++ctx->launches;
     return cuda_fail(ctx, launch_set_rows(ctx->dev, sid, k, v, pos, n_rows, (cudaStream_t)stream));
@@ -300,6 +311,12 @@ int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_st
     if (L.phase != kIdle) return ADSA_ESTATE;
     L.phase = kScored;
     L.cur_pos = cur_pos;
+    if (L.scores_pos == cur_pos) {   // carried in from the previous fused step: nothing to compute
+        if (!scores_out) return ADSA_OK;
+        ++ctx->launches;
+        return cuda_fail(ctx, launch_scores_copy(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
+    }
+    L.scores_pos = cur_pos;
     ++ctx->launches;
     return cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
 }
@@ -334,8 +351,12 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
     LayerState &L = ctx->layers[layer];
     if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
     L.phase = kAttended;
-    AttnPlan plan = plan_attn(ctx, L.rows_hi);
     ++ctx->launches;
+    StepPlan sp = plan_staged(ctx, L.rows_hi, false);
+    if (sp.cluster_size)
+        return cuda_fail(ctx, launch_step(ctx->dev, sp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
+                                          (cudaStream_t)stream));
+    AttnPlan plan = plan_attn(ctx, L.rows_hi);
     return cuda_fail(ctx, launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32,
                                       (cudaStream_t)stream));
 }
@@ -351,6 +372,7 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
     int cap = L.budget > mand ? L.budget : mand;
     L.rows_hi = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
     L.phase = kIdle;
+    L.scores_pos = -1;   // rows move and the scores of the next step were not computed
     ++ctx->launches;
     return cuda_fail(ctx, launch_kv_update(ctx->dev, layer, cur_pos, k_new, v_new, (cudaStream_t)stream));
 }
@@ -358,13 +380,42 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
 int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q, const void *k_new,
                     const void *v_new, void *out_bf16, adsa_stream_t stream)
 {
-    int rc = adsa_score(ctx, layer, cur_pos, nullptr, stream);
+    int rc = check_layer(ctx, layer);
     if (rc) return rc;
-    rc = adsa_select(ctx, layer, cur_pos, budget_rows, nullptr, nullptr, nullptr, nullptr, stream);
-    if (rc) return rc;
-    rc = adsa_sparse_decode_attn(ctx, layer, cur_pos, q, k_new, v_new, out_bf16, nullptr, stream);
-    if (rc) return rc;
-    return adsa_kv_update(ctx, layer, cur_pos, k_new, v_new, stream);
+    if (!q || !k_new || !v_new || !out_bf16 || cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kIdle && !(L.phase == kScored && L.cur_pos == cur_pos)) return ADSA_ESTATE;
+    StepPlan sp = plan_staged(ctx, L.rows_hi, true);
+    if (!sp.cluster_size) {   // a stream this long does not fit a cluster's shared memory: four kernels
+        if (L.phase == kIdle) {
+            rc = adsa_score(ctx, layer, cur_pos, nullptr, stream);
+            if (rc) return rc;
+        }
+        rc = adsa_select(ctx, layer, cur_pos, budget_rows, nullptr, nullptr, nullptr, nullptr, stream);
+        if (rc) return rc;
+        rc = adsa_sparse_decode_attn(ctx, layer, cur_pos, q, k_new, v_new, out_bf16, nullptr, stream);
+        if (rc) return rc;
+        return adsa_kv_update(ctx, layer, cur_pos, k_new, v_new, stream);
+    }
+    // capacity checks of adsa_select, before anything is launched
+    int mand = mandatory_rows_bound(ctx, cur_pos) + 1;
+    int cap = budget_rows > mand ? budget_rows : mand;
+    int after = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
+    if (after > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+    if (!pool_can_hold(ctx, layer, after > L.rows_hi ? after : L.rows_hi)) return ADSA_ENOMEM;
+    if (L.phase == kIdle && L.scores_pos != cur_pos) {   // no scores carried in (first step, or the cache was rewritten)
+        ++ctx->launches;
+        rc = cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, nullptr, (cudaStream_t)stream));
+        if (rc) return rc;
+    }
+    ++ctx->launches;
+    rc = cuda_fail(ctx, launch_step(ctx->dev, sp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
+                                    (cudaStream_t)stream));
+    L.rows_hi = after;
+    L.phase = kIdle;
+    L.cur_pos = cur_pos;
+    L.scores_pos = cur_pos + 1;   // the fused kernel left the scores of the next position behind
+    return rc;
 }
 
 int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q_host,
@@ -424,6 +475,12 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
 int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows)
 {
     if (!ctx || n_rows < 0) return ADSA_EINVAL;
+    StepPlan sp = plan_staged(ctx, n_rows, false);
+    if (sp.cluster_size) {
+        if (n_splits) *n_splits = sp.cluster_size;
+        if (chunk_rows) *chunk_rows = sp.chunk_rows;
+        return ADSA_OK;
+    }
     AttnPlan p = plan_attn(ctx, n_rows);
     if (n_splits) *n_splits = p.n_splits;
     if (chunk_rows) *chunk_rows = p.chunk_rows;
@@ -434,6 +491,13 @@ int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows)
 {
     if (!ctx || chunk_rows < 0) return ADSA_EINVAL;
     ctx->chunk_override = chunk_rows;
+    return ADSA_OK;
+}
+
+int adsa_set_staged(adsa_ctx *ctx, int enabled)
+{
+    if (!ctx) return ADSA_EINVAL;
+    ctx->no_staged = enabled ? 0 : 1;
     return ADSA_OK;
 }
 
@@ -475,7 +539,8 @@ namespace adsa {
 cudaError_t configure_kernels(const DevCtx &c)
 {
     cudaError_t e = configure_select_kernel(c);
-    return e != cudaSuccess ? e : configure_update_kernel(c);
+    if (e == cudaSuccess) e = configure_update_kernel(c);
+    return e != cudaSuccess ? e : configure_step_kernel(c);
 }
 
 }  // namespace adsa

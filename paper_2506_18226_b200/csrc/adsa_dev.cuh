@@ -26,7 +26,7 @@ struct DevCtx {
     float *inv_norm;
     int32_t *free_ring, *free_state;
     // workspace (one layer's worth, reused by every layer)
-    float *scores;          // [S][max_rows]
+    float *scores;          // [n_layers * S][max_rows]  Eq. 2 scores by slot; carried from one step to the next
     uint32_t *keep_mask;    // [S][mask_words]   bit s = slot s is retained
     int32_t *evict_slots;   // [S][max_rows]     ascending
     int32_t *counts;        // [S][4]            p, evicted, retained, K
@@ -123,5 +123,47 @@ __device__ __forceinline__ float warp_sum(float x)
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
 }
+
+// ---- rows and pages --------------------------------------------------------
+// Bring the number of pages a stream holds from `have` to `need` (one thread).
+// Returns false if the pool ran dry.
+__device__ inline bool resize_pages(const DevCtx &c, int32_t *pt, int have, int need)
+{
+    for (int pg = have; pg < need; ++pg) {
+        int page = pool_pop(c);
+        if (page < 0) {
+            for (int q = have; q < pg; ++q) pool_push(c, pt[q]);  // give back what this call took
+            return false;
+        }
+        pt[pg] = page;
+    }
+    for (int pg = need; pg < have; ++pg) pool_push(c, pt[pg]);
+    return true;
+}
+
+// Write one cache row: bf16 payload (padding elements zeroed), position and the
+// inverse V norm.  One warp per row; src rows hold d elements.
+__device__ inline void write_row(const DevCtx &c, const int32_t *pt, int sid, int slot, const __nv_bfloat16 *ksrc,
+                          const __nv_bfloat16 *vsrc, int pos)
+{
+    int lane = threadIdx.x & 31;
+    size_t off = row_offset(c, pt, slot);
+    float ss = 0.f;
+    const __nv_bfloat16 zero = __float2bfloat16(0.f);
+    for (int e = lane; e < c.row_stride; e += 32) {
+        __nv_bfloat16 kk = e < c.d ? ksrc[e] : zero;
+        __nv_bfloat16 vv = e < c.d ? vsrc[e] : zero;
+        c.k_pool[off + e] = kk;
+        c.v_pool[off + e] = vv;
+        float f = __bfloat162float(vv);
+        ss = fmaf(f, f, ss);
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) {
+        c.pos[(size_t)sid * c.max_rows + slot] = pos;
+        c.inv_norm[(size_t)sid * c.max_rows + slot] = 1.0f / fmaxf(sqrtf(ss), kNormEps);
+    }
+}
+
 
 }  // namespace adsa

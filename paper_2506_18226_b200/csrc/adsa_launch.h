@@ -30,6 +30,23 @@ size_t select_smem_bytes(const DevCtx &c);
 cudaError_t launch_attn(const DevCtx &c, const AttnPlan &plan, int layer, int cur_pos, const void *q,
                         const void *k_new, const void *v_new, void *out_bf16, float *out_f32, cudaStream_t st);
 
+// The staged cluster kernel (attention alone, or the whole layer-step fused).
+constexpr int kStepMaxGroups = 64;             // copy groups (mbarriers) per CTA
+constexpr int kStepSmemLimit = 200 * 1024;     // dynamic shared memory a CTA may ask for
+
+struct StepPlan {
+    int cluster_size;   // CTAs per stream (1, 2, 4 or 8); 0 = the stream does not fit, use the streaming kernels
+    int chunk_rows;     // rows per CTA
+    int group_rows;     // rows per copy group
+    size_t smem_bytes;
+};
+StepPlan plan_step(const DevCtx &c, int n_rows, bool fused, int sm_count, int chunk_target);
+cudaError_t launch_step(const DevCtx &c, const StepPlan &plan, bool fused, int layer, int cur_pos, int budget_rows,
+                        const void *q, const void *k_new, const void *v_new, void *out_bf16, float *out_f32,
+                        cudaStream_t st);
+cudaError_t configure_step_kernel(const DevCtx &c);
+cudaError_t launch_scores_copy(const DevCtx &c, int layer, int cur_pos, float *scores_out, cudaStream_t st);
+
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t configure_kernels(const DevCtx &c);
 cudaError_t configure_select_kernel(const DevCtx &c);

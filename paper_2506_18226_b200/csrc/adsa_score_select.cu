@@ -6,6 +6,7 @@
 
 #include "adsa_dev.cuh"
 #include "adsa_launch.h"
+#include "adsa_select.cuh"
 
 namespace adsa {
 
@@ -36,7 +37,7 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
     const int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
     const int32_t *pos = c.pos + (size_t)sid * c.max_rows;
     const float *inv_norm = c.inv_norm + (size_t)sid * c.max_rows;
-    float *scores = c.scores + (size_t)local * c.max_rows;
+    float *scores = c.scores + (size_t)sid * c.max_rows;
     if (scores_out) scores_out += (size_t)local * c.max_rows;
     const int n = c.n_live[sid];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -49,7 +50,7 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
     int cnt = 0;
-    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {
+    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {   // no shuffles inside: lanes may leave early
         int reg = region_of(c, pos[slot], cur_pos);
         if (reg == kRegionInvalid && sub == 0) set_status(c, ADSA_DEV_BAD_POSITION);
         if (reg != kRegionPrevious) continue;
@@ -87,8 +88,9 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 #pragma unroll
     for (int e = 0; e < 8; ++e) sv[e] = piece_ok ? s_vec[sub * 8 + e] : 0.f;
 
-    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {
-        int reg = region_of(c, pos[slot], cur_pos);
+    for (int sb = warp * RPW; sb < n; sb += kSSWarps * RPW) {   // warp-uniform bounds: all lanes join the shuffles
+        const int slot = sb + grp;
+        int reg = slot < n ? region_of(c, pos[slot], cur_pos) : kRegionInvalid;
         float dot = 0.f, self = 0.f;
         if (reg == kRegionPrevious && piece_ok) {
             float f[8];
@@ -101,7 +103,7 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
             dot += __shfl_xor_sync(0xffffffffu, dot, o);
             self += __shfl_xor_sync(0xffffffffu, self, o);
         }
-        if (sub == 0) {
+        if (sub == 0 && slot < n) {
             float S = CUDART_NAN_F;
             if (reg == kRegionPrevious) {
                 float inv = inv_norm[slot];
@@ -116,123 +118,25 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 }
 
 // ---------------------------------------------------------------------------
-// Eq. 3.  Each row of the previous region gets the 64-bit key
-//   (order-preserving image of the float score) << 32 | position,
-// so "score ascending, then position ascending" is plain unsigned order and all
-// keys are distinct.  The K lowest keys are found without sorting:
-//   K >= p      keep all;   K == 0  drop all;
-//   K == p - 1  (steady state of Section 4.2, one eviction per step) drop the maximum key;
-//   otherwise   most-significant-digit-first radix select, 8 bits per pass,
-//               stopping as soon as the bin of the K-th key is taken whole.
-// The result is a threshold on a masked key: keep iff (key & mask) <= thr.
+// Eq. 3 plus the always-kept regions: the threshold comes from block_select, this
+// kernel turns it into the keep mask, the retained / evicted lists and the counts.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t orderable(float s)
-{
-    uint32_t u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 __global__ void __launch_bounds__(kSSThreads)
 select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_slots, int32_t *sel_pos,
               int32_t *evict_pos, int32_t *counts_out)
 {
     extern __shared__ unsigned long long sm_keys[];  // [max_rows], then uint8 region[max_rows]
-    __shared__ int s_cnt[3];                          // prefix, local, previous
-    __shared__ int s_hist[256];
-    __shared__ unsigned long long s_max;
-    __shared__ int s_digit, s_krem, s_bin;
+    __shared__ SelScratch s_sel;
     __shared__ int s_wk[kSSWarps], s_we[kSSWarps], s_bk, s_be;
     const int local = blockIdx.x, sid = layer * c.S + local;
     const int32_t *pos = c.pos + (size_t)sid * c.max_rows;
-    const float *scores = c.scores + (size_t)local * c.max_rows;
+    const float *scores = c.scores + (size_t)sid * c.max_rows;
     uint8_t *region = reinterpret_cast<uint8_t *>(sm_keys + c.max_rows);
     const int n = c.n_live[sid];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
-    if (threadIdx.x == 0) { s_max = 0ull; s_bk = 0; s_be = 0; }
-    __syncthreads();
-
-    // keys and region sizes
-    unsigned long long my_max = 0ull;
-    for (int base = 0; base < n; base += kSSThreads) {
-        int slot = base + threadIdx.x;
-        int reg = kRegionInvalid;
-        if (slot < n) {
-            int ps = pos[slot];
-            reg = region_of(c, ps, cur_pos);
-            region[slot] = (uint8_t)reg;
-            unsigned long long key = ~0ull;
-            if (reg == kRegionPrevious) {
-                key = ((unsigned long long)orderable(scores[slot]) << 32) | (uint32_t)ps;
-                my_max = key > my_max ? key : my_max;
-            }
-            sm_keys[slot] = key;
-        }
-#pragma unroll
-        for (int r = 0; r < 3; ++r) {
-            unsigned b = __ballot_sync(0xffffffffu, reg == r);
-            if (lane == 0 && b) atomicAdd(&s_cnt[r], __popc(b));
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long other = __shfl_xor_sync(0xffffffffu, my_max, o);
-        my_max = other > my_max ? other : my_max;
-    }
-    if (lane == 0) atomicMax(&s_max, my_max);
-    __syncthreads();
-    const int n_pre = s_cnt[kRegionPrefix], n_loc = s_cnt[kRegionLocal], p = s_cnt[kRegionPrevious];
-    int K = budget_rows - n_pre - n_loc - 1;
-    K = K < 0 ? 0 : (K > p ? p : K);
-
-    unsigned long long mask = 0ull, thr = 0ull;  // keep iff (key & mask) <= thr
-    bool drop_all = false;
-    if (K >= p) {
-        mask = 0ull; thr = 0ull;                 // every key passes
-    } else if (K == 0) {
-        drop_all = true;
-    } else if (K == p - 1) {
-        mask = ~0ull; thr = s_max - 1ull;        // keys are distinct: everything below the maximum
-    } else {
-        int k_rem = K;
-        for (int shift = 56; shift >= 0; shift -= 8) {
-            s_hist[threadIdx.x] = 0;             // kSSThreads == 256 bins
-            __syncthreads();
-            for (int slot = threadIdx.x; slot < n; slot += kSSThreads) {
-                unsigned long long key = sm_keys[slot];
-                if (region[slot] == kRegionPrevious && (key & mask) == thr)
-                    atomicAdd(&s_hist[(int)((key >> shift) & 255ull)], 1);
-            }
-            __syncthreads();
-            if (warp == 0) {                     // find the bin holding the k_rem-th key of the current prefix
-                int h[8], tot = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { h[i] = s_hist[lane * 8 + i]; tot += h[i]; }
-                int incl = tot;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    int t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                int excl = incl - tot;
-                if (excl < k_rem && k_rem <= incl) {
-                    int cum = excl;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        if (cum < k_rem && k_rem <= cum + h[i]) { s_digit = lane * 8 + i; s_krem = k_rem - cum; s_bin = h[i]; }
-                        cum += h[i];
-                    }
-                }
-            }
-            __syncthreads();
-            thr |= (unsigned long long)s_digit << shift;
-            mask |= 255ull << shift;
-            k_rem = s_krem;
-            int bin = s_bin;
-            __syncthreads();
-            if (k_rem == bin) break;             // the whole bin is kept: masked compare decides
-        }
-    }
+    if (threadIdx.x == 0) { s_bk = 0; s_be = 0; }
+    const SelResult sel = block_select(c, pos, scores, n, cur_pos, budget_rows, sm_keys, region, s_sel);
+    const int p = sel.p, K = sel.K;
 
     // retained / evicted lists in ascending slot order, keep mask, counts
     uint32_t *keep_mask = c.keep_mask + (size_t)local * c.mask_words;
@@ -242,8 +146,7 @@ select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_sl
         int slot = base + threadIdx.x;
         bool live = slot < n, kept = false;
         if (live) {
-            kept = region[slot] != kRegionPrevious || (!drop_all && (sm_keys[slot] & mask) <= thr);
-            if (region[slot] == kRegionInvalid) kept = true;  // flagged by adsa_score; never silently dropped
+            kept = sel.keeps(region[slot], sm_keys[slot]);
         }
         unsigned bk = __ballot_sync(0xffffffffu, kept), be = __ballot_sync(0xffffffffu, live && !kept);
         if (lane == 0) {
@@ -275,6 +178,25 @@ select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_sl
         if (counts_out) { counts_out[local * 4 + 0] = p; counts_out[local * 4 + 1] = s_be;
                           counts_out[local * 4 + 2] = s_bk; counts_out[local * 4 + 3] = K; }
     }
+}
+
+// Scores carried in from the previous fused step, laid out like adsa_score's optional output:
+// by slot, NaN outside the previous region.
+__global__ void scores_copy_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
+{
+    const int local = blockIdx.x, sid = layer * c.S + local;
+    const int n = c.n_live[sid];
+    for (int slot = threadIdx.x; slot < n; slot += blockDim.x) {
+        int reg = region_of(c, c.pos[(size_t)sid * c.max_rows + slot], cur_pos);
+        scores_out[(size_t)local * c.max_rows + slot] =
+            reg == kRegionPrevious ? c.scores[(size_t)sid * c.max_rows + slot] : CUDART_NAN_F;
+    }
+}
+
+cudaError_t launch_scores_copy(const DevCtx &c, int layer, int cur_pos, float *scores_out, cudaStream_t st)
+{
+    scores_copy_kernel<<<c.S, 256, 0, st>>>(c, layer, cur_pos, scores_out);
+    return cudaGetLastError();
 }
 
 // ---- host launchers -------------------------------------------------------

@@ -46,9 +46,12 @@ class Stats:
 class LayerHarness:
     """One layer of an engine next to an OracleStreams of the same streams."""
 
-    def __init__(self, eng: AdsaEngine, layer: int, oracle_cap: int, score_variant: int = 0, sample=None):
+    def __init__(self, eng: AdsaEngine, layer: int, oracle_cap: int, score_variant: int = 0, sample=None,
+                 fused: bool = False):
+        """fused=False drives the four calls one by one; fused=True drives adsa_layer_step (one fused
+        kernel carrying the scores from step to step) and reads the selection off the cache contents."""
         cfg = eng.cfg
-        self.eng, self.layer = eng, layer
+        self.eng, self.layer, self.fused = eng, layer, fused
         self.S, self.d = eng.S, cfg.head_dim
         # sample: the streams (indices within the layer) the oracle follows; None = all
         self.sample = list(range(self.S)) if sample is None else list(sample)
@@ -96,13 +99,19 @@ class LayerHarness:
         dev = eng.device
         q, kn, vn = dev_bf16(q_bits, dev), dev_bf16(k_bits, dev), dev_bf16(v_bits, dev)
         self.scores.fill_(float("nan"))
-        eng.score(L, cur_pos, self.scores)
-        eng.select(L, cur_pos, budget, self.sel_slots, self.sel_pos, self.evict_pos, self.counts)
+        eng.score(L, cur_pos, self.scores)           # fused: the scores carried in from the previous step
         sid0 = eng.stream_index(L, 0, 0)
         pos_before = eng._t["pos"][sid0:sid0 + S].cpu().numpy()
         n_before = eng._t["n_live"][sid0:sid0 + S].cpu().numpy()
-        eng.sparse_decode_attn(L, cur_pos, q, kn, vn, self.out_bf16, self.out_f32)
-        eng.kv_update(L, cur_pos, kn, vn)
+        if self.fused:
+            eng.layer_step(L, cur_pos, budget, q, kn, vn, self.out_bf16)
+            self.out_f32.copy_(self.out_bf16.float())
+            pos_after = eng._t["pos"][sid0:sid0 + S].cpu().numpy()
+            n_after = eng._t["n_live"][sid0:sid0 + S].cpu().numpy()
+        else:
+            eng.select(L, cur_pos, budget, self.sel_slots, self.sel_pos, self.evict_pos, self.counts)
+            eng.sparse_decode_attn(L, cur_pos, q, kn, vn, self.out_bf16, self.out_f32)
+            eng.kv_update(L, cur_pos, kn, vn)
 
         qf = bf16_bits_to_f32(q_bits).reshape(S, d)[self.sample]
         kf = bf16_bits_to_f32(k_bits).reshape(S, d)[self.sample]
@@ -122,7 +131,18 @@ class LayerHarness:
         for i, s in enumerate(self.sample):
             st.streams_checked += 1
             n = int(n_before[s])
-            p, n_ev, n_keep, K = (int(x) for x in counts[s])
+            if self.fused:
+                before = set(pos_before[s, :n].tolist())
+                after = pos_after[s, :int(n_after[s])].tolist()
+                assert len(set(after)) == len(after) and cur_pos in after, (cur_pos, s)
+                g_keep = set(after) - {cur_pos}
+                g_ev = before - g_keep
+                assert g_keep <= before, (cur_pos, s)
+                n_keep, n_ev = len(g_keep), len(g_ev)
+                p = int(np.count_nonzero(~np.isnan(scores[s, :n])))
+            else:
+                p, n_ev, n_keep, K = (int(x) for x in counts[s])
+                g_keep, g_ev = set(sel_pos[s, :n_keep].tolist()), set(evict_pos[s, :n_ev].tolist())
             assert n_keep + n_ev == n, (cur_pos, s, n_keep, n_ev, n)
             assert p == len(res.cand_pos[i]), (cur_pos, s, p, len(res.cand_pos[i]))
             # Eq. 2 scores, matched by position
@@ -133,7 +153,6 @@ class LayerHarness:
                 st.max_score_err = max(st.max_score_err, err)
                 assert err <= SCORE_ATOL, f"score mismatch {err} at pos {cur_pos} stream {s}"
             # Eq. 3 + always-kept regions: retained / evicted position sets
-            g_keep, g_ev = set(sel_pos[s, :n_keep].tolist()), set(evict_pos[s, :n_ev].tolist())
             o_keep, o_ev = set(res.kept_pos[i].tolist()), set(res.evict_pos[i].tolist())
             assert len(g_keep) == n_keep and len(g_ev) == n_ev
             assert g_keep | g_ev == o_keep | o_ev
@@ -159,7 +178,8 @@ class LayerHarness:
             step_err_n += e16.size
             assert e16.max() <= OUT_MAX_ABS, f"attention mismatch {e16.max()} at pos {cur_pos} stream {s}"
             scale = max(1.0, float(np.abs(res.out[i]).max()))
-            assert e32.max() <= OUT_F32_MAX_ABS * scale, f"fp32 attention mismatch {e32.max()} at pos {cur_pos} stream {s}"
+            assert self.fused or e32.max() <= OUT_F32_MAX_ABS * scale, \
+                f"fp32 attention mismatch {e32.max()} at pos {cur_pos} stream {s}"
         # the mean is taken over the output tensor of the call ([batch, heads, d]), as the max is
         assert step_err_sum <= OUT_MEAN_ABS * max(1, step_err_n), \
             f"mean attention error {step_err_sum / max(1, step_err_n)} at pos {cur_pos}"

@@ -74,18 +74,25 @@ def test_create_checks_buffers_and_workspace():
     assert A.load().adsa_create(C.byref(cfg), C.byref(buf), C.byref(ctx)) == B.EINVAL
 
 
-def test_attention_plan_covers_all_rows_with_whole_mask_words():
+def test_attention_plan_covers_all_rows():
     lib = A.load()
     for batch, heads in [(1, 12), (2, 12), (16, 16), (32, 20), (64, 32)]:
         rc, ctx = _fake_ctx(_cfg(batch=batch, n_heads=heads, max_rows_per_stream=2424, n_pages=1 << 20))
         assert rc == 0
+        s, ch = C.c_int(0), C.c_int(0)
         for n in (0, 1, 31, 32, 33, 187, 571, 1211, 2423):
-            s, ch = C.c_int(0), C.c_int(0)
+            # staged kernel: a cluster of 1, 2, 4 or 8 CTAs per stream, each with a chunk of whole 8-row units
+            assert lib.adsa_plan_attn(ctx, n, C.byref(s), C.byref(ch)) == 0
+            assert s.value in (1, 2, 4, 8) and ch.value % 8 == 0 and s.value * ch.value >= n
+            assert ch.value * 64 * 4 <= 200 * 1024               # K and V of a chunk fit in shared memory
+        assert lib.adsa_set_attn_chunk_rows(ctx, 300) == 0         # chunk target: 571 rows -> 2 CTAs of 288 rows
+        assert lib.adsa_plan_attn(ctx, 571, C.byref(s), C.byref(ch)) == 0 and (s.value, ch.value) == (2, 288)
+        assert lib.adsa_set_attn_chunk_rows(ctx, 0) == 0
+        assert lib.adsa_set_staged(ctx, 0) == 0                    # streaming kernel: up to 32 chunks of whole mask words
+        for n in (0, 1, 33, 571, 2423):
             assert lib.adsa_plan_attn(ctx, n, C.byref(s), C.byref(ch)) == 0
             assert 1 <= s.value <= 32 and ch.value % 32 == 0 and s.value * ch.value >= n
             assert (s.value - 1) * ch.value < max(n, 1)          # no empty chunk
-        assert lib.adsa_set_attn_chunk_rows(ctx, 50) == 0          # rounded up to 64
-        assert lib.adsa_plan_attn(ctx, 571, C.byref(s), C.byref(ch)) == 0 and ch.value == 64 and s.value == 9
         lib.adsa_destroy(ctx)
 
 
