@@ -196,6 +196,9 @@ step_kernel(DevCtx c, StepArgs a)
 
     // ---- which rows are attended ---------------------------------------------------------------
     int n2 = n, p_next = 0;
+    // With a window of the current grid row only, the new row itself is a candidate of the next step
+    // when that step starts a new grid row.
+    const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
     if constexpr (FUSED) {
         for (int r = c0 + tid; r < c1; r += kStepThreads) inv_s[r - c0] = inv_norm[r];
         const SelResult sel = block_select(c, pos, scores, n, a.cur_pos, a.budget_rows, sm_keys, region, s_sel);
@@ -216,7 +219,7 @@ step_kernel(DevCtx c, StepArgs a)
         for (int o = 16; o > 0; o >>= 1) my_pn += __shfl_xor_sync(0xffffffffu, my_pn, o);
         if (lane == 0 && my_pn) atomicAdd(&s_pnext, my_pn);
         __syncthreads();
-        p_next = s_pnext;
+        p_next = s_pnext + (new_cand ? 1 : 0);
     } else {
         const uint32_t *gmask = c.keep_mask + (size_t)local * c.mask_words;
         for (int w = tid; w * 32 < n; w += kStepThreads) kmask[w] = gmask[w];
@@ -245,10 +248,19 @@ step_kernel(DevCtx c, StepArgs a)
         }
 #pragma unroll
         for (int o = 1; o < LPR; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        float inv_new = 0.f;
+        if (new_cand) {
+            float ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(vf[e], vf[e], ss);
+#pragma unroll
+            for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            inv_new = 1.0f / fmaxf(sqrtf(ss), kNormEps);
+        }
         if (grp == 0) {
             m = s; l = 1.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = vf[e];
+            for (int e = 0; e < 8; ++e) { acc[e] = vf[e]; sn[e] = inv_new * vf[e]; }
         }
     }
 
@@ -470,6 +482,23 @@ step_kernel(DevCtx c, StepArgs a)
                 }
             }
             if (rank == 0) {
+                if (warp == 0 && new_cand) {   // the new row's own score for the next step
+                    float vf[8], dot = 0.f, ss = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        int x = sub * 8 + e;
+                        vf[e] = x < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + x]) : 0.f;
+                        dot = fmaf(vf[e], sv[e], dot);
+                        ss = fmaf(vf[e], vf[e], ss);
+                    }
+#pragma unroll
+                    for (int o = 1; o < LPR; o <<= 1) {
+                        dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                        ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    }
+                    float inv = 1.0f / fmaxf(sqrtf(ss), kNormEps);
+                    if (lane == 0) scores[holes[ns]] = p_next > 1 ? (inv * dot - inv * inv * ss) / denom + 0.0f : 0.0f;
+                }
                 if (warp == 0)
                     write_row(c, pt, sid, holes[ns], a.k_new + (size_t)local * c.d, a.v_new + (size_t)local * c.d, a.cur_pos);
                 if (tid == 32) {
