@@ -197,9 +197,17 @@ ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, c
  * number of chunks per stream and rows per chunk.  Pure host arithmetic. */
 ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);
 
-/* 1 (default): attention and the layer-step use the staged cluster kernels whenever a stream fits a
- * cluster's shared memory; 0: always the streaming kernels (four per layer-step).  Same results. */
-ADSA_API int adsa_set_staged(adsa_ctx *ctx, int enabled);
+/* Which kernels adsa_sparse_decode_attn and adsa_layer_step use.  Same results in every mode.
+ *   1 (default) automatic: the persistent pipelined kernel (one CTA per SM, a ring of K/V tiles kept
+ *               full by bulk copies); if its buffers do not fit shared memory, the cluster kernel; if a
+ *               stream does not fit a cluster either, the streaming kernels
+ *   0 streaming kernels only (register-streaming attention; four kernels per layer-step)
+ *   2 cluster kernel (one thread-block cluster per stream), else streaming
+ *   3 persistent kernel, else streaming */
+ADSA_API int adsa_set_staged(adsa_ctx *ctx, int mode);
+
+/* Cap the persistent kernel's ring at max_stages stages (0 = as many as fit; at least 3 are used). */
+ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
 
 /* Override the rows per attention chunk (0 = choose automatically). */
 ADSA_API int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows);

@@ -86,7 +86,8 @@ struct adsa_ctx {
     std::vector<LayerState> layers;
     int sm_count = 148;
     int chunk_override = 0;
-    int no_staged = 0;   // 1: always use the streaming kernels (tests, comparisons)
+    int kernel_mode = 1;   // adsa_set_staged: 0 streaming, 1 automatic, 2 cluster kernel, 3 persistent kernel
+    int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -154,8 +155,15 @@ AttnPlan plan_attn(const adsa_ctx *ctx, int n_rows)
 // The staged cluster kernel's plan for streams of up to n_rows rows (cluster_size 0: does not fit).
 StepPlan plan_staged(const adsa_ctx *ctx, int n_rows, bool fused)
 {
-    if (ctx->no_staged) { StepPlan none = {}; return none; }
+    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 3) { StepPlan none = {}; return none; }
     return plan_step(ctx->dev, n_rows, fused, ctx->sm_count, ctx->chunk_override);
+}
+
+// The persistent kernel's plan (n_stages 0: not used).
+PStepPlan plan_persistent(const adsa_ctx *ctx, bool fused)
+{
+    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 2) { PStepPlan none = {}; return none; }
+    return plan_pstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
 }
 
 int check_layer(const adsa_ctx *ctx, int layer)
@@ -352,6 +360,10 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
     if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
     L.phase = kAttended;
     ++ctx->launches;
+    PStepPlan pp = plan_persistent(ctx, false);
+    if (pp.n_stages)
+        return cuda_fail(ctx, launch_pstep(ctx->dev, pp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
+                                           (cudaStream_t)stream));
     StepPlan sp = plan_staged(ctx, L.rows_hi, false);
     if (sp.cluster_size)
         return cuda_fail(ctx, launch_step(ctx->dev, sp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
@@ -385,8 +397,10 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (!q || !k_new || !v_new || !out_bf16 || cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
     LayerState &L = ctx->layers[layer];
     if (L.phase != kIdle && !(L.phase == kScored && L.cur_pos == cur_pos)) return ADSA_ESTATE;
-    StepPlan sp = plan_staged(ctx, L.rows_hi, true);
-    if (!sp.cluster_size) {   // a stream this long does not fit a cluster's shared memory: four kernels
+    PStepPlan pp = plan_persistent(ctx, true);
+    StepPlan sp = {};
+    if (!pp.n_stages) sp = plan_staged(ctx, L.rows_hi, true);
+    if (!pp.n_stages && !sp.cluster_size) {   // neither staged kernel fits this configuration: four kernels
         if (L.phase == kIdle) {
             rc = adsa_score(ctx, layer, cur_pos, nullptr, stream);
             if (rc) return rc;
@@ -409,8 +423,12 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
         if (rc) return rc;
     }
     ++ctx->launches;
-    rc = cuda_fail(ctx, launch_step(ctx->dev, sp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
-                                    (cudaStream_t)stream));
+    if (pp.n_stages)
+        rc = cuda_fail(ctx, launch_pstep(ctx->dev, pp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
+                                         nullptr, (cudaStream_t)stream));
+    else
+        rc = cuda_fail(ctx, launch_step(ctx->dev, sp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
+                                        nullptr, (cudaStream_t)stream));
     L.rows_hi = after;
     L.phase = kIdle;
     L.cur_pos = cur_pos;
@@ -475,6 +493,12 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
 int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows)
 {
     if (!ctx || n_rows < 0) return ADSA_EINVAL;
+    PStepPlan pp = plan_persistent(ctx, false);
+    if (pp.n_stages) {   // one CTA walks the whole stream, tile by tile
+        if (n_splits) *n_splits = 1;
+        if (chunk_rows) *chunk_rows = pp.tile_rows;
+        return ADSA_OK;
+    }
     StepPlan sp = plan_staged(ctx, n_rows, false);
     if (sp.cluster_size) {
         if (n_splits) *n_splits = sp.cluster_size;
@@ -494,10 +518,17 @@ int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows)
     return ADSA_OK;
 }
 
-int adsa_set_staged(adsa_ctx *ctx, int enabled)
+int adsa_set_staged(adsa_ctx *ctx, int mode)
 {
-    if (!ctx) return ADSA_EINVAL;
-    ctx->no_staged = enabled ? 0 : 1;
+    if (!ctx || mode < 0 || mode > 3) return ADSA_EINVAL;
+    ctx->kernel_mode = mode;
+    return ADSA_OK;
+}
+
+int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages)
+{
+    if (!ctx || max_stages < 0) return ADSA_EINVAL;
+    ctx->max_stages = max_stages;
     return ADSA_OK;
 }
 
@@ -540,7 +571,8 @@ cudaError_t configure_kernels(const DevCtx &c)
 {
     cudaError_t e = configure_select_kernel(c);
     if (e == cudaSuccess) e = configure_update_kernel(c);
-    return e != cudaSuccess ? e : configure_step_kernel(c);
+    if (e == cudaSuccess) e = configure_step_kernel(c);
+    return e != cudaSuccess ? e : configure_pstep_kernel(c);
 }
 
 }  // namespace adsa

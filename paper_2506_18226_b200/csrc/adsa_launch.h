@@ -47,6 +47,22 @@ cudaError_t launch_step(const DevCtx &c, const StepPlan &plan, bool fused, int l
 cudaError_t configure_step_kernel(const DevCtx &c);
 cudaError_t launch_scores_copy(const DevCtx &c, int layer, int cur_pos, float *scores_out, cudaStream_t st);
 
+// The persistent pipelined kernel (attention alone, or the whole layer-step fused).
+constexpr int kPMaxStages = 24;                // ring stages (a K tile + a V tile each)
+constexpr int kPSmemLimit = 220 * 1024;        // dynamic shared memory of the one CTA per SM
+
+struct PStepPlan {
+    int n_stages;       // 0 = the configuration does not fit
+    int grid;           // CTAs (at most one per SM)
+    int tile_rows;
+    size_t smem_bytes;
+};
+PStepPlan plan_pstep(const DevCtx &c, bool fused, int sm_count, int max_stages);
+cudaError_t launch_pstep(const DevCtx &c, const PStepPlan &plan, bool fused, int layer, int cur_pos, int budget_rows,
+                         const void *q, const void *k_new, const void *v_new, void *out_bf16, float *out_f32,
+                         cudaStream_t st);
+cudaError_t configure_pstep_kernel(const DevCtx &c);
+
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t configure_kernels(const DevCtx &c);
 cudaError_t configure_select_kernel(const DevCtx &c);

@@ -43,8 +43,14 @@ struct SelResult {
     }
 };
 
+// Barrier the selecting threads meet at: the whole block, or (persistent kernel) the 256 consumer
+// threads alone on a named barrier while the copy-issuing warp runs on.
+struct BlockSync { static __device__ __forceinline__ void sync() { __syncthreads(); } };
+struct ConsumerSync { static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); } };
+
 // Fills sm_keys[0..n) and region[0..n) (region id in bits 0-1, kCandNextBit) and returns the
-// threshold.  Must be called by all kSelThreads threads of the block.
+// threshold.  Must be called by kSelThreads threads with threadIdx.x = 0 .. kSelThreads-1.
+template <class Sync = BlockSync>
 __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restrict__ pos,
                                          const float *__restrict__ scores, int n, int cur_pos, int budget_rows,
                                          unsigned long long *sm_keys, uint8_t *region, SelScratch &s)
@@ -52,7 +58,7 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x < 3) s.cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) s.max_key = 0ull;
-    __syncthreads();
+    Sync::sync();
 
     unsigned long long my_max = 0ull;
     for (int base = 0; base < n; base += kSelThreads) {
@@ -83,7 +89,7 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
         my_max = other > my_max ? other : my_max;
     }
     if (lane == 0) atomicMax(&s.max_key, my_max);
-    __syncthreads();
+    Sync::sync();
 
     SelResult r;
     r.n_pre = s.cnt[kRegionPrefix]; r.n_loc = s.cnt[kRegionLocal]; r.p = s.cnt[kRegionPrevious];
@@ -101,13 +107,13 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
         int k_rem = K;
         for (int shift = 56; shift >= 0; shift -= 8) {
             s.hist[threadIdx.x] = 0;
-            __syncthreads();
+            Sync::sync();
             for (int slot = threadIdx.x; slot < n; slot += kSelThreads) {
                 unsigned long long key = sm_keys[slot];
                 if ((region[slot] & 3) == kRegionPrevious && (key & mask) == thr)
                     atomicAdd(&s.hist[(int)((key >> shift) & 255ull)], 1);
             }
-            __syncthreads();
+            Sync::sync();
             if (warp == 0) {                     // find the bin holding the k_rem-th key of the current prefix
                 int h[8], tot = 0;
 #pragma unroll
@@ -128,12 +134,12 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
                     }
                 }
             }
-            __syncthreads();
+            Sync::sync();
             thr |= (unsigned long long)s.digit << shift;
             mask |= 255ull << shift;
             k_rem = s.krem;
             int bin = s.bin;
-            __syncthreads();
+            Sync::sync();
             if (k_rem == bin) break;             // the whole bin is kept: masked compare decides
         }
         r.mask = mask; r.thr = thr;

@@ -80,8 +80,12 @@ def test_attention_plan_covers_all_rows():
         rc, ctx = _fake_ctx(_cfg(batch=batch, n_heads=heads, max_rows_per_stream=2424, n_pages=1 << 20))
         assert rc == 0
         s, ch = C.c_int(0), C.c_int(0)
+        for n in (0, 571, 2423):
+            # persistent kernel (the default): one CTA walks the whole stream in tiles of 64 rows (head_dim 64)
+            assert lib.adsa_plan_attn(ctx, n, C.byref(s), C.byref(ch)) == 0 and (s.value, ch.value) == (1, 64)
+        assert lib.adsa_set_staged(ctx, 2) == 0
         for n in (0, 1, 31, 32, 33, 187, 571, 1211, 2423):
-            # staged kernel: a cluster of 1, 2, 4 or 8 CTAs per stream, each with a chunk of whole 8-row units
+            # cluster kernel: a cluster of 1, 2, 4 or 8 CTAs per stream, each with a chunk of whole 8-row units
             assert lib.adsa_plan_attn(ctx, n, C.byref(s), C.byref(ch)) == 0
             assert s.value in (1, 2, 4, 8) and ch.value % 8 == 0 and s.value * ch.value >= n
             assert ch.value * 64 * 4 <= 200 * 1024               # K and V of a chunk fit in shared memory

@@ -15,16 +15,19 @@ def _harness():
     return harness
 
 
-MODES = ["calls", "fused", "streaming"]
-# calls: the four C-ABI calls one by one (attention by the staged cluster kernel);
-# fused: adsa_layer_step, one kernel per layer-step with the scores carried from step to step;
-# streaming: the four calls with the staged kernels switched off (the register-streaming attention).
+MODES = ["calls", "fused", "streaming", "cluster-calls", "cluster-fused"]
+# calls: the four C-ABI calls one by one (attention by the persistent pipelined kernel);
+# fused: adsa_layer_step, one persistent kernel per layer-step, scores carried from step to step;
+# streaming: the four calls with the staged kernels switched off (the register-streaming attention);
+# cluster-*: the same two ways of calling, with the one-cluster-per-stream kernel.
 
 
 def _apply_mode(eng, mode):
     if mode == "streaming":
-        eng.set_staged(False)
-    return mode == "fused"
+        eng.set_staged(0)
+    elif mode.startswith("cluster"):
+        eng.set_staged(2)
+    return mode.endswith("fused")
 
 
 def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=None, steps=None, n_prefix=None,
@@ -69,7 +72,7 @@ def test_small_shapes_full_trajectory(d, page_rows, T0, gh, gw, beta, chunk, mod
 
 
 @pytest.mark.parametrize("n_prefix_kind,rows_back", [("none", 1), ("text+5%", 1), ("text", 2), ("text", 0)])
-@pytest.mark.parametrize("mode", ["calls", "fused"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "cluster-fused"])
 def test_prefix_and_window_variants(n_prefix_kind, rows_back, mode):
     w = Workload("tiny-variants", 97, 1, 1, 4, 64, 10, 8, 8, 0.5, 1.0)
     n_prefix = {"none": 0, "text": w.n_text, "text+5%": w.n_text + 4}[n_prefix_kind]
@@ -125,7 +128,7 @@ def test_config2_full_trajectory(layer, mode):
     (5, 0.5, 8, 2),
     (5, 0.75, 6, 2),
 ])
-@pytest.mark.parametrize("mode", ["calls", "fused"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "cluster-fused"])
 def test_full_size_layer_steps(cfg, beta, n_sample, steps, mode):
     """One layer at the full size of configs 3-5, in the launch configuration the benchmark
     times, from a seeded late-generation state (cache full); the oracle follows a sample of streams."""
@@ -158,7 +161,7 @@ def test_full_size_layer_steps(cfg, beta, n_sample, steps, mode):
 # selection under structure: clusters, exact ties, equal and zero rows, any K
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("kind", ["clusters", "duplicates", "equal", "zeros", "iid"])
-@pytest.mark.parametrize("mode", ["calls", "fused"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "cluster-fused"])
 def test_selection_on_structured_values(kind, mode):
     H = _harness()
     T0, gh, gw, d = 4, 20, 16, 64
