@@ -199,11 +199,13 @@ ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int 
 
 /* Which kernels adsa_sparse_decode_attn and adsa_layer_step use.  Same results in every mode.
  *   1 (default) automatic: the persistent pipelined kernel (one CTA per SM, a ring of K/V tiles kept
- *               full by bulk copies); if its buffers do not fit shared memory, the cluster kernel; if a
- *               stream does not fit a cluster either, the streaming kernels
+ *               full by asynchronous copies), with tensor-core arithmetic when pool rows are 64
+ *               elements wide, else on the CUDA cores; if its buffers do not fit shared memory, the
+ *               cluster kernel; if a stream does not fit a cluster either, the streaming kernels
  *   0 streaming kernels only (register-streaming attention; four kernels per layer-step)
  *   2 cluster kernel (one thread-block cluster per stream), else streaming
- *   3 persistent kernel, else streaming */
+ *   3 persistent kernel on the CUDA cores, else streaming
+ *   4 persistent kernel with tensor-core arithmetic, else streaming */
 ADSA_API int adsa_set_staged(adsa_ctx *ctx, int mode);
 
 /* Cap the persistent kernel's ring at max_stages stages (0 = as many as fit; at least 3 are used). */

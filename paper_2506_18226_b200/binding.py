@@ -253,7 +253,7 @@ class AdsaEngine:
         self._call("adsa_set_attn_chunk_rows", chunk_rows)
 
     def set_staged(self, mode):
-        """0 streaming kernels, 1 automatic, 2 cluster kernel, 3 persistent kernel."""
+        """0 streaming kernels, 1 automatic, 2 cluster kernel, 3 persistent (CUDA cores), 4 persistent (MMA)."""
         self._call("adsa_set_staged", int(mode))
 
     def set_ring_stages(self, max_stages):

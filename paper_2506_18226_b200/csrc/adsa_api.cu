@@ -86,7 +86,9 @@ struct adsa_ctx {
     std::vector<LayerState> layers;
     int sm_count = 148;
     int chunk_override = 0;
-    int kernel_mode = 1;   // adsa_set_staged: 0 streaming, 1 automatic, 2 cluster kernel, 3 persistent kernel
+    int kernel_mode = 1;   // adsa_set_staged: 0 streaming, 1 automatic, 2 cluster, 3 persistent (CUDA cores), 4 persistent (MMA)
+    int mma_ok = 0;        // tensor maps of the pools exist: the MMA kernel may run
+    MStepMaps maps;
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
@@ -159,11 +161,27 @@ StepPlan plan_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     return plan_step(ctx->dev, n_rows, fused, ctx->sm_count, ctx->chunk_override);
 }
 
-// The persistent kernel's plan (n_stages 0: not used).
-PStepPlan plan_persistent(const adsa_ctx *ctx, bool fused)
+// The persistent kernels' plans (n_stages 0: not used).  *mma tells which of the two was planned.
+PStepPlan plan_persistent(const adsa_ctx *ctx, bool fused, bool *mma)
 {
-    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 2) { PStepPlan none = {}; return none; }
+    PStepPlan p = {};
+    *mma = false;
+    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 2) return p;
+    if (ctx->mma_ok && ctx->kernel_mode != 3) {
+        p = plan_mstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
+        if (p.n_stages) { *mma = true; return p; }
+    }
+    if (ctx->kernel_mode == 4) return p;
     return plan_pstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
+}
+
+cudaError_t launch_persistent(const adsa_ctx *ctx, const PStepPlan &pp, bool mma, bool fused, int layer, int cur_pos,
+                              int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
+                              float *out_f32, cudaStream_t st)
+{
+    if (mma)
+        return launch_mstep(ctx->dev, pp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
+    return launch_pstep(ctx->dev, pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
 }
 
 int check_layer(const adsa_ctx *ctx, int layer)
@@ -253,6 +271,10 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
         ctx->sm_count = sms;
         cudaError_t e = configure_kernels(d);
         if (e != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
+        if (mstep_supported(d) && build_mstep_maps(d, &ctx->maps) == 0) {
+            if (configure_mstep_kernel(d) != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
+            ctx->mma_ok = 1;
+        }
     } else {
         cudaGetLastError();  // no usable device: host-side planning still works, launches will fail
     }
@@ -360,10 +382,11 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
     if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
     L.phase = kAttended;
     ++ctx->launches;
-    PStepPlan pp = plan_persistent(ctx, false);
+    bool mma = false;
+    PStepPlan pp = plan_persistent(ctx, false, &mma);
     if (pp.n_stages)
-        return cuda_fail(ctx, launch_pstep(ctx->dev, pp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
-                                           (cudaStream_t)stream));
+        return cuda_fail(ctx, launch_persistent(ctx, pp, mma, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
+                                                (cudaStream_t)stream));
     StepPlan sp = plan_staged(ctx, L.rows_hi, false);
     if (sp.cluster_size)
         return cuda_fail(ctx, launch_step(ctx->dev, sp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
@@ -397,7 +420,8 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (!q || !k_new || !v_new || !out_bf16 || cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
     LayerState &L = ctx->layers[layer];
     if (L.phase != kIdle && !(L.phase == kScored && L.cur_pos == cur_pos)) return ADSA_ESTATE;
-    PStepPlan pp = plan_persistent(ctx, true);
+    bool mma = false;
+    PStepPlan pp = plan_persistent(ctx, true, &mma);
     StepPlan sp = {};
     if (!pp.n_stages) sp = plan_staged(ctx, L.rows_hi, true);
     if (!pp.n_stages && !sp.cluster_size) {   // neither staged kernel fits this configuration: four kernels
@@ -424,8 +448,8 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     }
     ++ctx->launches;
     if (pp.n_stages)
-        rc = cuda_fail(ctx, launch_pstep(ctx->dev, pp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
-                                         nullptr, (cudaStream_t)stream));
+        rc = cuda_fail(ctx, launch_persistent(ctx, pp, mma, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
+                                              nullptr, (cudaStream_t)stream));
     else
         rc = cuda_fail(ctx, launch_step(ctx->dev, sp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
                                         nullptr, (cudaStream_t)stream));
@@ -493,7 +517,8 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
 int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows)
 {
     if (!ctx || n_rows < 0) return ADSA_EINVAL;
-    PStepPlan pp = plan_persistent(ctx, false);
+    bool mma = false;
+    PStepPlan pp = plan_persistent(ctx, false, &mma);
     if (pp.n_stages) {   // one CTA walks the whole stream, tile by tile
         if (n_splits) *n_splits = 1;
         if (chunk_rows) *chunk_rows = pp.tile_rows;
@@ -520,7 +545,7 @@ int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows)
 
 int adsa_set_staged(adsa_ctx *ctx, int mode)
 {
-    if (!ctx || mode < 0 || mode > 3) return ADSA_EINVAL;
+    if (!ctx || mode < 0 || mode > 4) return ADSA_EINVAL;
     ctx->kernel_mode = mode;
     return ADSA_OK;
 }

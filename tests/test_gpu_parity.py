@@ -15,11 +15,13 @@ def _harness():
     return harness
 
 
-MODES = ["calls", "fused", "streaming", "cluster-calls", "cluster-fused"]
-# calls: the four C-ABI calls one by one (attention by the persistent pipelined kernel);
+MODES = ["calls", "fused", "streaming", "cluster-calls", "cluster-fused", "cores-calls", "cores-fused"]
+# calls: the four C-ABI calls one by one (attention by the persistent pipelined kernel, tensor-core
+#        arithmetic where the pool rows are 64 elements wide);
 # fused: adsa_layer_step, one persistent kernel per layer-step, scores carried from step to step;
 # streaming: the four calls with the staged kernels switched off (the register-streaming attention);
-# cluster-*: the same two ways of calling, with the one-cluster-per-stream kernel.
+# cluster-*: the same two ways of calling, with the one-cluster-per-stream kernel;
+# cores-*: the same, with the persistent kernel forced onto the CUDA cores.
 
 
 def _apply_mode(eng, mode):
@@ -27,6 +29,8 @@ def _apply_mode(eng, mode):
         eng.set_staged(0)
     elif mode.startswith("cluster"):
         eng.set_staged(2)
+    elif mode.startswith("cores"):
+        eng.set_staged(3)
     return mode.endswith("fused")
 
 
