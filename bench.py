@@ -55,6 +55,10 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--chunk-rows", type=int, default=0, help="override rows per attention chunk (0 = automatic)")
+    ap.add_argument("--page-rows", type=int, default=0, help="rows per pool page (0 = the largest divisor of the capacity up to 128)")
+    ap.add_argument("--kernel-mode", type=int, default=1,
+                    help="0 streaming, 1 automatic, 2 cluster, 3 persistent on CUDA cores, 4 persistent with MMA")
+    ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
     return ap.parse_args()
@@ -157,7 +161,7 @@ def run_ours(args, rank, world, local_rank):
     C, HW, T0, L = w.capacity(), w.n_cells, w.n_text, w.n_layers
     K = HW if args.steps is None else max(1, args.steps)
     W = max(3, args.warmup)
-    pr = pick_page_rows(C, hi=128)
+    pr = args.page_rows if args.page_rows else pick_page_rows(C, hi=128)
     pages_per_stream = -(-C // pr)
     eng = AdsaEngine(n_layers=L, batch=w.batch, n_heads=w.n_heads, head_dim=w.head_dim, n_text=T0, grid_h=w.grid_h,
                      grid_w=w.grid_w, max_rows_per_stream=max(C, T0 + 2 * w.grid_w), page_rows=pr,
@@ -165,6 +169,9 @@ def run_ours(args, rank, world, local_rank):
                      device=str(dev))
     if args.chunk_rows:
         eng.set_attn_chunk_rows(args.chunk_rows)
+    eng.set_staged(args.kernel_mode)
+    if args.ring_stages:
+        eng.set_ring_stages(args.ring_stages)
     (q, k, v), (pk, pv), ring = make_inputs(w, HW, dev, args.seed + 1000 * rank)
     out = torch.zeros((2, L, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
 

@@ -86,9 +86,9 @@ struct adsa_ctx {
     std::vector<LayerState> layers;
     int sm_count = 148;
     int chunk_override = 0;
-    int kernel_mode = 1;   // adsa_set_staged: 0 streaming, 1 automatic, 2 cluster, 3 persistent (CUDA cores), 4 persistent (MMA)
+    int kernel_mode = 1;   // adsa_set_staged: 0 streaming, 1 automatic, 2 cluster, 3 persistent (CUDA cores), 4 warp-per-stream (MMA)
     int mma_ok = 0;        // tensor maps of the pools exist: the MMA kernel may run
-    MStepMaps maps;
+    WStepMaps maps;
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
@@ -154,34 +154,41 @@ AttnPlan plan_attn(const adsa_ctx *ctx, int n_rows)
     return p;
 }
 
-// The staged cluster kernel's plan for streams of up to n_rows rows (cluster_size 0: does not fit).
-StepPlan plan_staged(const adsa_ctx *ctx, int n_rows, bool fused)
-{
-    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 3) { StepPlan none = {}; return none; }
-    return plan_step(ctx->dev, n_rows, fused, ctx->sm_count, ctx->chunk_override);
-}
+// Which of the staged kernels serves this context, in order of preference: the warp-per-stream MMA
+// kernel, the persistent CUDA-core kernel, the cluster kernel; none of them = the streaming kernels.
+struct StagedChoice {
+    WStepPlan wp;
+    PStepPlan pp;
+    StepPlan sp;
+    bool any() const { return wp.n_workers || pp.n_stages || sp.cluster_size; }
+};
 
-// The persistent kernels' plans (n_stages 0: not used).  *mma tells which of the two was planned.
-PStepPlan plan_persistent(const adsa_ctx *ctx, bool fused, bool *mma)
+StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
 {
-    PStepPlan p = {};
-    *mma = false;
-    if (ctx->kernel_mode == 0 || ctx->kernel_mode == 2) return p;
-    if (ctx->mma_ok && ctx->kernel_mode != 3) {
-        p = plan_mstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
-        if (p.n_stages) { *mma = true; return p; }
+    StagedChoice ch = {};
+    const int m = ctx->kernel_mode;
+    if (m == 0) return ch;
+    if ((m == 1 || m == 4) && ctx->mma_ok) {
+        ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
+        if (ch.wp.n_workers) return ch;
     }
-    if (ctx->kernel_mode == 4) return p;
-    return plan_pstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
+    if (m == 1 || m == 3) {
+        ch.pp = plan_pstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
+        if (ch.pp.n_stages) return ch;
+    }
+    if (m == 1 || m == 2) ch.sp = plan_step(ctx->dev, n_rows, fused, ctx->sm_count, ctx->chunk_override);
+    return ch;
 }
 
-cudaError_t launch_persistent(const adsa_ctx *ctx, const PStepPlan &pp, bool mma, bool fused, int layer, int cur_pos,
-                              int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                              float *out_f32, cudaStream_t st)
+cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fused, int layer, int cur_pos,
+                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
+                          float *out_f32, cudaStream_t st)
 {
-    if (mma)
-        return launch_mstep(ctx->dev, pp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
-    return launch_pstep(ctx->dev, pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
+    if (ch.wp.n_workers)
+        return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
+    if (ch.pp.n_stages)
+        return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
+    return launch_step(ctx->dev, ch.sp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
 }
 
 int check_layer(const adsa_ctx *ctx, int layer)
@@ -271,8 +278,8 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
         ctx->sm_count = sms;
         cudaError_t e = configure_kernels(d);
         if (e != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
-        if (mstep_supported(d) && build_mstep_maps(d, &ctx->maps) == 0) {
-            if (configure_mstep_kernel(d) != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
+        if (wstep_supported(d) && build_wstep_maps(d, &ctx->maps) == 0) {
+            if (configure_wstep_kernel(d) != cudaSuccess) { delete ctx; return ADSA_ECUDA; }
             ctx->mma_ok = 1;
         }
     } else {
@@ -382,15 +389,10 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
     if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
     L.phase = kAttended;
     ++ctx->launches;
-    bool mma = false;
-    PStepPlan pp = plan_persistent(ctx, false, &mma);
-    if (pp.n_stages)
-        return cuda_fail(ctx, launch_persistent(ctx, pp, mma, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
-                                                (cudaStream_t)stream));
-    StepPlan sp = plan_staged(ctx, L.rows_hi, false);
-    if (sp.cluster_size)
-        return cuda_fail(ctx, launch_step(ctx->dev, sp, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
-                                          (cudaStream_t)stream));
+    StagedChoice ch = choose_staged(ctx, L.rows_hi, false);
+    if (ch.any())
+        return cuda_fail(ctx, launch_staged(ctx, ch, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
+                                            (cudaStream_t)stream));
     AttnPlan plan = plan_attn(ctx, L.rows_hi);
     return cuda_fail(ctx, launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32,
                                       (cudaStream_t)stream));
@@ -420,11 +422,8 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (!q || !k_new || !v_new || !out_bf16 || cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
     LayerState &L = ctx->layers[layer];
     if (L.phase != kIdle && !(L.phase == kScored && L.cur_pos == cur_pos)) return ADSA_ESTATE;
-    bool mma = false;
-    PStepPlan pp = plan_persistent(ctx, true, &mma);
-    StepPlan sp = {};
-    if (!pp.n_stages) sp = plan_staged(ctx, L.rows_hi, true);
-    if (!pp.n_stages && !sp.cluster_size) {   // neither staged kernel fits this configuration: four kernels
+    StagedChoice ch = choose_staged(ctx, L.rows_hi, true);
+    if (!ch.any()) {   // no staged kernel fits this configuration: four kernels
         if (L.phase == kIdle) {
             rc = adsa_score(ctx, layer, cur_pos, nullptr, stream);
             if (rc) return rc;
@@ -447,12 +446,8 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
         if (rc) return rc;
     }
     ++ctx->launches;
-    if (pp.n_stages)
-        rc = cuda_fail(ctx, launch_persistent(ctx, pp, mma, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
-                                              nullptr, (cudaStream_t)stream));
-    else
-        rc = cuda_fail(ctx, launch_step(ctx->dev, sp, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16,
-                                        nullptr, (cudaStream_t)stream));
+    rc = cuda_fail(ctx, launch_staged(ctx, ch, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
+                                      (cudaStream_t)stream));
     L.rows_hi = after;
     L.phase = kIdle;
     L.cur_pos = cur_pos;
@@ -517,17 +512,15 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
 int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows)
 {
     if (!ctx || n_rows < 0) return ADSA_EINVAL;
-    bool mma = false;
-    PStepPlan pp = plan_persistent(ctx, false, &mma);
-    if (pp.n_stages) {   // one CTA walks the whole stream, tile by tile
+    StagedChoice ch = choose_staged(ctx, n_rows, false);
+    if (ch.wp.n_workers || ch.pp.n_stages) {   // one warp or one CTA walks the whole stream, tile by tile
         if (n_splits) *n_splits = 1;
-        if (chunk_rows) *chunk_rows = pp.tile_rows;
+        if (chunk_rows) *chunk_rows = ch.wp.n_workers ? 32 : ch.pp.tile_rows;
         return ADSA_OK;
     }
-    StepPlan sp = plan_staged(ctx, n_rows, false);
-    if (sp.cluster_size) {
-        if (n_splits) *n_splits = sp.cluster_size;
-        if (chunk_rows) *chunk_rows = sp.chunk_rows;
+    if (ch.sp.cluster_size) {
+        if (n_splits) *n_splits = ch.sp.cluster_size;
+        if (chunk_rows) *chunk_rows = ch.sp.chunk_rows;
         return ADSA_OK;
     }
     AttnPlan p = plan_attn(ctx, n_rows);

@@ -64,17 +64,23 @@ cudaError_t launch_pstep(const DevCtx &c, const PStepPlan &plan, bool fused, int
                          cudaStream_t st);
 cudaError_t configure_pstep_kernel(const DevCtx &c);
 
-// The persistent kernel with tensor-core arithmetic (pools with 64-element rows).
-struct MStepMaps {
+// The warp-per-stream kernel with tensor-core arithmetic (pools with 64-element rows).
+struct WStepMaps {
     CUtensorMap k[6], v[6];   // boxes of 1, 2, 4, 8, 16, 32 rows x 64 elements, 128-byte swizzle
 };
-bool mstep_supported(const DevCtx &c);
-int build_mstep_maps(const DevCtx &c, MStepMaps *out);   // 0 on success
-PStepPlan plan_mstep(const DevCtx &c, bool fused, int sm_count, int max_stages);
-cudaError_t launch_mstep(const DevCtx &c, const PStepPlan &plan, const MStepMaps &maps, bool fused, int layer, int cur_pos,
+struct WStepPlan {
+    int n_workers;      // warps per CTA, one stream each at a time; 0 = not supported / does not fit
+    int depth;          // tiles in flight per warp
+    int grid;
+    size_t smem_bytes;
+};
+bool wstep_supported(const DevCtx &c);
+int build_wstep_maps(const DevCtx &c, WStepMaps *out);   // 0 on success
+WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth);
+cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                          float *out_f32, cudaStream_t st);
-cudaError_t configure_mstep_kernel(const DevCtx &c);
+cudaError_t configure_wstep_kernel(const DevCtx &c);
 
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t configure_kernels(const DevCtx &c);

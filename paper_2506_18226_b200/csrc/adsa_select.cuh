@@ -147,4 +147,96 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
     return r;
 }
 
+// The same selection done by ONE warp (the warp-per-stream kernel): no block barrier, only
+// __syncwarp.  hist is 256 ints of the warp's own shared memory.  All 32 lanes must call it.
+__device__ inline SelResult warp_select(const DevCtx &c, const int32_t *pos, const float *scores, int n, int cur_pos,
+                                        int budget_rows, unsigned long long *sm_keys, uint8_t *region, int *hist)
+{
+    const int lane = threadIdx.x & 31;
+    int cnt[3] = {0, 0, 0};
+    unsigned long long my_max = 0ull;
+    for (int base = 0; base < n; base += 32) {
+        int slot = base + lane;
+        int reg = kRegionInvalid;
+        if (slot < n) {
+            int ps = pos[slot];
+            reg = region_of(c, ps, cur_pos);
+            uint8_t rb = (uint8_t)reg;
+            if (reg != kRegionInvalid && region_of(c, ps, cur_pos + 1) == kRegionPrevious) rb |= kCandNextBit;
+            region[slot] = rb;
+            unsigned long long key = ~0ull;
+            if (reg == kRegionPrevious) {
+                key = ((unsigned long long)orderable(scores[slot]) << 32) | (uint32_t)ps;
+                my_max = key > my_max ? key : my_max;
+            }
+            sm_keys[slot] = key;
+        }
+#pragma unroll
+        for (int r = 0; r < 3; ++r) cnt[r] += __popc(__ballot_sync(0xffffffffu, reg == r));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, my_max, o);
+        my_max = other > my_max ? other : my_max;
+    }
+    __syncwarp();
+    SelResult r;
+    r.n_pre = cnt[kRegionPrefix]; r.n_loc = cnt[kRegionLocal]; r.p = cnt[kRegionPrevious];
+    int K = budget_rows - r.n_pre - r.n_loc - 1;
+    K = K < 0 ? 0 : (K > r.p ? r.p : K);
+    r.K = K;
+    r.mask = 0ull; r.thr = 0ull; r.drop_all = false;
+    if (K >= r.p) {
+    } else if (K == 0) {
+        r.drop_all = true;
+    } else if (K == r.p - 1) {
+        r.mask = ~0ull; r.thr = my_max - 1ull;
+    } else {
+        unsigned long long mask = 0ull, thr = 0ull;
+        int k_rem = K;
+        for (int shift = 56; shift >= 0; shift -= 8) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) hist[lane * 8 + i] = 0;
+            __syncwarp();
+            for (int slot = lane; slot < n; slot += 32) {
+                unsigned long long key = sm_keys[slot];
+                if ((region[slot] & 3) == kRegionPrevious && (key & mask) == thr)
+                    atomicAdd(&hist[(int)((key >> shift) & 255ull)], 1);
+            }
+            __syncwarp();
+            int h[8], tot = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { h[i] = hist[lane * 8 + i]; tot += h[i]; }
+            int incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            int excl = incl - tot;
+            int digit = 0, krem = 0, bin = 0;
+            const bool mine = excl < k_rem && k_rem <= incl;   // exactly one lane holds the bin of the k_rem-th key
+            if (mine) {
+                int cum = excl;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (cum < k_rem && k_rem <= cum + h[i]) { digit = lane * 8 + i; krem = k_rem - cum; bin = h[i]; }
+                    cum += h[i];
+                }
+            }
+            const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+            digit = __shfl_sync(0xffffffffu, digit, src);
+            krem = __shfl_sync(0xffffffffu, krem, src);
+            bin = __shfl_sync(0xffffffffu, bin, src);
+            thr |= (unsigned long long)digit << shift;
+            mask |= 255ull << shift;
+            k_rem = krem;
+            __syncwarp();
+            if (k_rem == bin) break;
+        }
+        r.mask = mask; r.thr = thr;
+    }
+    return r;
+}
+
 }  // namespace adsa
