@@ -147,6 +147,30 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
     return r;
 }
 
+// Section 4.1 partition without a division per row: for a given current position the local window
+// is "pos >= lo", lo = first position of grid row (current row - rows_back), so a row's region is
+// two comparisons.  Equivalent to region_of.
+struct RegionCut {
+    int cur, lo;   // lo = INT_MAX when the current position is still inside the text condition
+};
+__device__ __forceinline__ RegionCut region_cut(const DevCtx &c, int cur_pos)
+{
+    RegionCut r;
+    r.cur = cur_pos;
+    r.lo = 0x7fffffff;
+    if (cur_pos >= c.n_text) {
+        int row = (cur_pos - c.n_text) / c.grid_w - c.rows_back;
+        r.lo = c.n_text + (row > 0 ? row : 0) * c.grid_w;
+    }
+    return r;
+}
+__device__ __forceinline__ int region_by_cut(const DevCtx &c, const RegionCut &k, int pos)
+{
+    if (pos < 0 || pos >= k.cur) return kRegionInvalid;
+    if (pos < c.n_prefix) return kRegionPrefix;
+    return pos >= k.lo ? kRegionLocal : kRegionPrevious;
+}
+
 // The same selection done by ONE warp (the warp-per-stream kernel): no block barrier, only
 // __syncwarp.  hist is 256 ints of the warp's own shared memory.  All 32 lanes must call it.
 __device__ inline SelResult warp_select(const DevCtx &c, const int32_t *pos, const float *scores, int n, int cur_pos,
@@ -155,14 +179,15 @@ __device__ inline SelResult warp_select(const DevCtx &c, const int32_t *pos, con
     const int lane = threadIdx.x & 31;
     int cnt[3] = {0, 0, 0};
     unsigned long long my_max = 0ull;
+    const RegionCut cut_now = region_cut(c, cur_pos), cut_next = region_cut(c, cur_pos + 1);
     for (int base = 0; base < n; base += 32) {
         int slot = base + lane;
         int reg = kRegionInvalid;
         if (slot < n) {
             int ps = pos[slot];
-            reg = region_of(c, ps, cur_pos);
+            reg = region_by_cut(c, cut_now, ps);
             uint8_t rb = (uint8_t)reg;
-            if (reg != kRegionInvalid && region_of(c, ps, cur_pos + 1) == kRegionPrevious) rb |= kCandNextBit;
+            if (reg != kRegionInvalid && region_by_cut(c, cut_next, ps) == kRegionPrevious) rb |= kCandNextBit;
             region[slot] = rb;
             unsigned long long key = ~0ull;
             if (reg == kRegionPrevious) {

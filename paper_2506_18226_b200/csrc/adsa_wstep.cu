@@ -63,7 +63,7 @@ constexpr int kWMaxDepth = 8;                     // stages per warp
 
 // Per-warp shared memory (offsets from the warp's base)
 struct WLayout {
-    uint32_t bars, hdr, pt, meta, keys, region, kmask, wsplit, hist, svec, stages;
+    uint32_t bars, hdr, pt, meta, keys, region, kmask, cmask, wsplit, hist, svec, stages;
     uint32_t meta_words, w_rows;
     uint32_t per_warp;
 };
@@ -82,6 +82,7 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     L.keys = off;   off += fused ? w_align((max_rows + 2) * 8, 16) : 0; // later reused: holes, survivors
     L.region = off; off += fused ? w_align(max_rows + kWTile, 16) : 0;
     L.kmask = off;  off += w_align((mask_words + 1) * 4, 16);
+    L.cmask = off;  off += fused ? w_align((mask_words + 1) * 4, 16) : 0;   // retained rows the next step scores
     L.w_rows = w_align(max_rows + kWTile, 32);
     L.wsplit = off; off += fused ? 3 * L.w_rows * 2 : 0;               // bf16 hi | mid | lo of the row weights
     L.hist = off;   off += fused ? 256 * 4 : 0;
@@ -121,6 +122,18 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// D = A * B (accumulator starts at zero)
+__device__ __forceinline__ void mma_bf16_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ float ex2(float x)   // 2^x, x <= 0 or -inf here
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 // two floats -> packed bf16x2 (lo in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
@@ -149,6 +162,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     unsigned long long *sm_keys = reinterpret_cast<unsigned long long *>(smem + L.keys);
     uint8_t *region = smem + L.region;
     uint32_t *kmask = reinterpret_cast<uint32_t *>(smem + L.kmask);
+    uint32_t *cmask = reinterpret_cast<uint32_t *>(smem + L.cmask);
     __nv_bfloat16 *wsplit = reinterpret_cast<__nv_bfloat16 *>(smem + L.wsplit);
     int *hist = reinterpret_cast<int *>(smem + L.hist);
     float *svec = reinterpret_cast<float *>(smem + L.svec);
@@ -169,6 +183,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     const int g = lane >> 2, t = lane & 3;          // MMA fragment coordinates
     const int mi = lane >> 3, lr = lane & 7;        // ldmatrix: matrix index, row within the matrix
     const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
+    // ldmatrix row addresses inside a tile.  Tile rows used by a lane are (multiple of 8) + lr, so the
+    // swizzle term is (chunk ^ lr) << 4 and every address is a per-lane base xor a small constant:
+    //   K, block nb, elements 0-31:   nb*1024 + k_off        (chunks mi);  elements 32-63: the same ^ 64
+    //   V / pass 2, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
+    const uint32_t k_off = (uint32_t)(lr * kWRowBytes + ((mi ^ lr) << 4));
+    const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
     const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
     int spin_limit = kCopySpinLimit;
     auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -230,6 +250,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const uint32_t bar = smem_u32(bars + stage);
             mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
             int r = r0;
+            {   // the common case: a whole tile inside one page is one box per pool
+                uint32_t pg = __umulhi((uint32_t)r0, c.pr_magic);
+                int in = r0 - (int)pg * c.page_rows;
+                if (r1 - r0 == kWTile && in + kWTile <= c.page_rows) {
+                    int y = pt_s[pg] * c.page_rows + in;
+                    if (pass == 0) tma_2d(kdst, &maps.k[5], 0, y, bar);
+                    tma_2d(vdst, &maps.v[5], 0, y, bar);
+                    r = r1;
+                }
+            }
             while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
                 uint32_t pg = __umulhi((uint32_t)r, c.pr_magic);
                 int in = r - (int)pg * c.page_rows;
@@ -274,9 +304,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 const bool kept = slot < n && sel.keeps(region[slot], sm_keys[slot]);
                 if (slot < n && (region[slot] & 3) == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
                 const unsigned bk = __ballot_sync(0xffffffffu, kept);
-                if (lane == 0) kmask[base >> 5] = bk;
                 const bool cand = kept && (region[slot] & kCandNextBit);
-                p_next += __popc(__ballot_sync(0xffffffffu, cand));
+                const unsigned bc = __ballot_sync(0xffffffffu, cand);
+                if (lane == 0) { kmask[base >> 5] = bk; cmask[base >> 5] = bc; }
+                p_next += __popc(bc);
                 // w = 1/|v| for the rows the next step scores, as three bf16 parts (24 bits)
                 float w = cand ? inv_s[slot] : 0.f;
                 __nv_bfloat16 h = __float2bfloat16_rn(w);
@@ -284,7 +315,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 __nv_bfloat16 md = __float2bfloat16_rn(r1);
                 __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(md));
                 wsplit[slot] = h; wsplit[L.w_rows + slot] = md; wsplit[2 * L.w_rows + slot] = lo;
-                if (slot >= n) region[slot] = 0;
             }
             p_next += new_cand ? 1 : 0;
         } else {
@@ -347,16 +377,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             wait(smem_u32(bars + stage), (consumed / D) & 1);
             const uint32_t kb = stages_u32 + stage * kWStageBytes, vb = kb + kWTileBytes;
             const int r0 = tl * kWTile;
-            const uint32_t kw = kmask[tl];
+            const uint32_t kw = kmask[tl] >> (2 * t);   // bit 8*nb + e: row 8*nb + 2t + e is retained
             float sc[4][4];
 #pragma unroll
             for (int nb = 0; nb < 4; ++nb) {   // S = q.K^T, blocks of 8 rows
-                sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
                 uint32_t kf0[4], kf1[4];
-                const int row = 8 * nb + lr;
-                ldsm_x4(kb + swz(row, mi), kf0);         // elements 0-31 of the 8 rows
-                ldsm_x4(kb + swz(row, 4 + mi), kf1);     // elements 32-63
-                mma_bf16(sc[nb], qa0[0], 0u, qa2[0], 0u, kf0[0], kf0[1]);
+                ldsm_x4(kb + nb * 1024 + k_off, kf0);          // elements 0-31 of the 8 rows
+                ldsm_x4(kb + nb * 1024 + (k_off ^ 64u), kf1);  // elements 32-63
+                mma_bf16_z(sc[nb], qa0[0], 0u, qa2[0], 0u, kf0[0], kf0[1]);
                 mma_bf16(sc[nb], qa0[1], 0u, qa2[1], 0u, kf0[2], kf0[3]);
                 mma_bf16(sc[nb], qa0[2], 0u, qa2[2], 0u, kf1[0], kf1[1]);
                 mma_bf16(sc[nb], qa0[3], 0u, qa2[3], 0u, kf1[2], kf1[3]);
@@ -367,7 +395,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             for (int nb = 0; nb < 4; ++nb) {
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    bool kept = (kw >> (8 * nb + 2 * t + e)) & 1u;
+                    bool kept = (kw >> (8 * nb + e)) & 1u;
                     x[nb][e] = kept ? sc[nb][e] * c.scale_log2e : -INFINITY;
                     mx = fmaxf(mx, x[nb][e]);
                 }
@@ -375,13 +403,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             const float m_new = fmaxf(m_run, mx);
-            const float corr = exp2f(m_run - m_new);
+            const float corr = ex2(m_run - m_new);
             m_run = m_new;
             float psum = 0.f;
 #pragma unroll
             for (int nb = 0; nb < 4; ++nb) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) { x[nb][e] = exp2f(x[nb][e] - m_new); psum += x[nb][e]; }
+                for (int e = 0; e < 2; ++e) { x[nb][e] = ex2(x[nb][e] - m_new); psum += x[nb][e]; }
             }
             l_run = fmaf(l_run, corr, psum);
             // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0
@@ -402,16 +430,18 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // O_tile = A'.V from zero, then folded into the running sums
             float ot[8][4];
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) ot[nb][0] = ot[nb][1] = ot[nb][2] = ot[nb][3] = 0.f;
+            for (int nbp = 0; nbp < 4; ++nbp) {
+                uint32_t vf[4];
+                ldsm_x4_t(vb + (v_off ^ (uint32_t)(nbp << 5)), vf);
+                mma_bf16_z(ot[2 * nbp], pa0[0], 0u, pa2[0], 0u, vf[0], vf[1]);
+                mma_bf16_z(ot[2 * nbp + 1], pa0[0], 0u, pa2[0], 0u, vf[2], vf[3]);
+            }
 #pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
-#pragma unroll
-                for (int nbp = 0; nbp < 4; ++nbp) {
-                    uint32_t vf[4];
-                    ldsm_x4_t(vb + swz(16 * ks + 8 * (mi & 1) + lr, 2 * nbp + (mi >> 1)), vf);
-                    mma_bf16(ot[2 * nbp], pa0[ks], 0u, pa2[ks], 0u, vf[0], vf[1]);
-                    mma_bf16(ot[2 * nbp + 1], pa0[ks], 0u, pa2[ks], 0u, vf[2], vf[3]);
-                }
+            for (int nbp = 0; nbp < 4; ++nbp) {
+                uint32_t vf[4];
+                ldsm_x4_t(vb + 2048 + (v_off ^ (uint32_t)(nbp << 5)), vf);
+                mma_bf16(ot[2 * nbp], pa0[1], 0u, pa2[1], 0u, vf[0], vf[1]);
+                mma_bf16(ot[2 * nbp + 1], pa0[1], 0u, pa2[1], 0u, vf[2], vf[3]);
             }
             release_and_refill();
             const float corr_row = g < 2 ? corr : 1.0f;     // the weight sums are not softmax-scaled
@@ -497,15 +527,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 const uint32_t vb = stages_u32 + stage * kWStageBytes + kWTileBytes;
                 const unsigned char *vtile = smem + L.stages + stage * kWStageBytes + kWTileBytes;
                 const int r0 = tl * kWTile;
+                const uint32_t cw = okay ? cmask[tl] : 0u;
                 float dt[2][4];
 #pragma unroll
                 for (int mbk = 0; mbk < 2; ++mbk) {
-                    dt[mbk][0] = dt[mbk][1] = dt[mbk][2] = dt[mbk][3] = 0.f;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         uint32_t af[4];
-                        ldsm_x4(vb + swz(16 * mbk + 8 * (mi & 1) + lr, 2 * ks + (mi >> 1)), af);
-                        mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                        ldsm_x4(vb + mbk * 2048 + (v_off ^ (uint32_t)(ks << 5)), af);
+                        if (ks == 0) mma_bf16_z(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                        else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                     }
                 }
 #pragma unroll
@@ -514,8 +545,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     for (int hh = 0; hh < 2; ++hh) {   // rows 16*mbk + 8*hh + g: columns 0, 1 in lane t = 0, column 2 in t = 1
                         float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
                         const int row = r0 + 16 * mbk + 8 * hh + g;
-                        const bool want = okay && t == 0 && ((kmask[tl] >> (16 * mbk + 8 * hh + g)) & 1u) &&
-                                          (region[row] & kCandNextBit);
+                        const bool want = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
                         if (want) {
                             float dot = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
                             float inv = inv_s[row], self = 1.0f;
