@@ -58,6 +58,7 @@ def parse_args():
     ap.add_argument("--page-rows", type=int, default=0, help="rows per pool page (0 = the largest divisor of the capacity up to 128)")
     ap.add_argument("--kernel-mode", type=int, default=1,
                     help="0 streaming, 1 automatic, 2 cluster, 3 persistent on CUDA cores, 4 persistent with MMA")
+    ap.add_argument("--stream-warps", type=int, default=0, help="warps per stream of the tensor-core kernel (0 = automatic)")
     ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
@@ -172,6 +173,8 @@ def run_ours(args, rank, world, local_rank):
     eng.set_staged(args.kernel_mode)
     if args.ring_stages:
         eng.set_ring_stages(args.ring_stages)
+    if args.stream_warps:
+        eng.set_stream_warps(args.stream_warps)
     (q, k, v), (pk, pv), ring = make_inputs(w, HW, dev, args.seed + 1000 * rank)
     out = torch.zeros((2, L, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
 

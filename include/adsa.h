@@ -198,18 +198,22 @@ ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, c
 ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);
 
 /* Which kernels adsa_sparse_decode_attn and adsa_layer_step use.  Same results in every mode.
- *   1 (default) automatic: when pool rows are 64 elements wide, the warp-per-stream kernel (every
- *               warp owns a stream, its own TMA tile ring, tensor-core arithmetic); else the
+ *   1 (default) automatic: when pool rows are 64 elements wide, the warp-group kernel (a few warps
+ *               own a stream, each with its own TMA tile ring; tensor-core arithmetic); else the
  *               persistent pipelined CUDA-core kernel (one CTA per SM, a producer warp feeding a
  *               ring of K/V tiles); if that does not fit shared memory, the cluster kernel; if a
  *               stream does not fit a cluster either, the streaming kernels
  *   0 streaming kernels only (register-streaming attention; four kernels per layer-step)
  *   2 cluster kernel (one thread-block cluster per stream), else streaming
  *   3 persistent CUDA-core kernel, else streaming
- *   4 warp-per-stream tensor-core kernel, else streaming */
+ *   4 warp-group tensor-core kernel, else streaming */
 ADSA_API int adsa_set_staged(adsa_ctx *ctx, int mode);
 
-/* Cap the tile ring (per CTA of the persistent kernel, per warp of the warp-per-stream kernel) at
+/* Warps that share a stream in the tensor-core kernel: 1 .. 4, or 0 = chosen from the number of
+ * streams per SM and the shared memory the configuration needs. */
+ADSA_API int adsa_set_stream_warps(adsa_ctx *ctx, int warps);
+
+/* Cap the tile ring (per CTA of the persistent kernel, per warp of the tensor-core kernel) at
  * max_stages stages (0 = as many as fit). */
 ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
 

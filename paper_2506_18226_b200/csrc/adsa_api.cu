@@ -90,6 +90,7 @@ struct adsa_ctx {
     int mma_ok = 0;        // tensor maps of the pools exist: the MMA kernel may run
     WStepMaps maps;
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
+    int stream_warps = 0;  // warps per stream of the warp-group kernel (0 = automatic)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -160,7 +161,7 @@ struct StagedChoice {
     WStepPlan wp;
     PStepPlan pp;
     StepPlan sp;
-    bool any() const { return wp.n_workers || pp.n_stages || sp.cluster_size; }
+    bool any() const { return wp.n_groups || pp.n_stages || sp.cluster_size; }
 };
 
 StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
@@ -169,8 +170,8 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     const int m = ctx->kernel_mode;
     if (m == 0) return ch;
     if ((m == 1 || m == 4) && ctx->mma_ok) {
-        ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
-        if (ch.wp.n_workers) return ch;
+        ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages, ctx->stream_warps);
+        if (ch.wp.n_groups) return ch;
     }
     if (m == 1 || m == 3) {
         ch.pp = plan_pstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages);
@@ -184,7 +185,7 @@ cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fuse
                           int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                           float *out_f32, cudaStream_t st)
 {
-    if (ch.wp.n_workers)
+    if (ch.wp.n_groups)
         return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
     if (ch.pp.n_stages)
         return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
@@ -513,9 +514,9 @@ int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_ro
 {
     if (!ctx || n_rows < 0) return ADSA_EINVAL;
     StagedChoice ch = choose_staged(ctx, n_rows, false);
-    if (ch.wp.n_workers || ch.pp.n_stages) {   // one warp or one CTA walks the whole stream, tile by tile
+    if (ch.wp.n_groups || ch.pp.n_stages) {   // one warp or one CTA walks the whole stream, tile by tile
         if (n_splits) *n_splits = 1;
-        if (chunk_rows) *chunk_rows = ch.wp.n_workers ? 32 : ch.pp.tile_rows;
+        if (chunk_rows) *chunk_rows = ch.wp.n_groups ? 32 : ch.pp.tile_rows;
         return ADSA_OK;
     }
     if (ch.sp.cluster_size) {
@@ -540,6 +541,13 @@ int adsa_set_staged(adsa_ctx *ctx, int mode)
 {
     if (!ctx || mode < 0 || mode > 4) return ADSA_EINVAL;
     ctx->kernel_mode = mode;
+    return ADSA_OK;
+}
+
+int adsa_set_stream_warps(adsa_ctx *ctx, int warps)
+{
+    if (!ctx || warps < 0 || warps > 4) return ADSA_EINVAL;
+    ctx->stream_warps = warps;
     return ADSA_OK;
 }
 

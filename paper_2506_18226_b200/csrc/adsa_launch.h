@@ -68,15 +68,17 @@ cudaError_t configure_pstep_kernel(const DevCtx &c);
 struct WStepMaps {
     CUtensorMap k[6], v[6];   // boxes of 1, 2, 4, 8, 16, 32 rows x 64 elements, 128-byte swizzle
 };
+constexpr int kWSmemLimit = 226 * 1024;        // dynamic shared memory of the one CTA per SM
 struct WStepPlan {
-    int n_workers;      // warps per CTA, one stream each at a time; 0 = not supported / does not fit
+    int n_groups;       // streams a CTA serves at a time; 0 = not supported / does not fit
+    int group_warps;    // warps that share a stream
     int depth;          // tiles in flight per warp
     int grid;
     size_t smem_bytes;
 };
 bool wstep_supported(const DevCtx &c);
 int build_wstep_maps(const DevCtx &c, WStepMaps *out);   // 0 on success
-WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth);
+WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps);
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                          float *out_f32, cudaStream_t st);

@@ -1,14 +1,16 @@
 // The warp-per-stream kernel with tensor-core arithmetic, for pools whose rows are
 // 64 elements (128 bytes) wide.  This is the kernel the benchmark's layer-step runs.
 //
-// Why one warp per stream.  A layer-step of one stream is a chain of short,
+// Why a few warps per stream.  A layer-step of one stream is a chain of short,
 // dependent phases (selection, attention sweep, reduction, score sweep, update).
-// Spread over a whole CTA each phase ends in a barrier and the SM idles on latency;
-// measured, a CTA-wide version spent 27 us per stream.  Here every warp is a
-// self-contained worker: it owns a stream from start to finish, keeps its own
-// metadata and its own small ring of tiles in shared memory, issues its own TMA
-// copies, and never waits for another warp.  Latency is hidden the way GPUs hide
-// it best, by the other warps of the SM being in different places of their chains.
+// Spread over a whole CTA each phase ends in a CTA barrier and the SM idles on
+// latency; measured, a CTA-wide version spent 27 us per stream.  Here a stream
+// belongs to a small group of warps (1 to 4, chosen so that the SM's streams fill
+// its warp slots): the tiles of the stream are dealt round-robin to the warps of the
+// group, each warp keeps its own ring of tiles in shared memory and issues its own
+// TMA copies, and the group meets only three times per stream (selection partials,
+// softmax partials, before the update) on a named barrier.  Latency is hidden the
+// way GPUs hide it best, by the other warps of the SM being elsewhere in their chains.
 //
 // Why tensor cores for a matrix-vector product.  One query per private KV stream is
 // 1 flop per byte, so arithmetic is no limit, but INSTRUCTIONS are: a B200 issues
@@ -27,9 +29,9 @@
 //
 // Pass 1, per tile:  S = q.K^T  (A = q in rows 0-7, B = K rows via ldmatrix);
 //   P = exp2(S*scale - m), split into bf16 hi + lo so the product keeps fp32-like
-//   accuracy;  O_tile = A'.V with A' rows {P_hi, P_lo, w_hi, w_mid, w_lo}, where
+//   accuracy;  O_tile = A'.V with A' rows {P_hi, P_lo, w_hi, w_lo}, where
 //   w_j = 1/|v_j| for the rows the next step will score and 0 otherwise: rows 0-1 of
-//   the result accumulate softmax.V, rows 2-4 accumulate s = sum of normalised rows.
+//   the result accumulate softmax.V, rows 2-3 accumulate s = sum of normalised rows.
 //   Each tile's product starts from zero and is folded into fp32 running sums with
 //   round-to-nearest FMAs, so tensor-core accumulation rounding never compounds
 //   beyond 32 rows.
@@ -38,8 +40,8 @@
 //   S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), Eq. 1-2 for the next step (u_i.u_i = 1
 //   unless |v_i| was clamped, in which case it is computed from the row).
 // Then the Section 4.2 update.  All rows of a stream are copied, retained or not
-// (one row per step is not); rows of a partial last tile that were not copied hold
-// older finite data and are masked; the ring is zeroed once at kernel start.
+// (one row per step is not); the rows of a partial last tile that the copy does not
+// write are cleared first, so that a zero weight never meets a NaN pattern.
 //
 // Every wait on a copy is bounded: if it runs out the warp raises
 // ADSA_DEV_COPY_TIMEOUT, shortens its later waits and runs to the end (all accesses
@@ -60,45 +62,7 @@ constexpr int kWRowBytes = 128;                   // 64 bf16
 constexpr int kWTileBytes = kWTile * kWRowBytes;  // one K (or V) tile
 constexpr int kWStageBytes = 2 * kWTileBytes;
 constexpr int kWMaxDepth = 8;                     // stages per warp
-
-// Per-warp shared memory (offsets from the warp's base)
-struct WLayout {
-    uint32_t bars, hdr, pt, meta, keys, region, kmask, cmask, wsplit, hist, svec, stages;
-    uint32_t meta_words, w_rows;
-    uint32_t per_warp;
-};
-
-__host__ __device__ inline uint32_t w_align(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
-
-__host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mask_words, int depth, bool fused)
-{
-    WLayout L;
-    uint32_t off = 0;
-    L.bars = off;   off += (kWMaxDepth + 2) * 8;
-    L.hdr = off;    off += 16;
-    L.pt = off;     off += w_align(max_pages * 4, 16);
-    L.meta_words = w_align(max_rows + 8, 4);
-    L.meta = off;   off += fused ? 3 * L.meta_words * 4 : 0;            // pos | carried scores | inverse norms
-    L.keys = off;   off += fused ? w_align((max_rows + 2) * 8, 16) : 0; // later reused: holes, survivors
-    L.region = off; off += fused ? w_align(max_rows + kWTile, 16) : 0;
-    L.kmask = off;  off += w_align((mask_words + 1) * 4, 16);
-    L.cmask = off;  off += fused ? w_align((mask_words + 1) * 4, 16) : 0;   // retained rows the next step scores
-    L.w_rows = w_align(max_rows + kWTile, 32);
-    L.wsplit = off; off += fused ? 3 * L.w_rows * 2 : 0;               // bf16 hi | mid | lo of the row weights
-    L.hist = off;   off += fused ? 256 * 4 : 0;
-    L.svec = off;   off += 64 * 4;
-    off = w_align(off, 1024);                                          // the swizzle pattern repeats every 1024 bytes
-    L.stages = off; off += depth * kWStageBytes;
-    L.per_warp = w_align(off, 1024);
-    return L;
-}
-
-struct WStepArgs {
-    int layer, cur_pos, budget_rows, depth, n_workers;   // n_workers = warps per CTA
-    const __nv_bfloat16 *q, *k_new, *v_new;
-    __nv_bfloat16 *out_bf16;
-    float *out_f32;
-};
+constexpr int kWMaxGroupWarps = 4;                // warps that may share a stream
 
 // ---- PTX wrappers ---------------------------------------------------------
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
@@ -109,23 +73,23 @@ __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap *map, int
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4])
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 // D += A(16x16, row) * B(16x8, col), bf16 in, fp32 accumulate
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // D = A * B (accumulator starts at zero)
 __device__ __forceinline__ void mma_bf16_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                  : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 __device__ __forceinline__ float ex2(float x)   // 2^x, x <= 0 or -inf here
@@ -146,39 +110,91 @@ __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p 
 // byte offset of 16-byte chunk c of row r inside a tile written with the 128-byte swizzle
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * kWRowBytes + ((c ^ (r & 7)) << 4)); }
 
-template <bool FUSED>
-__global__ void __launch_bounds__(256, 1)
+// Shared memory of one group (the G warps that share a stream): a fixed part, then one ring per warp.
+struct WLayout {
+    uint32_t bars, hdr, pt, inv, keys, prevm, candm, kmask, cmask, wsplit, hist, part, rings;
+    uint32_t inv_words, w_rows, mwords;
+    uint32_t ring_bytes;    // one warp's ring
+    uint32_t per_group;
+};
+
+__host__ __device__ inline uint32_t w_align(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
+
+__host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mask_words, int depth, int G, bool fused)
+{
+    WLayout L;
+    uint32_t off = 0;
+    L.bars = off;   off += (kWMaxGroupWarps * kWMaxDepth + 2) * 8;       // tile barriers per warp, then the metadata barrier
+    L.hdr = off;    off += kWMaxGroupWarps * 32 + 32;                     // per-warp selection partials, then the threshold
+    L.pt = off;     off += w_align(max_pages * 4, 16);
+    L.inv_words = w_align(max_rows + 8, 4);
+    L.inv = off;    off += fused ? L.inv_words * 4 : 0;                   // inverse norms by slot
+    L.keys = off;   off += fused ? w_align((max_rows + 2) * 8, 16) : 0;   // later reused: holes, survivors
+    L.mwords = mask_words + 1;
+    L.prevm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows of the previous region
+    L.candm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows in the previous region of the next step
+    L.kmask = off;  off += w_align(L.mwords * 4, 16);                     // retained rows
+    L.cmask = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // retained rows the next step scores
+    L.w_rows = w_align(max_rows + kWTile, 32);
+    L.wsplit = off; off += fused ? 2 * L.w_rows * 2 : 0;                  // bf16 hi | lo of the row weights
+    L.part = off;   off += kWMaxGroupWarps * 132 * 4;                     // per warp: acc[64] | s[64] | m, l
+    L.hist = L.part;                                                      // radix histogram: used before any partial state exists
+    off = w_align(off, 1024);                                             // the swizzle pattern repeats every 1024 bytes
+    L.rings = off;
+    L.ring_bytes = depth * kWStageBytes;
+    L.per_group = off + G * L.ring_bytes;
+    return L;
+}
+
+struct WStepArgs {
+    int layer, cur_pos, budget_rows, depth;
+    int group_warps, n_groups;   // warps per stream, groups per CTA
+    const __nv_bfloat16 *q, *k_new, *v_new;
+    __nv_bfloat16 *out_bf16;
+    float *out_f32;
+};
+
+struct WSelPartial {      // what one warp of a group found in its share of the rows (32 bytes)
+    unsigned long long max_key;
+    int max_slot, n_pre, n_loc, p, n_cand, n_cand_not_prev;
+};
+
+template <bool FUSED, int MAXW>
+__global__ void __launch_bounds__(MAXW * 32, 1)
 wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int D = a.depth;
-    const WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, D, FUSED);
-    unsigned char *smem = smem_all + (size_t)warp * L.per_warp;
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + L.bars);   // [0..D) tiles, [kWMaxDepth] metadata
-    const uint32_t bar_meta = smem_u32(bars + kWMaxDepth);
-    const uint32_t stages_u32 = smem_u32(smem + L.stages);
+    const int G = a.group_warps, D = a.depth;
+    const int gi = warp / G, rk = warp - gi * G;      // group in the CTA, rank in the group
+    const WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, D, G, FUSED);
+    unsigned char *smem = smem_all + (size_t)gi * L.per_group;
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + L.bars) + rk * kWMaxDepth;
+    const uint32_t bar_meta = smem_u32(reinterpret_cast<unsigned long long *>(smem + L.bars) + kWMaxGroupWarps * kWMaxDepth);
+    unsigned char *ring = smem + L.rings + (size_t)rk * L.ring_bytes;
+    const uint32_t stages_u32 = smem_u32(ring);
+    WSelPartial *sel_part = reinterpret_cast<WSelPartial *>(smem + L.hdr);
+    unsigned long long *sel_thr = reinterpret_cast<unsigned long long *>(smem + L.hdr + kWMaxGroupWarps * 32);
     int32_t *pt_s = reinterpret_cast<int32_t *>(smem + L.pt);
     unsigned long long *sm_keys = reinterpret_cast<unsigned long long *>(smem + L.keys);
-    uint8_t *region = smem + L.region;
+    uint32_t *prevm = reinterpret_cast<uint32_t *>(smem + L.prevm);
+    uint32_t *candm = reinterpret_cast<uint32_t *>(smem + L.candm);
     uint32_t *kmask = reinterpret_cast<uint32_t *>(smem + L.kmask);
     uint32_t *cmask = reinterpret_cast<uint32_t *>(smem + L.cmask);
     __nv_bfloat16 *wsplit = reinterpret_cast<__nv_bfloat16 *>(smem + L.wsplit);
     int *hist = reinterpret_cast<int *>(smem + L.hist);
-    float *svec = reinterpret_cast<float *>(smem + L.svec);
-    if (warp >= a.n_workers) return;
+    float *part = reinterpret_cast<float *>(smem + L.part);
 
     if (lane == 0) {
         for (int s = 0; s < D; ++s) mbar_init(smem_u32(bars + s), 1);
-        mbar_init(bar_meta, 1);
+        if (rk == 0) mbar_init(bar_meta, 1);
         mbar_init_fence();
     }
-    {   // zero the ring once: rows a partial tile never receives must hold finite numbers
-        uint4 *z = reinterpret_cast<uint4 *>(smem + L.stages);
-        for (int i = lane; i < D * kWStageBytes / 16; i += 32) z[i] = make_uint4(0u, 0u, 0u, 0u);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncwarp();
+    __syncthreads();   // the only CTA-wide barrier: every warp is still here
+    auto group_sync = [&]() {
+        if (G == 1) __syncwarp();
+        else asm volatile("bar.sync %0, %1;" ::"r"(1 + gi), "r"(32 * G) : "memory");
+    };
 
     const int g = lane >> 2, t = lane & 3;          // MMA fragment coordinates
     const int mi = lane >> 3, lr = lane & 7;        // ldmatrix: matrix index, row within the matrix
@@ -189,7 +205,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     //   V / pass 2, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
     const uint32_t k_off = (uint32_t)(lr * kWRowBytes + ((mi ^ lr) << 4));
     const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
-    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
+    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g == 3 ? 1 : 0) * L.w_rows);
+    const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     int spin_limit = kCopySpinLimit;
     auto wait = [&](uint32_t bar, uint32_t parity) {
         if (!mbar_wait_sleepy(bar, parity, spin_limit)) {
@@ -200,135 +217,15 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 
     uint32_t issued = 0, consumed = 0;   // tiles of this warp since kernel start (stage = count % D)
     int streams_done = 0;
-    const int stride = gridDim.x * a.n_workers;
-    for (int local = warp * gridDim.x + blockIdx.x; local < c.S; local += stride, ++streams_done) {
+    const int stride = gridDim.x * a.n_groups;
+    for (int local = gi * gridDim.x + blockIdx.x; local < c.S; local += stride, ++streams_done) {
         const int sid = a.layer * c.S + local;
         int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
+        const float *inv_g = c.inv_norm + (size_t)sid * c.max_rows;
+        // ---- everything that only needs addresses is requested first --------------------------------
         int n = c.n_live[sid];
-        if (n < 0 || n > c.max_rows) { if (lane == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
-        const int np = (n + c.page_rows - 1) / c.page_rows;
-        for (int pg = lane; pg < np; pg += 32) pt_s[pg] = pt[pg];
-        const int n_tiles = (n + kWTile - 1) / kWTile;
-        const int total = FUSED ? 2 * n_tiles : n_tiles;   // pass 1 tiles, then pass 2 tiles (V only)
-
-        // ---- metadata: aligned interior by bulk copy, ragged ends by plain loads -------------------
-        const int32_t *pos_s = nullptr;
-        const float *scores_s = nullptr, *inv_s = nullptr;
-        if constexpr (FUSED) {
-            const void *src[3] = {c.pos + (size_t)sid * c.max_rows, c.scores + (size_t)sid * c.max_rows,
-                                  c.inv_norm + (size_t)sid * c.max_rows};
-            uint32_t meta_tx = 0;
-            const uint32_t *base[3];
-#pragma unroll
-            for (int k = 0; k < 3; ++k) {
-                const uint32_t *gp = reinterpret_cast<const uint32_t *>(src[k]);
-                uint32_t *d = reinterpret_cast<uint32_t *>(smem + L.meta) + k * L.meta_words;
-                const int lead = (int)(((uintptr_t)gp >> 2) & 3);
-                const int head = min(n, (4 - lead) & 3);
-                const int body = (n - head) & ~3;
-                if (lane < head) d[lead + lane] = gp[lane];
-                if (lane < n - head - body) d[lead + head + body + lane] = gp[head + body + lane];
-                if (lane == 0 && body > 0) {
-                    bulk_g2s(smem_u32(d + lead + head), gp + head, (uint32_t)body * 4u, bar_meta);
-                    meta_tx += (uint32_t)body * 4u;
-                }
-                base[k] = d + lead;
-            }
-            if (lane == 0) mbar_expect_tx(bar_meta, meta_tx);
-            pos_s = reinterpret_cast<const int32_t *>(base[0]);
-            scores_s = reinterpret_cast<const float *>(base[1]);
-            inv_s = reinterpret_cast<const float *>(base[2]);
-        }
-        __syncwarp();
-
-        // ---- the warp's own copy pipeline ----------------------------------------------------------
-        auto issue = [&](int u) {   // lane 0 only: tile u of this stream into the next free stage
-            const int stage = issued % D;
-            const int pass = u >= n_tiles ? 1 : 0, tl = pass ? u - n_tiles : u;
-            const int r0 = tl * kWTile, r1 = min(n, r0 + kWTile);
-            const uint32_t kdst = stages_u32 + stage * kWStageBytes, vdst = kdst + kWTileBytes;
-            const uint32_t bar = smem_u32(bars + stage);
-            mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
-            int r = r0;
-            {   // the common case: a whole tile inside one page is one box per pool
-                uint32_t pg = __umulhi((uint32_t)r0, c.pr_magic);
-                int in = r0 - (int)pg * c.page_rows;
-                if (r1 - r0 == kWTile && in + kWTile <= c.page_rows) {
-                    int y = pt_s[pg] * c.page_rows + in;
-                    if (pass == 0) tma_2d(kdst, &maps.k[5], 0, y, bar);
-                    tma_2d(vdst, &maps.v[5], 0, y, bar);
-                    r = r1;
-                }
-            }
-            while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
-                uint32_t pg = __umulhi((uint32_t)r, c.pr_magic);
-                int in = r - (int)pg * c.page_rows;
-                int cnt = min(r1 - r, c.page_rows - in);
-                int y = pt_s[pg] * c.page_rows + in;
-                uint32_t off = (uint32_t)(r - r0) * kWRowBytes;
-                r += cnt;
-                while (cnt > 0) {
-                    int hb = 31 - __clz(cnt);
-                    hb = hb > 5 ? 5 : hb;
-                    if (pass == 0) tma_2d(kdst + off, &maps.k[hb], 0, y, bar);
-                    tma_2d(vdst + off, &maps.v[hb], 0, y, bar);
-                    y += 1 << hb; off += (uint32_t)kWRowBytes << hb; cnt -= 1 << hb;
-                }
-            }
-        };
-        int next_issue = 0;
-        if (lane == 0) {
-            for (; next_issue < total && next_issue < D; ++next_issue, ++issued) issue(next_issue);
-        }
-        next_issue = __shfl_sync(0xffffffffu, next_issue, 0);
-        issued = __shfl_sync(0xffffffffu, issued, 0);
-        // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
-        auto release_and_refill = [&]() {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (next_issue < total) {
-                if (lane == 0) issue(next_issue);
-                ++next_issue; ++issued;
-            }
-        };
-
-        // ---- which rows are attended, and the weights of the rows the next step scores -------------
-        int n2 = n, p_next = 0;
-        if constexpr (FUSED) {
-            wait(bar_meta, streams_done & 1);
-            const SelResult sel = warp_select(c, pos_s, scores_s, n, a.cur_pos, a.budget_rows, sm_keys, region, hist);
-            n2 = n - (sel.p - sel.K) + 1;
-            const int n_pad = n_tiles * kWTile;
-            for (int base = 0; base < n_pad; base += 32) {
-                const int slot = base + lane;
-                const bool kept = slot < n && sel.keeps(region[slot], sm_keys[slot]);
-                if (slot < n && (region[slot] & 3) == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
-                const unsigned bk = __ballot_sync(0xffffffffu, kept);
-                const bool cand = kept && (region[slot] & kCandNextBit);
-                const unsigned bc = __ballot_sync(0xffffffffu, cand);
-                if (lane == 0) { kmask[base >> 5] = bk; cmask[base >> 5] = bc; }
-                p_next += __popc(bc);
-                // w = 1/|v| for the rows the next step scores, as three bf16 parts (24 bits)
-                float w = cand ? inv_s[slot] : 0.f;
-                __nv_bfloat16 h = __float2bfloat16_rn(w);
-                float r1 = w - __bfloat162float(h);
-                __nv_bfloat16 md = __float2bfloat16_rn(r1);
-                __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(md));
-                wsplit[slot] = h; wsplit[L.w_rows + slot] = md; wsplit[2 * L.w_rows + slot] = lo;
-            }
-            p_next += new_cand ? 1 : 0;
-        } else {
-            const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
-            for (int w = lane; w < n_tiles; w += 32) {
-                uint32_t bits = gm[w];
-                int valid = n - w * 32;
-                kmask[w] = valid >= 32 ? bits : (bits & ((1u << valid) - 1u));
-            }
-        }
-        __syncwarp();
-
-        // ---- q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements ---------
-        uint32_t qa0[4], qa2[4];
+        for (int pg = lane; pg < c.max_pages; pg += 32) pt_s[pg] = pt[pg];   // every warp of the group writes the same values
+        uint32_t qa0[4], qa2[4];   // q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements
         {
             const uint32_t *q2 = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d);   // c.d is even
 #pragma unroll
@@ -338,9 +235,271 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
         }
-        // ---- the new row starts the running state: weight 1 in A' row 0, its 1/|v| in row 2 --------
-        float m_run, l_run, o_run[8][2];
-        {
+        if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
+        const int n_tiles = (n + kWTile - 1) / kWTile;
+        const int mt = rk < n_tiles ? (n_tiles - rk + G - 1) / G : 0;   // this warp's tiles: rk, rk + G, ...
+        const int total = FUSED ? 2 * mt : mt;                          // pass 1 tiles, then pass 2 tiles (V only)
+        const float *inv_s = nullptr;
+        if constexpr (FUSED) {
+            // inverse norms into shared memory: aligned interior by bulk copy, ragged ends by plain loads
+            const uint32_t *gp = reinterpret_cast<const uint32_t *>(inv_g);
+            uint32_t *d = reinterpret_cast<uint32_t *>(smem + L.inv);
+            const int lead = (int)(((uintptr_t)gp >> 2) & 3);
+            inv_s = reinterpret_cast<const float *>(d + lead);
+            if (rk == 0) {
+                const int head = min(n, (4 - lead) & 3);
+                const int body = (n - head) & ~3;
+                if (lane < head) d[lead + lane] = gp[lane];
+                if (lane < n - head - body) d[lead + head + body + lane] = gp[head + body + lane];
+                __syncwarp();
+                if (lane == 0) {
+                    if (body > 0) bulk_g2s(smem_u32(d + lead + head), gp + head, (uint32_t)body * 4u, bar_meta);
+                    mbar_expect_tx(bar_meta, (uint32_t)body * 4u);
+                }
+            }
+        }
+        __syncwarp();
+
+        // ---- the warp's own copy pipeline ----------------------------------------------------------
+        // Tiles of this warp, in issue order: u = 0 .. mt-1 are pass 1 (K and V), u = mt .. 2mt-1 pass 2 (V).
+        int cur_pg = 0, cur_in = 0;   // page and row-in-page of the next tile to issue (lane 0's copy is the one used)
+        auto seek = [&](int tl) {
+            cur_pg = (int)__umulhi((uint32_t)(tl * kWTile), c.pr_magic);
+            cur_in = tl * kWTile - cur_pg * c.page_rows;
+        };
+        seek(rk);
+        auto issue = [&](int u) {   // lane 0 only: this warp's u-th tile of the stream into the next free stage
+            const int stage = issued % D;
+            const int pass = u >= mt ? 1 : 0, tl = rk + (pass ? u - mt : u) * G;
+            if (u == mt) seek(rk);
+            const int r0 = tl * kWTile, r1 = min(n, r0 + kWTile);
+            const uint32_t kdst = stages_u32 + stage * kWStageBytes, vdst = kdst + kWTileBytes;
+            const uint32_t bar = smem_u32(bars + stage);
+            mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
+            if (r1 - r0 == kWTile && cur_in + kWTile <= c.page_rows) {
+                // the common case: a whole tile inside one page is one box per pool
+                const int y = pt_s[cur_pg] * c.page_rows + cur_in;
+                if (pass == 0) tma_2d(kdst, &maps.k[5], 0, y, bar);
+                tma_2d(vdst, &maps.v[5], 0, y, bar);
+            } else {
+                int r = r0, pg = cur_pg, in = cur_in;
+                while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
+                    int cnt = min(r1 - r, c.page_rows - in);
+                    int y = pt_s[pg] * c.page_rows + in;
+                    uint32_t off = (uint32_t)(r - r0) * kWRowBytes;
+                    r += cnt; in = 0; ++pg;
+                    while (cnt > 0) {
+                        int hb = 31 - __clz(cnt);
+                        hb = hb > 5 ? 5 : hb;
+                        if (pass == 0) tma_2d(kdst + off, &maps.k[hb], 0, y, bar);
+                        tma_2d(vdst + off, &maps.v[hb], 0, y, bar);
+                        y += 1 << hb; off += (uint32_t)kWRowBytes << hb; cnt -= 1 << hb;
+                    }
+                }
+            }
+            cur_in += G * kWTile;   // the warp's next tile is G tiles further on
+            while (cur_in >= c.page_rows) { cur_in -= c.page_rows; ++cur_pg; }
+        };
+        // Rows of a partial tile that the copy does not write must hold finite numbers (their weights
+        // are zero, and 0 * NaN would not be): all lanes clear them before the tile is requested.
+        auto clear_tail = [&](int u) {
+            const int tl = rk + (u >= mt ? u - mt : u) * G;
+            const int rows = min(n, (tl + 1) * kWTile) - tl * kWTile;
+            if (rows < kWTile) {
+                uint4 *z = reinterpret_cast<uint4 *>(ring + (issued % D) * kWStageBytes);
+                for (int i = rows * 8 + lane; i < kWTile * 8; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
+            }
+        };
+        int next_issue = 0;
+        for (; next_issue < total && next_issue < D; ++next_issue, ++issued) {
+            clear_tail(next_issue);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) issue(next_issue);
+        }
+        // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
+        auto release_and_refill = [&]() {
+            if (next_issue < total) clear_tail(next_issue);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (next_issue < total) {
+                if (lane == 0) issue(next_issue);
+                ++next_issue; ++issued;
+            }
+        };
+        // the barrier of the tile after the current one is tested early, so that the test's latency
+        // overlaps the arithmetic; `ready` is true when that test already saw the tile complete
+        bool ready = false;
+        auto peek_next = [&](bool more) {
+            const uint32_t nx = consumed + 1;
+            ready = more && mbar_try_wait(smem_u32(bars + nx % D), (nx / D) & 1);
+        };
+
+        // ---- which rows are attended, and the weights of the rows the next step scores -------------
+        // Each warp of the group looks at the 32-row blocks it will also sweep (rk, rk + G, ...).
+        int n2 = n, p_next = 0, n_evict = 0, evict_slot = -1;
+        if constexpr (FUSED) {
+            const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
+            const float *sc_g = c.scores + (size_t)sid * c.max_rows;
+            WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
+            unsigned long long my_key = 0ull;
+            int my_slot = -1;
+            for (int b0 = rk; b0 < n_tiles; b0 += 4 * G) {   // four blocks per round: their loads overlap
+                int ps[4];
+                float sc[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int slot = (b0 + u * G) * 32 + lane;
+                    const bool live = b0 + u * G < n_tiles && slot < n;
+                    ps[u] = live ? pos_g[slot] : -1;
+                    sc[u] = live ? sc_g[slot] : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int b = b0 + u * G;
+                    if (b >= n_tiles) break;
+                    const int slot = b * 32 + lane;
+                    const bool live = slot < n;
+                    const int reg = live ? region_by_cut(c, cut_now, ps[u]) : -1;
+                    const bool is_prev = reg == kRegionPrevious;
+                    const bool is_cand = live && reg != kRegionInvalid && region_by_cut(c, cut_next, ps[u]) == kRegionPrevious;
+                    if (live && reg == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
+                    unsigned long long key = ~0ull;
+                    if (is_prev) {
+                        key = ((unsigned long long)orderable(sc[u]) << 32) | (uint32_t)ps[u];
+                        if (key > my_key) { my_key = key; my_slot = slot; }
+                    }
+                    if (live) sm_keys[slot] = key;
+                    const unsigned bp = __ballot_sync(0xffffffffu, is_prev), bc = __ballot_sync(0xffffffffu, is_cand);
+                    mine.n_pre += __popc(__ballot_sync(0xffffffffu, reg == kRegionPrefix));
+                    mine.n_loc += __popc(__ballot_sync(0xffffffffu, reg == kRegionLocal));
+                    mine.p += __popc(bp);
+                    mine.n_cand += __popc(bc);
+                    mine.n_cand_not_prev += __popc(bc & ~bp);
+                    if (lane == 0) { prevm[b] = bp; candm[b] = bc; }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                unsigned long long ok = __shfl_xor_sync(0xffffffffu, my_key, o);
+                int os = __shfl_xor_sync(0xffffffffu, my_slot, o);
+                if (ok > my_key) { my_key = ok; my_slot = os; }
+            }
+            mine.max_key = my_key; mine.max_slot = my_slot;
+            if (lane == 0) sel_part[rk] = mine;
+            group_sync();
+            int n_pre = 0, n_loc = 0, p = 0, n_cand = 0, n_cand_np = 0;
+            unsigned long long max_key = 0ull;
+            int max_slot = -1;
+            for (int w = 0; w < G; ++w) {
+                const WSelPartial o = sel_part[w];
+                n_pre += o.n_pre; n_loc += o.n_loc; p += o.p; n_cand += o.n_cand; n_cand_np += o.n_cand_not_prev;
+                if (o.max_key > max_key) { max_key = o.max_key; max_slot = o.max_slot; }
+            }
+            int K = a.budget_rows - n_pre - n_loc - 1;
+            K = K < 0 ? 0 : (K > p ? p : K);
+            n_evict = p - K;
+            n2 = n - n_evict + 1;
+            wait(bar_meta, streams_done & 1);   // the inverse norms are in shared memory
+            const bool general = K > 0 && K < p - 1;
+            if (!general) {
+                if (K == p - 1 && p > 0) evict_slot = max_slot;
+                const bool drop_prev = K == 0 && p > 0;
+                for (int b = rk; b < n_tiles; b += G) {
+                    const int valid = n - b * 32;
+                    uint32_t keep = valid >= 32 ? 0xffffffffu : ((1u << valid) - 1u);
+                    if (drop_prev) keep &= ~prevm[b];
+                    if (evict_slot >= 0 && (evict_slot >> 5) == b) keep &= ~(1u << (evict_slot & 31));
+                    if (lane == 0) { kmask[b] = keep; cmask[b] = candm[b] & keep; }
+                }
+                p_next = K >= p ? n_cand : drop_prev ? n_cand_np : n_cand - ((candm[evict_slot >> 5] >> (evict_slot & 31)) & 1u);
+            } else {
+                // arbitrary K: radix select over all keys by the first warp, then every warp marks every block
+                if (rk == 0) {
+                    unsigned long long mask = 0ull, thr = 0ull;
+                    int k_rem = K;
+                    for (int shift = 56; shift >= 0; shift -= 8) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) hist[lane * 8 + i] = 0;
+                        __syncwarp();
+                        for (int slot = lane; slot < n; slot += 32) {
+                            unsigned long long key = sm_keys[slot];
+                            if (((prevm[slot >> 5] >> (slot & 31)) & 1u) && (key & mask) == thr)
+                                atomicAdd(&hist[(int)((key >> shift) & 255ull)], 1);
+                        }
+                        __syncwarp();
+                        int h[8], tot = 0;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { h[i] = hist[lane * 8 + i]; tot += h[i]; }
+                        int incl = tot;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            int tt = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= o) incl += tt;
+                        }
+                        int excl = incl - tot, digit = 0, krem = 0, bin = 0;
+                        const bool own = excl < k_rem && k_rem <= incl;   // exactly one lane holds the bin of the k_rem-th key
+                        if (own) {
+                            int cum = excl;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (cum < k_rem && k_rem <= cum + h[i]) { digit = lane * 8 + i; krem = k_rem - cum; bin = h[i]; }
+                                cum += h[i];
+                            }
+                        }
+                        const int src = __ffs(__ballot_sync(0xffffffffu, own)) - 1;
+                        digit = __shfl_sync(0xffffffffu, digit, src);
+                        krem = __shfl_sync(0xffffffffu, krem, src);
+                        bin = __shfl_sync(0xffffffffu, bin, src);
+                        thr |= (unsigned long long)digit << shift;
+                        mask |= 255ull << shift;
+                        k_rem = krem;
+                        __syncwarp();
+                        if (k_rem == bin) break;             // the whole bin is kept: masked compare decides
+                    }
+                    if (lane == 0) { sel_thr[0] = mask; sel_thr[1] = thr; }
+                }
+                group_sync();
+                const unsigned long long mask = sel_thr[0], thr = sel_thr[1];
+                for (int b = 0; b < n_tiles; ++b) {   // all blocks: the compaction lists need them all
+                    const int slot = b * 32 + lane;
+                    const bool live = slot < n;
+                    const bool is_prev = (prevm[b] >> lane) & 1u;
+                    const bool kept = live && (!is_prev || (sm_keys[slot] & mask) <= thr);
+                    const unsigned bk = __ballot_sync(0xffffffffu, kept);
+                    const unsigned bcm = candm[b] & bk;
+                    p_next += __popc(bcm);
+                    __syncwarp();
+                    if (lane == 0) { kmask[b] = bk; cmask[b] = bcm; }   // every warp writes the same words
+                }
+            }
+            p_next += new_cand ? 1 : 0;
+            __syncwarp();
+            // w = 1/|v| for the retained rows the next step scores, as two bf16 parts (16 bits: the
+            // relative error 2^-17 of a weight moves a score by less than 1e-7)
+            for (int b = rk; b < n_tiles; b += G) {
+                const int slot = b * 32 + lane;
+                const bool cand = (cmask[b] >> lane) & 1u;
+                float w = cand ? inv_s[slot] : 0.f;
+                __nv_bfloat16 h = __float2bfloat16_rn(w);
+                __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(h));
+                wsplit[slot] = h; wsplit[L.w_rows + slot] = lo;
+            }
+        } else {
+            const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
+            for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {
+                uint32_t bits = gm[b];
+                int valid = n - b * 32;
+                kmask[b] = valid >= 32 ? bits : (bits & ((1u << valid) - 1u));
+            }
+        }
+        __syncwarp();
+
+        // ---- the running state; the first warp starts from the new row: weight 1 in A' row 0, its 1/|v| in row 2 ----
+        float m_run = -FLT_MAX, l_run = 0.f, o_run[8][2];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) { o_run[nb][0] = 0.f; o_run[nb][1] = 0.f; }
+        if (rk == 0) {
             float s = 0.f, ss = 0.f;
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
@@ -372,9 +531,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
 
         // ---- pass 1 --------------------------------------------------------------------------------
-        for (int tl = 0; tl < n_tiles; ++tl, ++consumed) {
+        for (int tl = rk; tl < n_tiles; tl += G, ++consumed) {
             const int stage = consumed % D;
-            wait(smem_u32(bars + stage), (consumed / D) & 1);
+            if (!ready) wait(smem_u32(bars + stage), (consumed / D) & 1);
             const uint32_t kb = stages_u32 + stage * kWStageBytes, vb = kb + kWTileBytes;
             const int r0 = tl * kWTile;
             const uint32_t kw = kmask[tl] >> (2 * t);   // bit 8*nb + e: row 8*nb + 2t + e is retained
@@ -389,6 +548,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 mma_bf16(sc[nb], qa0[2], 0u, qa2[2], 0u, kf1[0], kf1[1]);
                 mma_bf16(sc[nb], qa0[3], 0u, qa2[3], 0u, kf1[2], kf1[3]);
             }
+            peek_next(tl + G < n_tiles || FUSED);
             // this lane's 8 logits: rows 8*nb + 2t, 8*nb + 2t + 1 (the same in every lane group)
             float x[4][2], mx = -INFINITY;
 #pragma unroll
@@ -412,7 +572,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 for (int e = 0; e < 2; ++e) { x[nb][e] = ex2(x[nb][e] - m_new); psum += x[nb][e]; }
             }
             l_run = fmaf(l_run, corr, psum);
-            // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0
+            // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_lo, 0, 0, 0, 0
             uint32_t pa0[2], pa2[2];
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
@@ -424,8 +584,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     w0 = w_role[(r0 + 16 * ks + 2 * t) >> 1];
                     w2 = w_role[(r0 + 16 * ks + 8 + 2 * t) >> 1];
                 }
-                pa0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
-                pa2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
+                pa0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 3 ? w0 : 0u;
+                pa2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 3 ? w2 : 0u;
             }
             // O_tile = A'.V from zero, then folded into the running sums
             float ot[8][4];
@@ -452,18 +612,40 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
         }
 
-        // ---- softmax.V = rows 0 + 1 over l; s = rows 2 + 3 + 4 -------------------------------------
+        // ---- this warp's state: softmax.V = rows 0 + 1, s = rows 2 + 3; then the warps of the group ----
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        const float inv_l = 1.0f / l_run;
+        {
+            float *w = part + rk * 132;
 #pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
-            float v0 = o_run[nb][0], v1 = o_run[nb][1];
-            float a0 = __shfl_down_sync(0xffffffffu, v0, 4), a1 = __shfl_down_sync(0xffffffffu, v1, 4);
-            float b0 = __shfl_down_sync(0xffffffffu, v0, 8), b1 = __shfl_down_sync(0xffffffffu, v1, 8);
-            const int xx = 8 * nb + 2 * t;
-            if (g == 0 && xx < c.d) {
-                float o0 = (v0 + a0) * inv_l, o1 = (v1 + a1) * inv_l;
+            for (int nb = 0; nb < 8; ++nb) {
+                float v0 = o_run[nb][0], v1 = o_run[nb][1];
+                float a0 = __shfl_down_sync(0xffffffffu, v0, 4), a1 = __shfl_down_sync(0xffffffffu, v1, 4);
+                const int xx = 8 * nb + 2 * t;
+                if (g == 0) { w[xx] = v0 + a0; w[xx + 1] = v1 + a1; }
+                if (g == 2) { w[64 + xx] = v0 + a0; w[64 + xx + 1] = v1 + a1; }
+            }
+            if (lane == 0) { w[128] = m_run; w[129] = l_run; }
+        }
+        group_sync();
+        float sv0, sv1;   // s[2*lane], s[2*lane + 1]
+        {
+            float M = -FLT_MAX;
+            for (int w = 0; w < G; ++w) M = fmaxf(M, part[w * 132 + 128]);
+            float Lb = 0.f, A0 = 0.f, A1 = 0.f;
+            sv0 = 0.f; sv1 = 0.f;
+            for (int w = 0; w < G; ++w) {
+                const float *ws = part + w * 132;
+                float wgt = exp2f(ws[128] - M);
+                Lb = fmaf(ws[129], wgt, Lb);
+                A0 = fmaf(ws[2 * lane], wgt, A0);
+                A1 = fmaf(ws[2 * lane + 1], wgt, A1);
+                sv0 += ws[64 + 2 * lane];
+                sv1 += ws[64 + 2 * lane + 1];
+            }
+            const int xx = 2 * lane;
+            if (rk == 0 && xx < c.d) {
+                float o0 = A0 / Lb, o1 = A1 / Lb;
                 if (a.out_f32) {
                     a.out_f32[(size_t)local * c.d + xx] = o0;
                     if (xx + 1 < c.d) a.out_f32[(size_t)local * c.d + xx + 1] = o1;
@@ -471,61 +653,68 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 if (a.out_bf16)
                     *reinterpret_cast<uint32_t *>(a.out_bf16 + (size_t)local * c.d + xx) = pack_bf16(o0, o1);
             }
-            if (g == 2) { svec[xx] = (v0 + a0) + b0; svec[xx + 1] = (v1 + a1) + b1; }
         }
-        __syncwarp();
 
         if constexpr (FUSED) {
             // ---- Section 4.2 bookkeeping: holes below the new length, survivors above it ----------
             int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;   // keys are dead now
-            int nh = 0, ns = 0;
-            const int top = max(n, n2);
-            for (int base = 0; base < top; base += 32) {
-                const int s = base + lane;
-                const bool kept = s < n && ((kmask[s >> 5] >> (s & 31)) & 1u);
-                const bool is_hole = s < n2 && !kept, is_surv = s >= n2 && s < n && kept;
-                const unsigned bh = __ballot_sync(0xffffffffu, is_hole), bs = __ballot_sync(0xffffffffu, is_surv);
-                const unsigned below = (1u << lane) - 1u;
-                if (is_hole) holes[nh + __popc(bh & below)] = s;
-                if (is_surv) surv[ns + __popc(bs & below)] = s;
-                nh += __popc(bh); ns += __popc(bs);
+            int nh = 1, ns = 0, last_hole = n;   // nothing evicted: the new row goes to the end
+            if (n_evict == 1 && evict_slot >= 0) {
+                last_hole = evict_slot;          // one eviction: the new row takes its place
+            } else if (n_evict > 0) {
+                // the general case; every warp builds the same lists (identical values to the same places)
+                nh = 0;
+                const int top = max(n, n2);
+                for (int base = 0; base < top; base += 32) {
+                    const int s = base + lane;
+                    const bool kept = s < n && ((kmask[s >> 5] >> (s & 31)) & 1u);
+                    const bool is_hole = s < n2 && !kept, is_surv = s >= n2 && s < n && kept;
+                    const unsigned bh = __ballot_sync(0xffffffffu, is_hole), bs = __ballot_sync(0xffffffffu, is_surv);
+                    const unsigned below = (1u << lane) - 1u;
+                    if (is_hole) holes[nh + __popc(bh & below)] = s;
+                    if (is_surv) surv[ns + __popc(bs & below)] = s;
+                    nh += __popc(bh); ns += __popc(bs);
+                }
+                __syncwarp();
+                last_hole = nh > ns && nh > 0 ? holes[ns] : n;
             }
-            __syncwarp();
             const int have = (n + c.page_rows - 1) / c.page_rows, need = (n2 + c.page_rows - 1) / c.page_rows;
             int okay = 1;
             if (lane == 0) {
-                if (nh != ns + 1) { set_status(c, ADSA_DEV_BAD_EVICT); okay = 0; }
-                else if (n2 > c.max_rows) { set_status(c, ADSA_DEV_ROW_OVERFLOW); okay = 0; }
-                else if (need > have && !resize_pages(c, pt, have, need)) okay = 0;
+                if (nh != ns + 1) { if (rk == 0) set_status(c, ADSA_DEV_BAD_EVICT); okay = 0; }
+                else if (n2 > c.max_rows) { if (rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); okay = 0; }
+                else if (rk == 0 && need > have && !resize_pages(c, pt, have, need)) okay = 0;
             }
             okay = __shfl_sync(0xffffffffu, okay, 0);
             __syncwarp();   // lane 0 may have written a page-table entry the others are about to read
             const float denom = (float)(p_next - 1);
             float *scores = c.scores + (size_t)sid * c.max_rows;
 
-            // s as the B operand: columns 0, 1, 2 = its bf16 hi, mid, lo parts
+            // s as the B operand: columns 0, 1, 2 = its bf16 hi, mid, lo parts (s[2*lane..] sits in lane `lane`)
             uint32_t sb0[4], sb1[4];
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-                float v[4] = {svec[16 * ks + 2 * t], svec[16 * ks + 2 * t + 1], svec[16 * ks + 2 * t + 8], svec[16 * ks + 2 * t + 9]};
-                float part[4];
+                const int e0 = 16 * ks + 2 * t;   // elements e0, e0 + 1 live in lane e0 / 2; e0 + 8, e0 + 9 in lane e0 / 2 + 4
+                float v[4] = {__shfl_sync(0xffffffffu, sv0, e0 >> 1), __shfl_sync(0xffffffffu, sv1, e0 >> 1),
+                              __shfl_sync(0xffffffffu, sv0, (e0 >> 1) + 4), __shfl_sync(0xffffffffu, sv1, (e0 >> 1) + 4)};
+                float pr[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     float h = __bfloat162float(__float2bfloat16_rn(v[i]));
                     float md = __bfloat162float(__float2bfloat16_rn(v[i] - h));
                     float lo = __bfloat162float(__float2bfloat16_rn(v[i] - h - md));
-                    part[i] = g == 0 ? h : g == 1 ? md : g == 2 ? lo : 0.f;
+                    pr[i] = g == 0 ? h : g == 1 ? md : g == 2 ? lo : 0.f;
                 }
-                sb0[ks] = pack_bf16(part[0], part[1]);
-                sb1[ks] = pack_bf16(part[2], part[3]);
+                sb0[ks] = pack_bf16(pr[0], pr[1]);
+                sb1[ks] = pack_bf16(pr[2], pr[3]);
             }
 
             // ---- pass 2: dot_i = v_i . s, S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), at the row's new slot ----
-            for (int tl = 0; tl < n_tiles; ++tl, ++consumed) {
+            for (int tl = rk; tl < n_tiles; tl += G, ++consumed) {
                 const int stage = consumed % D;
-                wait(smem_u32(bars + stage), (consumed / D) & 1);
+                if (!ready) wait(smem_u32(bars + stage), (consumed / D) & 1);
                 const uint32_t vb = stages_u32 + stage * kWStageBytes + kWTileBytes;
-                const unsigned char *vtile = smem + L.stages + stage * kWStageBytes + kWTileBytes;
+                const unsigned char *vtile = ring + stage * kWStageBytes + kWTileBytes;
                 const int r0 = tl * kWTile;
                 const uint32_t cw = okay ? cmask[tl] : 0u;
                 float dt[2][4];
@@ -539,40 +728,55 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                     }
                 }
+                peek_next(tl + G < n_tiles);
+                // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
+                float sval[4], invv[4], dotv[4];
+                bool want[4], rare = false;
 #pragma unroll
-                for (int mbk = 0; mbk < 2; ++mbk) {
+                for (int i = 0; i < 4; ++i) {
+                    const int mbk = i >> 1, hh = i & 1;
+                    const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
+                    const int row = r0 + 16 * mbk + 8 * hh + g;
+                    want[i] = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
+                    invv[i] = inv_s[min(row, n - 1)];
+                    dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
+                    sval[i] = p_next > 1 ? (invv[i] * dotv[i] - 1.0f) / denom + 0.0f : 0.0f;
+                    rare |= want[i] && (invv[i] >= 1.0f / kNormEps || row >= n2);
+                }
+                if (!__any_sync(0xffffffffu, rare)) {
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {   // rows 16*mbk + 8*hh + g: columns 0, 1 in lane t = 0, column 2 in t = 1
-                        float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
-                        const int row = r0 + 16 * mbk + 8 * hh + g;
-                        const bool want = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
-                        if (want) {
-                            float dot = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
-                            float inv = inv_s[row], self = 1.0f;
-                            if (inv >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
-                                float ss = 0.f;
-                                for (int ch = 0; ch < 8; ++ch) {
-                                    float f[8];
-                                    unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
-                                    for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-                                }
-                                self = inv * inv * ss;
+                    for (int i = 0; i < 4; ++i)
+                        if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (!want[i]) continue;
+                        const int mbk = i >> 1, hh = i & 1, row = r0 + 16 * mbk + 8 * hh + g;
+                        float s_out = sval[i];
+                        if (invv[i] >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
+                            float ss = 0.f;
+                            for (int ch = 0; ch < 8; ++ch) {
+                                float f[8];
+                                unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
+                                for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
                             }
-                            int dst = row;
-                            if (row >= n2) {   // a survivor: it moves into the hole of the same rank
-                                int lo_i = 0, hi_i = ns - 1;
-                                while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
-                                dst = holes[lo_i];
-                            }
-                            scores[dst] = p_next > 1 ? (inv * dot - self) / denom + 0.0f : 0.0f;
+                            s_out = p_next > 1 ? (invv[i] * dotv[i] - invv[i] * invv[i] * ss) / denom + 0.0f : 0.0f;
                         }
+                        int dst = row;
+                        if (row >= n2) {   // a survivor: it moves into the hole of the same rank
+                            int lo_i = 0, hi_i = ns - 1;
+                            while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
+                            dst = holes[lo_i];
+                        }
+                        scores[dst] = s_out;
                     }
                 }
                 release_and_refill();
             }
+            group_sync();   // every warp's copies of this stream have landed before rows move or pages are freed
 
-            // ---- the update itself ---------------------------------------------------------------
-            if (okay) {
+            // ---- the update itself, by the first warp ---------------------------------------------------
+            if (okay && rk == 0) {
                 for (int i = 0; i < ns; ++i) {   // survivors move down: 8 + 8 pieces of 16 bytes
                     const int row = surv[i], dst = holes[i];
                     size_t so = row_offset(c, pt, row), go = row_offset(c, pt, dst);
@@ -581,7 +785,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         reinterpret_cast<uint4 *>(pool + go)[lane & 7] = reinterpret_cast<const uint4 *>(pool + so)[lane & 7];
                     }
                     if (lane == 0) {
-                        c.pos[(size_t)sid * c.max_rows + dst] = pos_s[row];
+                        c.pos[(size_t)sid * c.max_rows + dst] = c.pos[(size_t)sid * c.max_rows + row];
                         c.inv_norm[(size_t)sid * c.max_rows + dst] = inv_s[row];
                     }
                 }
@@ -591,7 +795,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     for (int e = 0; e < 2; ++e) {
                         int xx = 2 * lane + e;
                         float vf = xx < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + xx]) : 0.f;
-                        dot = fmaf(vf, svec[xx], dot);
+                        dot = fmaf(vf, e == 0 ? sv0 : sv1, dot);
                         ss = fmaf(vf, vf, ss);
                     }
 #pragma unroll
@@ -600,16 +804,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         ss += __shfl_xor_sync(0xffffffffu, ss, o);
                     }
                     float inv = 1.0f / fmaxf(sqrtf(ss), kNormEps);
-                    if (lane == 0) scores[holes[ns]] = p_next > 1 ? (inv * dot - inv * inv * ss) / denom + 0.0f : 0.0f;
+                    if (lane == 0) scores[last_hole] = p_next > 1 ? (inv * dot - inv * inv * ss) / denom + 0.0f : 0.0f;
                 }
-                write_row(c, pt, sid, holes[ns], a.k_new + (size_t)local * c.d, a.v_new + (size_t)local * c.d, a.cur_pos);
+                write_row(c, pt, sid, last_hole, a.k_new + (size_t)local * c.d, a.v_new + (size_t)local * c.d, a.cur_pos);
                 if (lane == 0) {
                     if (need < have) resize_pages(c, pt, have, need);
                     c.n_live[sid] = n2;
                 }
             }
         }
-        __syncwarp();   // the stream's shared buffers are free for the next one
+        group_sync();   // the stream's shared buffers are free for the next one
     }
 }
 
@@ -651,32 +855,40 @@ int build_wstep_maps(const DevCtx &c, WStepMaps *out)
 cudaError_t configure_wstep_kernel(const DevCtx &c)
 {
     (void)c;
-    cudaError_t e = cudaFuncSetAttribute(wstep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemLimit);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(wstep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemLimit);
+    cudaError_t e = cudaFuncSetAttribute(wstep_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    return e;
 }
 
-// Workers (warps) per CTA and ring depth per worker: enough workers that every stream of the layer
-// has one if possible, at most 8, as many as fit with a ring of at least 2 (preferably 3+) stages.
-WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth)
+// Groups per CTA, warps per group and ring depth per warp.  As many groups as the SM has streams to
+// serve (at most 8), then as many warps per group as shared memory and the 16 warps of a CTA allow
+// with a ring of at least two tiles each.  group_warps > 0 fixes the group size.
+WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps)
 {
     WStepPlan p = {};
     if (!wstep_supported(c)) return p;
-    int want = (c.S + sm_count - 1) / sm_count;
-    want = want < 1 ? 1 : want > 8 ? 8 : want;
-    int cap = max_depth > 0 && max_depth < kWMaxDepth ? max_depth : kWMaxDepth;
-    for (int w = want; w >= 1; --w) {
-        const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, fused).per_warp;
-        if ((uint64_t)fixed * w >= (uint64_t)kPSmemLimit) continue;
-        int depth = (int)((kPSmemLimit - 1024) / w - fixed) / kWStageBytes;
-        depth = depth > cap ? cap : depth;
-        if (depth < 2 || (depth < 3 && w > 1)) continue;
-        WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, fused);
-        if ((uint64_t)L.per_warp * w + 1024 > (uint64_t)kPSmemLimit) { if (--depth < 2) continue; L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, fused); }
-        p.n_workers = w; p.depth = depth; p.smem_bytes = (size_t)L.per_warp * w;
-        int ctas = (c.S + w - 1) / w;
-        p.grid = ctas < sm_count ? ctas : sm_count;
-        return p;
+    int groups = (c.S + sm_count - 1) / sm_count;
+    groups = groups < 1 ? 1 : groups > 8 ? 8 : groups;
+    const int cap = max_depth > 0 && max_depth < kWMaxDepth ? max_depth : kWMaxDepth;
+    for (; groups >= 1; --groups) {
+        for (int G = group_warps > 0 ? group_warps : kWMaxGroupWarps; G >= 1; --G) {
+            if (G > kWMaxGroupWarps || groups * G > 16) { if (group_warps > 0) break; continue; }
+            const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused).per_group;
+            const long long room = (long long)kWSmemLimit / groups - fixed;
+            int depth = room > 0 ? (int)(room / ((long long)G * kWStageBytes)) : 0;
+            depth = depth > cap ? cap : depth;
+            if (depth >= 2 || (depth >= 1 && G == 1 && groups == 1)) {
+                WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, G, fused);
+                p.n_groups = groups; p.group_warps = G; p.depth = depth;
+                p.smem_bytes = (size_t)L.per_group * groups;
+                int ctas = (c.S + groups - 1) / groups;
+                p.grid = ctas < sm_count ? ctas : sm_count;
+                return p;
+            }
+            if (group_warps > 0) break;
+        }
     }
     return p;
 }
@@ -686,12 +898,18 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
                          float *out_f32, cudaStream_t st)
 {
     WStepArgs a;
-    a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth; a.n_workers = plan.n_workers;
+    a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
+    a.group_warps = plan.group_warps; a.n_groups = plan.n_groups;
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
-    const int threads = plan.n_workers * 32;
-    if (fused) wstep_kernel<true><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-    else wstep_kernel<false><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+    const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
+    if (warps <= 8) {
+        if (fused) wstep_kernel<true, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+        else wstep_kernel<false, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+    } else {
+        if (fused) wstep_kernel<true, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+        else wstep_kernel<false, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+    }
     return cudaGetLastError();
 }
 
