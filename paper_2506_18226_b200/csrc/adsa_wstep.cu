@@ -29,9 +29,9 @@
 //
 // Pass 1, per tile:  S = q.K^T  (A = q in rows 0-7, B = K rows via ldmatrix);
 //   P = exp2(S*scale - m), split into bf16 hi + lo so the product keeps fp32-like
-//   accuracy;  O_tile = A'.V with A' rows {P_hi, P_lo, w_hi, w_lo}, where
+//   accuracy;  O_tile = A'.V with A' rows {P_hi, P_lo, w_hi, w_mid, w_lo}, where
 //   w_j = 1/|v_j| for the rows the next step will score and 0 otherwise: rows 0-1 of
-//   the result accumulate softmax.V, rows 2-3 accumulate s = sum of normalised rows.
+//   the result accumulate softmax.V, rows 2-4 accumulate s = sum of normalised rows.
 //   Each tile's product starts from zero and is folded into fp32 running sums with
 //   round-to-nearest FMAs, so tensor-core accumulation rounding never compounds
 //   beyond 32 rows.
@@ -129,14 +129,19 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     L.pt = off;     off += w_align(max_pages * 4, 16);
     L.inv_words = w_align(max_rows + 8, 4);
     L.inv = off;    off += fused ? L.inv_words * 4 : 0;                   // inverse norms by slot
-    L.keys = off;   off += fused ? w_align((max_rows + 2) * 8, 16) : 0;   // later reused: holes, survivors
+    L.w_rows = w_align(max_rows + kWTile, 32);
+    // one region, three lives: selection keys; then the row weights (bf16 hi | mid | lo) during pass 1;
+    // then the compaction lists (holes, survivors)
+    {
+        uint32_t kb = w_align((max_rows + 2) * 8, 16), wb = 3 * L.w_rows * 2;
+        L.keys = off; L.wsplit = off;
+        off += fused ? (kb > wb ? kb : wb) : 0;
+    }
     L.mwords = mask_words + 1;
     L.prevm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows of the previous region
     L.candm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows in the previous region of the next step
     L.kmask = off;  off += w_align(L.mwords * 4, 16);                     // retained rows
     L.cmask = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // retained rows the next step scores
-    L.w_rows = w_align(max_rows + kWTile, 32);
-    L.wsplit = off; off += fused ? 2 * L.w_rows * 2 : 0;                  // bf16 hi | lo of the row weights
     L.part = off;   off += kWMaxGroupWarps * 132 * 4;                     // per warp: acc[64] | s[64] | m, l
     L.hist = L.part;                                                      // radix histogram: used before any partial state exists
     off = w_align(off, 1024);                                             // the swizzle pattern repeats every 1024 bytes
@@ -205,7 +210,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     //   V / pass 2, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
     const uint32_t k_off = (uint32_t)(lr * kWRowBytes + ((mi ^ lr) << 4));
     const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
-    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g == 3 ? 1 : 0) * L.w_rows);
+    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     int spin_limit = kCopySpinLimit;
     auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -475,15 +480,18 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             p_next += new_cand ? 1 : 0;
             __syncwarp();
-            // w = 1/|v| for the retained rows the next step scores, as two bf16 parts (16 bits: the
-            // relative error 2^-17 of a weight moves a score by less than 1e-7)
+            // w = 1/|v| for the retained rows the next step scores, as three bf16 parts (24 bits); they
+            // take the place of the keys, which nobody reads any more
+            if (general) group_sync();
             for (int b = rk; b < n_tiles; b += G) {
                 const int slot = b * 32 + lane;
                 const bool cand = (cmask[b] >> lane) & 1u;
                 float w = cand ? inv_s[slot] : 0.f;
                 __nv_bfloat16 h = __float2bfloat16_rn(w);
-                __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(h));
-                wsplit[slot] = h; wsplit[L.w_rows + slot] = lo;
+                float r1 = w - __bfloat162float(h);
+                __nv_bfloat16 md = __float2bfloat16_rn(r1);
+                __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(md));
+                wsplit[slot] = h; wsplit[L.w_rows + slot] = md; wsplit[2 * L.w_rows + slot] = lo;
             }
         } else {
             const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
@@ -572,7 +580,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 for (int e = 0; e < 2; ++e) { x[nb][e] = ex2(x[nb][e] - m_new); psum += x[nb][e]; }
             }
             l_run = fmaf(l_run, corr, psum);
-            // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_lo, 0, 0, 0, 0
+            // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0
             uint32_t pa0[2], pa2[2];
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
@@ -584,8 +592,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     w0 = w_role[(r0 + 16 * ks + 2 * t) >> 1];
                     w2 = w_role[(r0 + 16 * ks + 8 + 2 * t) >> 1];
                 }
-                pa0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 3 ? w0 : 0u;
-                pa2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 3 ? w2 : 0u;
+                pa0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
+                pa2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
             }
             // O_tile = A'.V from zero, then folded into the running sums
             float ot[8][4];
@@ -612,7 +620,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
         }
 
-        // ---- this warp's state: softmax.V = rows 0 + 1, s = rows 2 + 3; then the warps of the group ----
+        // ---- this warp's state: softmax.V = rows 0 + 1, s = rows 2 + 3 + 4; then the warps of the group ----
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
         {
@@ -621,9 +629,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             for (int nb = 0; nb < 8; ++nb) {
                 float v0 = o_run[nb][0], v1 = o_run[nb][1];
                 float a0 = __shfl_down_sync(0xffffffffu, v0, 4), a1 = __shfl_down_sync(0xffffffffu, v1, 4);
+                float b0 = __shfl_down_sync(0xffffffffu, v0, 8), b1 = __shfl_down_sync(0xffffffffu, v1, 8);
                 const int xx = 8 * nb + 2 * t;
                 if (g == 0) { w[xx] = v0 + a0; w[xx + 1] = v1 + a1; }
-                if (g == 2) { w[64 + xx] = v0 + a0; w[64 + xx + 1] = v1 + a1; }
+                if (g == 2) { w[64 + xx] = (v0 + a0) + b0; w[64 + xx + 1] = (v1 + a1) + b1; }
             }
             if (lane == 0) { w[128] = m_run; w[129] = l_run; }
         }
