@@ -27,11 +27,14 @@
 // (page pieces are cut into boxes of 32, 16, .. 1 rows: one tensor map per height).
 // The warp's lane 0 issues tile u + depth as soon as tile u has been read.
 //
-// Pass 1, per tile:  S = q.K^T  (A = q in rows 0-7, B = K rows via ldmatrix);
+// Pass 1, per tile:  S = K.q  (A = 16 rows of K via ldmatrix, B = q in every column);
 //   P = exp2(S*scale - m), split into bf16 hi + lo so the product keeps fp32-like
-//   accuracy;  O_tile = A'.V with A' rows {P_hi, P_lo, w_hi, w_mid, w_lo}, where
-//   w_j = 1/|v_j| for the rows the next step will score and 0 otherwise: rows 0-1 of
-//   the result accumulate softmax.V, rows 2-4 accumulate s = sum of normalised rows.
+//   accuracy;  O^T_tile = V^T.B' (A = V^T via transposing ldmatrix) with B' columns
+//   {P_hi, P_lo, w_hi, w_mid, w_lo}, where w_j = 1/|v_j| for the rows the next step will
+//   score and 0 otherwise: columns 0-1 of the result accumulate softmax.V, columns 2-4
+//   accumulate s = sum of normalised rows.  This orientation puts the long dimensions
+//   (rows, head elements) on M, so a 32-row tile costs 16 MMAs instead of 32; on this
+//   part the legacy mma.sync pipe is slow enough for that to matter (measured).
 //   Each tile's product starts from zero and is folded into fp32 running sums with
 //   round-to-nearest FMAs, so tensor-core accumulation rounding never compounds
 //   beyond 32 rows.
@@ -206,10 +209,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
     // ldmatrix row addresses inside a tile.  Tile rows used by a lane are (multiple of 8) + lr, so the
     // swizzle term is (chunk ^ lr) << 4 and every address is a per-lane base xor a small constant:
-    //   K, block nb, elements 0-31:   nb*1024 + k_off        (chunks mi);  elements 32-63: the same ^ 64
-    //   V / pass 2, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
-    const uint32_t k_off = (uint32_t)(lr * kWRowBytes + ((mi ^ lr) << 4));
+    //   rows of K or V as the A operand, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
     const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
+    //   V^T (transposing loads), rows 16*a + 8*(mi>>1) + lr, chunk 2*b + (mi&1):   a*2048 + (vt_off ^ (b << 5))
+    const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
     const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     int spin_limit = kCopySpinLimit;
@@ -503,10 +506,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
         __syncwarp();
 
-        // ---- the running state; the first warp starts from the new row: weight 1 in A' row 0, its 1/|v| in row 2 ----
-        float m_run = -FLT_MAX, l_run = 0.f, o_run[8][2];
+        // ---- the running state; the first warp starts from the new row: weight 1 for role 0, its 1/|v| for role 2 ----
+        // o_run[md][0..3]: dimension 16*md + g (0, 1) and 16*md + g + 8 (2, 3), roles 2t (0, 2) and 2t + 1 (1, 3), where
+        // role 0/1 = softmax.V through P_hi / P_lo and roles 2/3/4 = s through w_hi / w_mid / w_lo.
+        float m_run = -FLT_MAX, l_run = 0.f, o_run[4][4];
 #pragma unroll
-        for (int nb = 0; nb < 8; ++nb) { o_run[nb][0] = 0.f; o_run[nb][1] = 0.f; }
+        for (int md = 0; md < 4; ++md) { o_run[md][0] = o_run[md][1] = o_run[md][2] = o_run[md][3] = 0.f; }
         if (rk == 0) {
             float s = 0.f, ss = 0.f;
 #pragma unroll
@@ -525,16 +530,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             const float inv_new = new_cand ? 1.0f / fmaxf(sqrtf(ss), kNormEps) : 0.f;
             m_run = s * c.scale_log2e;
-            l_run = t == 0 ? 1.f : 0.f;   // summed over the four t lanes at the end
-            const float wrow = g == 0 ? 1.f : g == 2 ? inv_new : 0.f;
+            l_run = g == 0 ? 1.f : 0.f;   // summed over the eight g lanes at the end
+            const float wrole = t == 0 ? 1.f : t == 1 ? inv_new : 0.f;   // role 0 in lanes t = 0, role 2 in lanes t = 1
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    int xx = 8 * nb + 2 * t + e;
-                    float vf = xx < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + xx]) : 0.f;
-                    o_run[nb][e] = wrow * vf;
-                }
+            for (int md = 0; md < 4; ++md) {
+                int x0 = 16 * md + g, x1 = x0 + 8;
+                o_run[md][0] = wrole * (x0 < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + x0]) : 0.f);
+                o_run[md][2] = wrole * (x1 < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + x1]) : 0.f);
             }
         }
 
@@ -544,95 +546,97 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (!ready) wait(smem_u32(bars + stage), (consumed / D) & 1);
             const uint32_t kb = stages_u32 + stage * kWStageBytes, vb = kb + kWTileBytes;
             const int r0 = tl * kWTile;
-            const uint32_t kw = kmask[tl] >> (2 * t);   // bit 8*nb + e: row 8*nb + 2t + e is retained
-            float sc[4][4];
+            const uint32_t kw = kmask[tl] >> g;   // bits 0, 8, 16, 24: rows g, g + 8, g + 16, g + 24 are retained
+            // S = K.q: A = 16 rows of K, B = q in every column, so every lane of a group of four holds the
+            // logits of rows 16*mb + g (c0 = c1) and 16*mb + g + 8 (c2 = c3)
+            float sc[2][4];
 #pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {   // S = q.K^T, blocks of 8 rows
-                uint32_t kf0[4], kf1[4];
-                ldsm_x4(kb + nb * 1024 + k_off, kf0);          // elements 0-31 of the 8 rows
-                ldsm_x4(kb + nb * 1024 + (k_off ^ 64u), kf1);  // elements 32-63
-                mma_bf16_z(sc[nb], qa0[0], 0u, qa2[0], 0u, kf0[0], kf0[1]);
-                mma_bf16(sc[nb], qa0[1], 0u, qa2[1], 0u, kf0[2], kf0[3]);
-                mma_bf16(sc[nb], qa0[2], 0u, qa2[2], 0u, kf1[0], kf1[1]);
-                mma_bf16(sc[nb], qa0[3], 0u, qa2[3], 0u, kf1[2], kf1[3]);
-            }
-            peek_next(tl + G < n_tiles || FUSED);
-            // this lane's 8 logits: rows 8*nb + 2t, 8*nb + 2t + 1 (the same in every lane group)
-            float x[4][2], mx = -INFINITY;
+            for (int mb = 0; mb < 2; ++mb) {
 #pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    bool kept = (kw >> (8 * nb + e)) & 1u;
-                    x[nb][e] = kept ? sc[nb][e] * c.scale_log2e : -INFINITY;
-                    mx = fmaxf(mx, x[nb][e]);
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t kf[4];
+                    ldsm_x4(kb + mb * 2048 + (v_off ^ (uint32_t)(ks << 5)), kf);
+                    if (ks == 0) mma_bf16_z(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
+                    else mma_bf16(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                 }
             }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            peek_next(tl + G < n_tiles || FUSED);
+            float x[2][2], mx = -INFINITY;   // x[mb][h]: row 16*mb + 8*h + g
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    bool kept = (kw >> (16 * mb + 8 * h)) & 1u;
+                    x[mb][h] = kept ? sc[mb][2 * h] * c.scale_log2e : -INFINITY;
+                    mx = fmaxf(mx, x[mb][h]);
+                }
+            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
             const float m_new = fmaxf(m_run, mx);
             const float corr = ex2(m_run - m_new);
             m_run = m_new;
             float psum = 0.f;
 #pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {
+            for (int mb = 0; mb < 2; ++mb) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) { x[nb][e] = ex2(x[nb][e] - m_new); psum += x[nb][e]; }
+                for (int h = 0; h < 2; ++h) { x[mb][h] = ex2(x[mb][h] - m_new); psum += x[mb][h]; }
             }
             l_run = fmaf(l_run, corr, psum);
-            // A' fragments for the two 16-row k-steps: row g of A' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0
-            uint32_t pa0[2], pa2[2];
+            // B' fragments for the two 16-row k-steps of O^T = V^T.B': column g of B' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0.
+            // The weights of rows 2t, 2t + 1 (+ 8) of a k-step sit in the lanes of groups g' = 2t and 2t + 1.
+            uint32_t pb0[2], pb2[2];
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
-                uint32_t h0 = pack_bf16(x[2 * ks][0], x[2 * ks][1]), h2 = pack_bf16(x[2 * ks + 1][0], x[2 * ks + 1][1]);
-                uint32_t l0 = pack_bf16(x[2 * ks][0] - bf16_lo(h0), x[2 * ks][1] - bf16_hi(h0));
-                uint32_t l2 = pack_bf16(x[2 * ks + 1][0] - bf16_lo(h2), x[2 * ks + 1][1] - bf16_hi(h2));
+                const float p00 = __shfl_sync(0xffffffffu, x[ks][0], 8 * t), p01 = __shfl_sync(0xffffffffu, x[ks][0], 8 * t + 4);
+                const float p10 = __shfl_sync(0xffffffffu, x[ks][1], 8 * t), p11 = __shfl_sync(0xffffffffu, x[ks][1], 8 * t + 4);
+                uint32_t h0 = pack_bf16(p00, p01), h2 = pack_bf16(p10, p11);
+                uint32_t l0 = pack_bf16(p00 - bf16_lo(h0), p01 - bf16_hi(h0));
+                uint32_t l2 = pack_bf16(p10 - bf16_lo(h2), p11 - bf16_hi(h2));
                 uint32_t w0 = 0u, w2 = 0u;
                 if constexpr (FUSED) {
                     w0 = w_role[(r0 + 16 * ks + 2 * t) >> 1];
                     w2 = w_role[(r0 + 16 * ks + 8 + 2 * t) >> 1];
                 }
-                pa0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
-                pa2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
+                pb0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
+                pb2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
             }
-            // O_tile = A'.V from zero, then folded into the running sums
-            float ot[8][4];
+            // O^T_tile = V^T.B' from zero (A = V^T through transposing ldmatrix), then folded into the running sums
+            float ot[4][4];
 #pragma unroll
-            for (int nbp = 0; nbp < 4; ++nbp) {
+            for (int md = 0; md < 4; ++md) {
                 uint32_t vf[4];
-                ldsm_x4_t(vb + (v_off ^ (uint32_t)(nbp << 5)), vf);
-                mma_bf16_z(ot[2 * nbp], pa0[0], 0u, pa2[0], 0u, vf[0], vf[1]);
-                mma_bf16_z(ot[2 * nbp + 1], pa0[0], 0u, pa2[0], 0u, vf[2], vf[3]);
+                ldsm_x4_t(vb + (vt_off ^ (uint32_t)(md << 5)), vf);
+                mma_bf16_z(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[0], pb2[0]);
             }
 #pragma unroll
-            for (int nbp = 0; nbp < 4; ++nbp) {
+            for (int md = 0; md < 4; ++md) {
                 uint32_t vf[4];
-                ldsm_x4_t(vb + 2048 + (v_off ^ (uint32_t)(nbp << 5)), vf);
-                mma_bf16(ot[2 * nbp], pa0[1], 0u, pa2[1], 0u, vf[0], vf[1]);
-                mma_bf16(ot[2 * nbp + 1], pa0[1], 0u, pa2[1], 0u, vf[2], vf[3]);
+                ldsm_x4_t(vb + 2048 + (vt_off ^ (uint32_t)(md << 5)), vf);
+                mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[1], pb2[1]);
             }
             release_and_refill();
-            const float corr_row = g < 2 ? corr : 1.0f;     // the weight sums are not softmax-scaled
+            const float corr_role = t == 0 ? corr : 1.0f;     // roles 0, 1 carry softmax weights; the weight sums are not rescaled
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                o_run[nb][0] = fmaf(o_run[nb][0], corr_row, ot[nb][0]);
-                o_run[nb][1] = fmaf(o_run[nb][1], corr_row, ot[nb][1]);
+            for (int md = 0; md < 4; ++md) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o_run[md][i] = fmaf(o_run[md][i], corr_role, ot[md][i]);
             }
         }
 
-        // ---- this warp's state: softmax.V = rows 0 + 1, s = rows 2 + 3 + 4; then the warps of the group ----
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        // ---- this warp's state: softmax.V = roles 0 + 1, s = roles 2 + 3 + 4; then the warps of the group ----
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 4);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 8);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
         {
             float *w = part + rk * 132;
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                float v0 = o_run[nb][0], v1 = o_run[nb][1];
-                float a0 = __shfl_down_sync(0xffffffffu, v0, 4), a1 = __shfl_down_sync(0xffffffffu, v1, 4);
-                float b0 = __shfl_down_sync(0xffffffffu, v0, 8), b1 = __shfl_down_sync(0xffffffffu, v1, 8);
-                const int xx = 8 * nb + 2 * t;
-                if (g == 0) { w[xx] = v0 + a0; w[xx + 1] = v1 + a1; }
-                if (g == 2) { w[64 + xx] = (v0 + a0) + b0; w[64 + xx + 1] = (v1 + a1) + b1; }
+            for (int md = 0; md < 4; ++md) {
+                const float lo0 = __shfl_down_sync(0xffffffffu, o_run[md][0], 1), lo2 = __shfl_down_sync(0xffffffffu, o_run[md][2], 1);
+                const int x0 = 16 * md + g, x1 = x0 + 8;
+                if (t == 0) { w[x0] = o_run[md][0] + o_run[md][1]; w[x1] = o_run[md][2] + o_run[md][3]; }
+                if (t == 1) { w[64 + x0] = (o_run[md][0] + o_run[md][1]) + lo0; w[64 + x1] = (o_run[md][2] + o_run[md][3]) + lo2; }
             }
             if (lane == 0) { w[128] = m_run; w[129] = l_run; }
         }
