@@ -37,8 +37,9 @@ from adsa_workloads import get_workload, late_state, pick_page_rows  # noqa: E40
 METRIC, UNIT = "image_tokens_per_s", "image-tokens/s"
 INPUT_RING_BYTES = 24 << 30   # q/k/v for all steps are kept in HBM up to this size, else a ring of steps is cycled
 
-# DRAM bytes per launch of the attention kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload; None until a capture exists for that workload.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
+# under profiles/, keyed by workload; None where no capture of the current kernel exists.
+STEP_DRAM_TRAFFIC_BYTES = {}
 ATTN_DRAM_TRAFFIC_BYTES = {}
 
 
@@ -162,7 +163,10 @@ def run_ours(args, rank, world, local_rank):
     C, HW, T0, L = w.capacity(), w.n_cells, w.n_text, w.n_layers
     K = HW if args.steps is None else max(1, args.steps)
     W = max(3, args.warmup)
-    pr = args.page_rows if args.page_rows else pick_page_rows(C, hi=128)
+    # Large pages keep a stream's rows contiguous, so that one TMA box covers a whole tile; the default is
+    # the largest divisor of the capacity up to 1024 rows (cfg4: one 572-row page per stream), which also
+    # makes a full stream occupy whole pages: pool bytes = the budget's share of dense, exactly.
+    pr = args.page_rows if args.page_rows else pick_page_rows(C, hi=1024)
     pages_per_stream = -(-C // pr)
     eng = AdsaEngine(n_layers=L, batch=w.batch, n_heads=w.n_heads, head_dim=w.head_dim, n_text=T0, grid_h=w.grid_h,
                      grid_w=w.grid_w, max_rows_per_stream=max(C, T0 + 2 * w.grid_w), page_rows=pr,
@@ -188,12 +192,24 @@ def run_ours(args, rank, world, local_rank):
         eng.token_step(T0 + g, C, q[g % ring], k[g % ring], v[g % ring], out[g & 1])
 
     # ---- warm-up generation; its last cells also time the attention kernel on its own ----------
-    M = min(8, HW)
+    M = min(8, HW // 2)
     start_generation()
-    for g in range(HW - M):
+    for g in range(HW - 2 * M):
         decode(g)
-    attn_ms, attn_launches = 0.0, 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the fused layer-step kernel on its own, cache full: L launches per cell, each a different layer's KV
+    step_ms, step_launches = 0.0, 0
+    for g in range(HW - 2 * M, HW - M):
+        torch.cuda.synchronize(dev)
+        n0 = eng.launch_count()
+        e0.record()
+        decode(g)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        step_ms += e0.elapsed_time(e1)
+        step_launches += eng.launch_count() - n0
+    rows_step = int(eng._t["n_live"].max().item())
+    attn_ms, attn_launches = 0.0, 0
     for g in range(HW - M, HW):
         cur, r = T0 + g, g % ring
         for l in range(L):
@@ -280,16 +296,29 @@ def run_ours(args, rank, world, local_rank):
 
     if rank != 0:
         return
-    # ---- roofline of the dominant kernel (attention), steady state ------------------------------
+    # ---- rooflines, steady state (cache full, one eviction per step) ----------------------------
+    # The dominant kernel is the fused layer-step (one launch per layer-step: select, attend, the next
+    # step's scores, update).  Algorithmic bytes per stream: retained rows x (K + V) + 16 B of metadata per
+    # live row (position, carried score, inverse norm read; next score written) + q, k_new, v_new, out and
+    # the new row's K and V.  The attention kernel alone (adsa_sparse_decode_attn) is reported beside it.
     peak, peak_kind = peaks()
+    d2 = w.head_dim * 2
     retained = rows_full - 1 if rows_full == C else rows_full          # one eviction per step once full
-    attn_bytes = w.streams_per_layer * (retained * 2 * w.head_dim * 2 + 4 * w.head_dim * 2)
+    step_bytes = w.streams_per_layer * (retained * 2 * d2 + rows_step * 16 + 6 * d2)
+    step_us = step_ms * 1e3 / max(1, step_launches)
+    step_gbs = step_bytes / (step_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": "fused layer-step (adsa_layer_step / adsa_token_step)", "achieved": step_gbs,
+                "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8000": step_gbs / 8000.0, "us_per_launch": step_us, "launches_timed": step_launches,
+                "algorithmic_bytes_per_launch": step_bytes, "traffic": STEP_DRAM_TRAFFIC_BYTES.get(args.workload)}
+    attn_bytes = w.streams_per_layer * (retained * 2 * d2 + 4 * d2)
     attn_us = attn_ms * 1e3 / attn_launches
     achieved = attn_bytes / (attn_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": "attn_kernel (adsa_sparse_decode_attn)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8000": achieved / 8000.0, "us_per_launch": attn_us, "launches_timed": attn_launches,
-                "algorithmic_bytes_per_launch": attn_bytes, "traffic": ATTN_DRAM_TRAFFIC_BYTES.get(args.workload)}
+    roofline_attn = {"bound": "hbm", "kernel": "attention alone (adsa_sparse_decode_attn)", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8000": achieved / 8000.0, "us_per_launch": attn_us,
+                     "launches_timed": attn_launches, "algorithmic_bytes_per_launch": attn_bytes,
+                     "traffic": ATTN_DRAM_TRAFFIC_BYTES.get(args.workload)}
 
     line = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -304,7 +333,7 @@ def run_ours(args, rank, world, local_rank):
                    "inputs": f"q/k/v ring of {ring} steps resident in HBM"},
         "us_per_layer_step": ms * 1e3 / (K * L),
         "batch_rows_per_s": tokens / (ms * 1e-3) * (w.batch / prompts),
-        "gpu_launches": launches, "clocks": clocks, "roofline": roofline,
+        "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_attn": roofline_attn,
         "kv_pool": {"peak_bytes": peak_pool_bytes, "dense_bytes": w.dense_kv_bytes(),
                     "ratio": peak_pool_bytes / w.dense_kv_bytes(), "budget_fraction": w.beta},
     }

@@ -223,7 +223,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
     };
 
-    uint32_t issued = 0, consumed = 0;   // tiles of this warp since kernel start (stage = count % D)
+    // The warp's ring positions, kept without divisions: stage to fill next, stage to read next and the
+    // parity of the barrier phase that read waits for (it flips each time the ring wraps).
+    int i_stage = 0, c_stage = 0;
+    uint32_t c_par = 0;
     int streams_done = 0;
     const int stride = gridDim.x * a.n_groups;
     for (int local = gi * gridDim.x + blockIdx.x; local < c.S; local += stride, ++streams_done) {
@@ -277,7 +280,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         };
         seek(rk);
         auto issue = [&](int u) {   // lane 0 only: this warp's u-th tile of the stream into the next free stage
-            const int stage = issued % D;
+            const int stage = i_stage;
             const int pass = u >= mt ? 1 : 0, tl = rk + (pass ? u - mt : u) * G;
             if (u == mt) seek(rk);
             const int r0 = tl * kWTile, r1 = min(n, r0 + kWTile);
@@ -314,33 +317,44 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const int tl = rk + (u >= mt ? u - mt : u) * G;
             const int rows = min(n, (tl + 1) * kWTile) - tl * kWTile;
             if (rows < kWTile) {
-                uint4 *z = reinterpret_cast<uint4 *>(ring + (issued % D) * kWStageBytes);
+                uint4 *z = reinterpret_cast<uint4 *>(ring + i_stage * kWStageBytes);
                 for (int i = rows * 8 + lane; i < kWTile * 8; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
             }
         };
         int next_issue = 0;
-        for (; next_issue < total && next_issue < D; ++next_issue, ++issued) {
+        for (; next_issue < total && next_issue < D; ++next_issue) {
             clear_tail(next_issue);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) issue(next_issue);
+            i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
         }
         // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
+        // (the reads are complete once their results have been used, which in-order issue guarantees
+        // for this thread and __syncwarp for the others; a fence is needed only after the generic-proxy
+        // stores of clear_tail)
+        const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
+        const int partial_u = partial_tl >= 0 && (partial_tl - rk) % G == 0 && partial_tl >= rk ? (partial_tl - rk) / G : -1;
         auto release_and_refill = [&]() {
-            if (next_issue < total) clear_tail(next_issue);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
             if (next_issue < total) {
+                if (partial_u >= 0 && (next_issue == partial_u || next_issue == partial_u + mt)) {
+                    clear_tail(next_issue);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                __syncwarp();
                 if (lane == 0) issue(next_issue);
-                ++next_issue; ++issued;
+                ++next_issue;
+                i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
             }
+            c_stage = c_stage + 1 == D ? 0 : c_stage + 1;   // the stage just read is done with
+            if (c_stage == 0) c_par ^= 1u;
         };
         // the barrier of the tile after the current one is tested early, so that the test's latency
         // overlaps the arithmetic; `ready` is true when that test already saw the tile complete
         bool ready = false;
         auto peek_next = [&](bool more) {
-            const uint32_t nx = consumed + 1;
-            ready = more && mbar_try_wait(smem_u32(bars + nx % D), (nx / D) & 1);
+            const int ns = c_stage + 1 == D ? 0 : c_stage + 1;
+            ready = more && mbar_try_wait(smem_u32(bars + ns), ns == 0 ? c_par ^ 1u : c_par);
         };
 
         // ---- which rows are attended, and the weights of the rows the next step scores -------------
@@ -352,18 +366,19 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
             unsigned long long my_key = 0ull;
             int my_slot = -1;
-            for (int b0 = rk; b0 < n_tiles; b0 += 4 * G) {   // four blocks per round: their loads overlap
-                int ps[4];
-                float sc[4];
+            constexpr int kRound = 10;   // blocks per round: their loads are all in flight together
+            for (int b0 = rk; b0 < n_tiles; b0 += kRound * G) {
+                int ps[kRound];
+                float sc[kRound];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kRound; ++u) {
                     const int slot = (b0 + u * G) * 32 + lane;
                     const bool live = b0 + u * G < n_tiles && slot < n;
                     ps[u] = live ? pos_g[slot] : -1;
                     sc[u] = live ? sc_g[slot] : 0.f;
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kRound; ++u) {
                     const int b = b0 + u * G;
                     if (b >= n_tiles) break;
                     const int slot = b * 32 + lane;
@@ -541,9 +556,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
 
         // ---- pass 1 --------------------------------------------------------------------------------
-        for (int tl = rk; tl < n_tiles; tl += G, ++consumed) {
-            const int stage = consumed % D;
-            if (!ready) wait(smem_u32(bars + stage), (consumed / D) & 1);
+        for (int tl = rk; tl < n_tiles; tl += G) {
+            const int stage = c_stage;
+            if (!ready) wait(smem_u32(bars + stage), c_par);
             const uint32_t kb = stages_u32 + stage * kWStageBytes, vb = kb + kWTileBytes;
             const int r0 = tl * kWTile;
             const uint32_t kw = kmask[tl] >> g;   // bits 0, 8, 16, 24: rows g, g + 8, g + 16, g + 24 are retained
@@ -701,6 +716,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             okay = __shfl_sync(0xffffffffu, okay, 0);
             __syncwarp();   // lane 0 may have written a page-table entry the others are about to read
             const float denom = (float)(p_next - 1);
+            const float rden = p_next > 1 ? 1.0f / denom : 0.0f;   // p' <= 1: every score is 0
             float *scores = c.scores + (size_t)sid * c.max_rows;
 
             // s as the B operand: columns 0, 1, 2 = its bf16 hi, mid, lo parts (s[2*lane..] sits in lane `lane`)
@@ -723,9 +739,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
 
             // ---- pass 2: dot_i = v_i . s, S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), at the row's new slot ----
-            for (int tl = rk; tl < n_tiles; tl += G, ++consumed) {
-                const int stage = consumed % D;
-                if (!ready) wait(smem_u32(bars + stage), (consumed / D) & 1);
+            for (int tl = rk; tl < n_tiles; tl += G) {
+                const int stage = c_stage;
+                if (!ready) wait(smem_u32(bars + stage), c_par);
                 const uint32_t vb = stages_u32 + stage * kWStageBytes + kWTileBytes;
                 const unsigned char *vtile = ring + stage * kWStageBytes + kWTileBytes;
                 const int r0 = tl * kWTile;
@@ -753,7 +769,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     want[i] = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
                     invv[i] = inv_s[min(row, n - 1)];
                     dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
-                    sval[i] = p_next > 1 ? (invv[i] * dotv[i] - 1.0f) / denom + 0.0f : 0.0f;
+                    sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
                     rare |= want[i] && (invv[i] >= 1.0f / kNormEps || row >= n2);
                 }
                 if (!__any_sync(0xffffffffu, rare)) {
@@ -773,7 +789,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                                 unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
                                 for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
                             }
-                            s_out = p_next > 1 ? (invv[i] * dotv[i] - invv[i] * invv[i] * ss) / denom + 0.0f : 0.0f;
+                            s_out = (invv[i] * dotv[i] - invv[i] * invv[i] * ss) * rden + 0.0f;
                         }
                         int dst = row;
                         if (row >= n2) {   // a survivor: it moves into the hole of the same rank
@@ -817,7 +833,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         ss += __shfl_xor_sync(0xffffffffu, ss, o);
                     }
                     float inv = 1.0f / fmaxf(sqrtf(ss), kNormEps);
-                    if (lane == 0) scores[last_hole] = p_next > 1 ? (inv * dot - inv * inv * ss) / denom + 0.0f : 0.0f;
+                    if (lane == 0) scores[last_hole] = (inv * dot - inv * inv * ss) * rden + 0.0f;
                 }
                 write_row(c, pt, sid, last_hole, a.k_new + (size_t)local * c.d, a.v_new + (size_t)local * c.d, a.cur_pos);
                 if (lane == 0) {
