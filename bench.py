@@ -39,8 +39,8 @@ INPUT_RING_BYTES = 24 << 30   # q/k/v for all steps are kept in HBM up to this s
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/, keyed by workload; None where no capture of the current kernel exists.
-STEP_DRAM_TRAFFIC_BYTES = {}
-ATTN_DRAM_TRAFFIC_BYTES = {}
+STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 104699904 + 4275456}    # profiles/step_kernel_cfg4_2layers.md
+ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94049024 + 4710144}     # profiles/attn_kernel_cfg4_2layers.md
 
 
 def parse_args():

@@ -912,8 +912,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
                 WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, G, fused);
                 p.n_groups = groups; p.group_warps = G; p.depth = depth;
                 p.smem_bytes = (size_t)L.per_group * groups;
-                int ctas = (c.S + groups - 1) / groups;
-                p.grid = ctas < sm_count ? ctas : sm_count;
+                p.grid = c.S < sm_count ? c.S : sm_count;   // spread the streams over every SM
                 return p;
             }
             if (group_warps > 0) break;
