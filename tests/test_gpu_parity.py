@@ -196,6 +196,27 @@ def test_repeat_runs_are_bit_identical(mode):
         assert np.array_equal(o[0], outs[0][0]) and np.array_equal(o[1], outs[0][1])
 
 
+@pytest.mark.parametrize("warps,depth", [(1, 2), (2, 2), (3, 3), (4, 2), (1, 8), (2, 0)])
+def test_tensor_core_kernel_group_sizes_and_ring_depths(warps, depth):
+    """The warp-group kernel with 1-4 warps per stream and several ring depths: a trajectory that grows,
+    fills up and evicts, on a grid whose rows are not a multiple of the 32-row tile."""
+    H = _harness()
+    w = Workload("groups", 96, 1, 2, 3, 64, 40, 12, 11, 0.55, 1.0)
+    C = w.capacity()
+    for fused in (True, False):
+        eng = H.engine_for(w, capacity=C, page_rows=13)
+        eng.set_staged(4)
+        eng.set_stream_warps(warps)
+        eng.set_ring_stages(depth)
+        lh = H.LayerHarness(eng, 0, oracle_cap=w.l_max + 1, fused=fused)
+        k, v = prefix_kv(w, 4, 0)
+        lh.prefill(k, v, 0)
+        for g in range(w.n_cells):
+            q, kn, vn = layer_step_qkv(w, 4, 0, g)
+            lh.step(q, kn, vn, w.n_text + g, C)
+        assert eng.get_status()[0] == 0 and lh.stats.steps == w.n_cells
+
+
 # ---------------------------------------------------------------------------
 # the one-call and host-buffer entry points agree with the four separate calls
 # ---------------------------------------------------------------------------
