@@ -213,6 +213,12 @@ ADSA_API int adsa_set_staged(adsa_ctx *ctx, int mode);
  * streams per SM and the shared memory the configuration needs. */
 ADSA_API int adsa_set_stream_warps(adsa_ctx *ctx, int warps);
 
+/* 1 (default): the fused tensor-core kernel scores the next step's rows during its attention sweep
+ * whenever the sum of normalised rows carried in from the previous step can be updated in closed form
+ * (no eviction, or one; no rows leaving the local window); 0: it always makes a second sweep over V.
+ * Same results up to rounding of the carried sum. */
+ADSA_API int adsa_set_single_sweep(adsa_ctx *ctx, int enabled);
+
 /* Cap the tile ring (per CTA of the persistent kernel, per warp of the tensor-core kernel) at
  * max_stages stages (0 = as many as fit). */
 ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);

@@ -23,12 +23,13 @@ struct LayerState {
     int budget = 0;
     int rows_hi = 0;   // upper bound of n_live over the layer's streams
     int scores_pos = -1;  // the carried scores (DevCtx::scores) are Eq. 2 for a step at this position; -1 = stale
+    int svec_pos = -1;    // the carried sum of normalised rows (DevCtx::svec) belongs to that position too; -1 = none
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, evict_slots, counts, partials, tickets, status, staging, total;
+    size_t scores, keep_mask, evict_slots, counts, partials, tickets, svec, status, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -44,6 +45,7 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.counts = off;      off = align_up(off + S * 4 * sizeof(int32_t), 256);
     w.partials = off;    off = align_up(off + S * kMaxSplits * (size_t)(cfg.row_stride + 2) * sizeof(float), 256);
     w.tickets = off;     off = align_up(off + S * sizeof(int32_t), 256);
+    w.svec = off;        off = align_up(off + S * (size_t)cfg.n_layers * 256 * sizeof(float), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
     w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
@@ -91,6 +93,7 @@ struct adsa_ctx {
     WStepMaps maps;
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int stream_warps = 0;  // warps per stream of the warp-group kernel (0 = automatic)
+    int no_single_sweep = 0;  // 1: the fused tensor-core kernel always makes its second sweep (tests, comparisons)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -183,10 +186,11 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
 
 cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fused, int layer, int cur_pos,
                           int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                          float *out_f32, cudaStream_t st)
+                          float *out_f32, cudaStream_t st, bool have_svec = false)
 {
     if (ch.wp.n_groups)
-        return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
+        return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st,
+                            have_svec && !ctx->no_single_sweep);
     if (ch.pp.n_stages)
         return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
     return launch_step(ctx->dev, ch.sp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
@@ -250,6 +254,7 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.counts = (int32_t *)(w + ws.counts);
     d.partials = (float *)(w + ws.partials);
     d.tickets = (int32_t *)(w + ws.tickets);
+    d.svec = (float *)(w + ws.svec);
     d.status = (uint32_t *)(w + ws.status);
     d.d = cfg->head_dim;
     d.row_stride = cfg->row_stride;
@@ -317,6 +322,7 @@ int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, co
     if (!pool_can_hold(ctx, layer, L.rows_hi + n_rows)) return ADSA_ENOMEM;
     L.rows_hi += n_rows;
     L.scores_pos = -1;
+    L.svec_pos = -1;
     ++ctx->launches;
     return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
 }
@@ -335,6 +341,7 @@ int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, 
     if (!pool_can_hold(ctx, layer, hi)) return ADSA_ENOMEM;
     L.rows_hi = hi;
     L.scores_pos = -1;
+    L.svec_pos = -1;
     int sid = (layer * ctx->cfg.batch + b) * ctx->cfg.n_heads + h;
     ++ctx->launches;
     return cuda_fail(ctx, launch_set_rows(ctx->dev, sid, k, v, pos, n_rows, (cudaStream_t)stream));
@@ -355,6 +362,7 @@ int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_st
         return cuda_fail(ctx, launch_scores_copy(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
     }
     L.scores_pos = cur_pos;
+    L.svec_pos = -1;   // the stand-alone score kernel does not leave the sum behind
     ++ctx->launches;
     return cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
 }
@@ -411,6 +419,7 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
     L.rows_hi = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
     L.phase = kIdle;
     L.scores_pos = -1;   // rows move and the scores of the next step were not computed
+    L.svec_pos = -1;
     ++ctx->launches;
     return cuda_fail(ctx, launch_kv_update(ctx->dev, layer, cur_pos, k_new, v_new, (cudaStream_t)stream));
 }
@@ -443,16 +452,19 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (!pool_can_hold(ctx, layer, after > L.rows_hi ? after : L.rows_hi)) return ADSA_ENOMEM;
     if (L.phase == kIdle && L.scores_pos != cur_pos) {   // no scores carried in (first step, or the cache was rewritten)
         ++ctx->launches;
+        L.svec_pos = -1;
         rc = cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, nullptr, (cudaStream_t)stream));
         if (rc) return rc;
     }
+    const bool have_svec = L.svec_pos == cur_pos;
     ++ctx->launches;
     rc = cuda_fail(ctx, launch_staged(ctx, ch, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
-                                      (cudaStream_t)stream));
+                                      (cudaStream_t)stream, have_svec));
     L.rows_hi = after;
     L.phase = kIdle;
     L.cur_pos = cur_pos;
     L.scores_pos = cur_pos + 1;   // the fused kernel left the scores of the next position behind
+    L.svec_pos = ch.wp.n_groups ? cur_pos + 1 : -1;   // ... and the tensor-core kernel the sum they were made from
     return rc;
 }
 
@@ -548,6 +560,13 @@ int adsa_set_stream_warps(adsa_ctx *ctx, int warps)
 {
     if (!ctx || warps < 0 || warps > 4) return ADSA_EINVAL;
     ctx->stream_warps = warps;
+    return ADSA_OK;
+}
+
+int adsa_set_single_sweep(adsa_ctx *ctx, int enabled)
+{
+    if (!ctx) return ADSA_EINVAL;
+    ctx->no_single_sweep = enabled ? 0 : 1;
     return ADSA_OK;
 }
 

@@ -32,6 +32,7 @@ struct DevCtx {
     int32_t *counts;        // [S][4]            p, evicted, retained, K
     float *partials;        // [S][kMaxSplits][partial_stride]
     int32_t *tickets;       // [S]
+    float *svec;            // [n_layers * S][256]  s = sum of the normalised V rows the next step scores (carried with the scores)
     uint32_t *status;       // [1]
     int d, row_stride, page_rows, n_pages, max_rows, max_pages, mask_words, S;
     int partial_stride;     // floats per split partial: row_stride + 2 (m, l)

@@ -157,6 +157,7 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
 struct WStepArgs {
     int layer, cur_pos, budget_rows, depth;
     int group_warps, n_groups;   // warps per stream, groups per CTA
+    int have_svec;               // the sum of normalised rows of this step's previous region was carried in
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
     float *out_f32;
@@ -246,10 +247,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
         }
+        float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
+        if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
         const int n_tiles = (n + kWTile - 1) / kWTile;
         const int mt = rk < n_tiles ? (n_tiles - rk + G - 1) / G : 0;   // this warp's tiles: rk, rk + G, ...
-        const int total = FUSED ? 2 * mt : mt;                          // pass 1 tiles, then pass 2 tiles (V only)
+        int total = mt;   // pass 1 tiles; the fused kernel adds pass 2 tiles (V only) unless it can score during pass 1
         const float *inv_s = nullptr;
         if constexpr (FUSED) {
             // inverse norms into shared memory: aligned interior by bulk copy, ragged ends by plain loads
@@ -357,9 +360,97 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             ready = more && mbar_try_wait(smem_u32(bars + ns), ns == 0 ? c_par ^ 1u : c_par);
         };
 
+        // s (lane-distributed: s[2*lane], s[2*lane + 1]) as the B operand of the score product: columns
+        // 0, 1, 2 = its bf16 hi, mid, lo parts
+        uint32_t sb0[4] = {0u, 0u, 0u, 0u}, sb1[4] = {0u, 0u, 0u, 0u};
+        auto make_sb = [&](float s0, float s1) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const int e0 = 16 * ks + 2 * t;   // elements e0, e0 + 1 live in lane e0 / 2; e0 + 8, e0 + 9 in lane e0 / 2 + 4
+                float v[4] = {__shfl_sync(0xffffffffu, s0, e0 >> 1), __shfl_sync(0xffffffffu, s1, e0 >> 1),
+                              __shfl_sync(0xffffffffu, s0, (e0 >> 1) + 4), __shfl_sync(0xffffffffu, s1, (e0 >> 1) + 4)};
+                float pr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float h = __bfloat162float(__float2bfloat16_rn(v[i]));
+                    float md = __bfloat162float(__float2bfloat16_rn(v[i] - h));
+                    float lo = __bfloat162float(__float2bfloat16_rn(v[i] - h - md));
+                    pr[i] = g == 0 ? h : g == 1 ? md : g == 2 ? lo : 0.f;
+                }
+                sb0[ks] = pack_bf16(pr[0], pr[1]);
+                sb1[ks] = pack_bf16(pr[2], pr[3]);
+            }
+        };
+        // Eq. 1-2 for the next step on one tile of V rows: dot_i = v_i . s by MMA,
+        // S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), written at the row's new slot
+        int list_ns = 0, n2 = n;   // survivors of the general compaction; live rows after the update
+        float rden = 0.f;
+        auto score_tile = [&](uint32_t vb, const unsigned char *vtile, int tl, uint32_t cw) {
+            float *scores = c.scores + (size_t)sid * c.max_rows;
+            int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
+            const int r0 = tl * kWTile;
+            float dt[2][4];
+#pragma unroll
+            for (int mbk = 0; mbk < 2; ++mbk) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t af[4];
+                    ldsm_x4(vb + mbk * 2048 + (v_off ^ (uint32_t)(ks << 5)), af);
+                    if (ks == 0) mma_bf16_z(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                    else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                }
+            }
+            // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
+            float sval[4], invv[4], dotv[4];
+            bool want[4], rare = false;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int mbk = i >> 1, hh = i & 1;
+                const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
+                const int row = r0 + 16 * mbk + 8 * hh + g;
+                want[i] = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
+                invv[i] = inv_s[min(row, n - 1)];
+                dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
+                sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
+                rare |= want[i] && (invv[i] >= 1.0f / kNormEps || row >= n2);
+            }
+            if (!__any_sync(0xffffffffu, rare)) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (!want[i]) continue;
+                    const int mbk = i >> 1, hh = i & 1, row = r0 + 16 * mbk + 8 * hh + g;
+                    float s_out = sval[i];
+                    if (invv[i] >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
+                        float ss = 0.f;
+                        for (int ch = 0; ch < 8; ++ch) {
+                            float f[8];
+                            unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
+                            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+                        }
+                        s_out = (invv[i] * dotv[i] - invv[i] * invv[i] * ss) * rden + 0.0f;
+                    }
+                    int dst = row;
+                    if (row >= n2) {   // a survivor: it moves into the hole of the same rank
+                        int lo_i = 0, hi_i = list_ns - 1;
+                        while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
+                        dst = holes[lo_i];
+                    }
+                    scores[dst] = s_out;
+                }
+            }
+        };
+
         // ---- which rows are attended, and the weights of the rows the next step scores -------------
         // Each warp of the group looks at the 32-row blocks it will also sweep (rk, rk + G, ...).
-        int n2 = n, p_next = 0, n_evict = 0, evict_slot = -1;
+        int p_next = 0, n_evict = 0, evict_slot = -1;
+        // Single sweep: when the next step's previous region is this step's minus the evicted row (no
+        // row leaves the local window, at most one eviction), its sum of normalised rows is the carried
+        // sum minus that row, known before the sweep, and the next scores are taken during pass 1.
+        bool single = false;
         if constexpr (FUSED) {
             const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
             const float *sc_g = c.scores + (size_t)sid * c.max_rows;
@@ -497,6 +588,19 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             p_next += new_cand ? 1 : 0;
+            single = a.have_svec && !general && n_evict <= 1 && n_cand_np == 0 && !new_cand;
+            if (!single) total = 2 * mt;
+            rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;   // p' <= 1: every score is 0
+            if (single) {
+                float sp0 = st0, sp1 = st1;
+                if (evict_slot >= 0) {   // s' = s - u_e: the evicted row leaves the previous region
+                    const uint32_t ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
+                    const float inv_e = inv_s[evict_slot];
+                    sp0 = fmaf(-inv_e, bf16_lo(ve), sp0);
+                    sp1 = fmaf(-inv_e, bf16_hi(ve), sp1);
+                }
+                make_sb(sp0, sp1);
+            }
             __syncwarp();
             // w = 1/|v| for the retained rows the next step scores, as three bf16 parts (24 bits); they
             // take the place of the keys, which nobody reads any more
@@ -575,7 +679,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     else mma_bf16(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                 }
             }
-            peek_next(tl + G < n_tiles || FUSED);
+            peek_next(tl + G < n_tiles || (FUSED && !single));
             float x[2][2], mx = -INFINITY;   // x[mb][h]: row 16*mb + 8*h + g
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
@@ -631,6 +735,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 ldsm_x4_t(vb + 2048 + (vt_off ^ (uint32_t)(md << 5)), vf);
                 mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[1], pb2[1]);
             }
+            if constexpr (FUSED) {
+                if (single) score_tile(vb, ring + stage * kWStageBytes + kWTileBytes, tl, n2 <= c.max_rows ? cmask[tl] : 0u);
+            }
             release_and_refill();
             const float corr_role = t == 0 ? corr : 1.0f;     // roles 0, 1 carry softmax weights; the weight sums are not rescaled
 #pragma unroll
@@ -684,6 +791,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
 
         if constexpr (FUSED) {
+            if (rk == 0) {   // carried to the next step together with the scores
+                c.svec[(size_t)sid * 256 + 2 * lane] = sv0;
+                c.svec[(size_t)sid * 256 + 2 * lane + 1] = sv1;
+            }
             // ---- Section 4.2 bookkeeping: holes below the new length, survivors above it ----------
             int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;   // keys are dead now
             int nh = 1, ns = 0, last_hole = n;   // nothing evicted: the new row goes to the end
@@ -706,6 +817,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 __syncwarp();
                 last_hole = nh > ns && nh > 0 ? holes[ns] : n;
             }
+            list_ns = ns;
             const int have = (n + c.page_rows - 1) / c.page_rows, need = (n2 + c.page_rows - 1) / c.page_rows;
             int okay = 1;
             if (lane == 0) {
@@ -715,92 +827,19 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             okay = __shfl_sync(0xffffffffu, okay, 0);
             __syncwarp();   // lane 0 may have written a page-table entry the others are about to read
-            const float denom = (float)(p_next - 1);
-            const float rden = p_next > 1 ? 1.0f / denom : 0.0f;   // p' <= 1: every score is 0
             float *scores = c.scores + (size_t)sid * c.max_rows;
 
-            // s as the B operand: columns 0, 1, 2 = its bf16 hi, mid, lo parts (s[2*lane..] sits in lane `lane`)
-            uint32_t sb0[4], sb1[4];
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const int e0 = 16 * ks + 2 * t;   // elements e0, e0 + 1 live in lane e0 / 2; e0 + 8, e0 + 9 in lane e0 / 2 + 4
-                float v[4] = {__shfl_sync(0xffffffffu, sv0, e0 >> 1), __shfl_sync(0xffffffffu, sv1, e0 >> 1),
-                              __shfl_sync(0xffffffffu, sv0, (e0 >> 1) + 4), __shfl_sync(0xffffffffu, sv1, (e0 >> 1) + 4)};
-                float pr[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float h = __bfloat162float(__float2bfloat16_rn(v[i]));
-                    float md = __bfloat162float(__float2bfloat16_rn(v[i] - h));
-                    float lo = __bfloat162float(__float2bfloat16_rn(v[i] - h - md));
-                    pr[i] = g == 0 ? h : g == 1 ? md : g == 2 ? lo : 0.f;
+            if (!single) {
+                // ---- pass 2: the next step's scores from a second sweep over V, against the sum just completed ----
+                make_sb(sv0, sv1);
+                for (int tl = rk; tl < n_tiles; tl += G) {
+                    const int stage = c_stage;
+                    if (!ready) wait(smem_u32(bars + stage), c_par);
+                    peek_next(tl + G < n_tiles);
+                    score_tile(stages_u32 + stage * kWStageBytes + kWTileBytes, ring + stage * kWStageBytes + kWTileBytes, tl,
+                               okay ? cmask[tl] : 0u);
+                    release_and_refill();
                 }
-                sb0[ks] = pack_bf16(pr[0], pr[1]);
-                sb1[ks] = pack_bf16(pr[2], pr[3]);
-            }
-
-            // ---- pass 2: dot_i = v_i . s, S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), at the row's new slot ----
-            for (int tl = rk; tl < n_tiles; tl += G) {
-                const int stage = c_stage;
-                if (!ready) wait(smem_u32(bars + stage), c_par);
-                const uint32_t vb = stages_u32 + stage * kWStageBytes + kWTileBytes;
-                const unsigned char *vtile = ring + stage * kWStageBytes + kWTileBytes;
-                const int r0 = tl * kWTile;
-                const uint32_t cw = okay ? cmask[tl] : 0u;
-                float dt[2][4];
-#pragma unroll
-                for (int mbk = 0; mbk < 2; ++mbk) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        uint32_t af[4];
-                        ldsm_x4(vb + mbk * 2048 + (v_off ^ (uint32_t)(ks << 5)), af);
-                        if (ks == 0) mma_bf16_z(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
-                        else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
-                    }
-                }
-                peek_next(tl + G < n_tiles);
-                // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
-                float sval[4], invv[4], dotv[4];
-                bool want[4], rare = false;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int mbk = i >> 1, hh = i & 1;
-                    const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
-                    const int row = r0 + 16 * mbk + 8 * hh + g;
-                    want[i] = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
-                    invv[i] = inv_s[min(row, n - 1)];
-                    dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
-                    sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
-                    rare |= want[i] && (invv[i] >= 1.0f / kNormEps || row >= n2);
-                }
-                if (!__any_sync(0xffffffffu, rare)) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if (!want[i]) continue;
-                        const int mbk = i >> 1, hh = i & 1, row = r0 + 16 * mbk + 8 * hh + g;
-                        float s_out = sval[i];
-                        if (invv[i] >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
-                            float ss = 0.f;
-                            for (int ch = 0; ch < 8; ++ch) {
-                                float f[8];
-                                unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
-                                for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-                            }
-                            s_out = (invv[i] * dotv[i] - invv[i] * invv[i] * ss) * rden + 0.0f;
-                        }
-                        int dst = row;
-                        if (row >= n2) {   // a survivor: it moves into the hole of the same rank
-                            int lo_i = 0, hi_i = ns - 1;
-                            while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
-                            dst = holes[lo_i];
-                        }
-                        scores[dst] = s_out;
-                    }
-                }
-                release_and_refill();
             }
             group_sync();   // every warp's copies of this stream have landed before rows move or pages are freed
 
@@ -923,9 +962,10 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                         float *out_f32, cudaStream_t st)
+                         float *out_f32, cudaStream_t st, bool have_svec)
 {
     WStepArgs a;
+    a.have_svec = have_svec ? 1 : 0;
     a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
     a.group_warps = plan.group_warps; a.n_groups = plan.n_groups;
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;

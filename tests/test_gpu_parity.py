@@ -15,10 +15,12 @@ def _harness():
     return harness
 
 
-MODES = ["calls", "fused", "streaming", "cluster-calls", "cluster-fused", "cores-calls", "cores-fused"]
+MODES = ["calls", "fused", "two-sweep-fused", "streaming", "cluster-calls", "cluster-fused", "cores-calls", "cores-fused"]
 # calls: the four C-ABI calls one by one (attention by the persistent pipelined kernel, tensor-core
 #        arithmetic where the pool rows are 64 elements wide);
 # fused: adsa_layer_step, one persistent kernel per layer-step, scores carried from step to step;
+# two-sweep-fused: the fused kernel always scoring in a second sweep over V (by default it scores during the
+#        attention sweep whenever the carried sum of normalised rows can be updated in closed form);
 # streaming: the four calls with the staged kernels switched off (the register-streaming attention);
 # cluster-*: the same two ways of calling, with the one-cluster-per-stream kernel;
 # cores-*: the same, with the persistent kernel forced onto the CUDA cores.
@@ -31,6 +33,8 @@ def _apply_mode(eng, mode):
         eng.set_staged(2)
     elif mode.startswith("cores"):
         eng.set_staged(3)
+    elif mode.startswith("two-sweep"):
+        eng.set_single_sweep(False)
     return mode.endswith("fused")
 
 
@@ -132,7 +136,7 @@ def test_config2_full_trajectory(layer, mode):
     (5, 0.5, 8, 2),
     (5, 0.75, 6, 2),
 ])
-@pytest.mark.parametrize("mode", ["calls", "fused", "cluster-fused"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused", "cluster-fused"])
 def test_full_size_layer_steps(cfg, beta, n_sample, steps, mode):
     """One layer at the full size of configs 3-5, in the launch configuration the benchmark
     times, from a seeded late-generation state (cache full); the oracle follows a sample of streams."""
