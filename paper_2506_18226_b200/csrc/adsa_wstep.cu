@@ -247,6 +247,23 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
         }
+        constexpr int kRound = 10;   // 32-row blocks whose selection inputs are fetched together
+        int ps0[kRound];
+        float sc0[kRound];
+        if constexpr (FUSED) {
+            // positions and carried scores of this warp's first blocks: requested before n is known (the
+            // arrays hold max_rows entries per stream, whatever n is), so that one memory latency covers
+            // every load of the prologue
+            const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
+            const float *sc_g = c.scores + (size_t)sid * c.max_rows;
+#pragma unroll
+            for (int u = 0; u < kRound; ++u) {
+                const int slot = (rk + u * G) * 32 + lane;
+                const bool in = slot < c.max_rows;
+                ps0[u] = in ? pos_g[slot] : -1;
+                sc0[u] = in ? sc_g[slot] : 0.f;
+            }
+        }
         float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
         if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
@@ -385,11 +402,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), written at the row's new slot
         int list_ns = 0, n2 = n;   // survivors of the general compaction; live rows after the update
         float rden = 0.f;
-        auto score_tile = [&](uint32_t vb, const unsigned char *vtile, int tl, uint32_t cw) {
-            float *scores = c.scores + (size_t)sid * c.max_rows;
-            int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
-            const int r0 = tl * kWTile;
-            float dt[2][4];
+        // (two halves, so that the products can be issued early and their results used later)
+        auto score_mma = [&](uint32_t vb, float (&dt)[2][4]) {
 #pragma unroll
             for (int mbk = 0; mbk < 2; ++mbk) {
 #pragma unroll
@@ -400,6 +414,11 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                 }
             }
+        };
+        auto score_write = [&](const float (&dt)[2][4], const unsigned char *vtile, int tl, uint32_t cw) {
+            float *scores = c.scores + (size_t)sid * c.max_rows;
+            int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
+            const int r0 = tl * kWTile;
             // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
             float sval[4], invv[4], dotv[4];
             bool want[4], rare = false;
@@ -457,12 +476,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
             unsigned long long my_key = 0ull;
             int my_slot = -1;
-            constexpr int kRound = 10;   // blocks per round: their loads are all in flight together
-            for (int b0 = rk; b0 < n_tiles; b0 += kRound * G) {
+            for (int b0 = rk; b0 < n_tiles; b0 += kRound * G) {   // kRound blocks per round: their loads overlap
                 int ps[kRound];
                 float sc[kRound];
 #pragma unroll
                 for (int u = 0; u < kRound; ++u) {
+                    if (b0 == rk) { ps[u] = ps0[u]; sc[u] = sc0[u]; continue; }   // the first round came with the prologue
                     const int slot = (b0 + u * G) * 32 + lane;
                     const bool live = b0 + u * G < n_tiles && slot < n;
                     ps[u] = live ? pos_g[slot] : -1;
@@ -485,8 +504,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     }
                     if (live) sm_keys[slot] = key;
                     const unsigned bp = __ballot_sync(0xffffffffu, is_prev), bc = __ballot_sync(0xffffffffu, is_cand);
-                    mine.n_pre += __popc(__ballot_sync(0xffffffffu, reg == kRegionPrefix));
-                    mine.n_loc += __popc(__ballot_sync(0xffffffffu, reg == kRegionLocal));
                     mine.p += __popc(bp);
                     mine.n_cand += __popc(bc);
                     mine.n_cand_not_prev += __popc(bc & ~bp);
@@ -502,15 +519,15 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             mine.max_key = my_key; mine.max_slot = my_slot;
             if (lane == 0) sel_part[rk] = mine;
             group_sync();
-            int n_pre = 0, n_loc = 0, p = 0, n_cand = 0, n_cand_np = 0;
+            int p = 0, n_cand = 0, n_cand_np = 0;
             unsigned long long max_key = 0ull;
             int max_slot = -1;
             for (int w = 0; w < G; ++w) {
                 const WSelPartial o = sel_part[w];
-                n_pre += o.n_pre; n_loc += o.n_loc; p += o.p; n_cand += o.n_cand; n_cand_np += o.n_cand_not_prev;
+                p += o.p; n_cand += o.n_cand; n_cand_np += o.n_cand_not_prev;
                 if (o.max_key > max_key) { max_key = o.max_key; max_slot = o.max_slot; }
             }
-            int K = a.budget_rows - n_pre - n_loc - 1;
+            int K = a.budget_rows - (n - p) - 1;   // every live row outside the previous region is kept; 1 = the new row
             K = K < 0 ? 0 : (K > p ? p : K);
             n_evict = p - K;
             n2 = n - n_evict + 1;
@@ -680,6 +697,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             peek_next(tl + G < n_tiles || (FUSED && !single));
+            float dts[2][4];   // the score products of this tile, started before the softmax arithmetic
+            if constexpr (FUSED) {
+                if (single) score_mma(vb, dts);
+            }
             float x[2][2], mx = -INFINITY;   // x[mb][h]: row 16*mb + 8*h + g
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
@@ -736,7 +757,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[1], pb2[1]);
             }
             if constexpr (FUSED) {
-                if (single) score_tile(vb, ring + stage * kWStageBytes + kWTileBytes, tl, n2 <= c.max_rows ? cmask[tl] : 0u);
+                if (single) score_write(dts, ring + stage * kWStageBytes + kWTileBytes, tl, n2 <= c.max_rows ? cmask[tl] : 0u);
             }
             release_and_refill();
             const float corr_role = t == 0 ? corr : 1.0f;     // roles 0, 1 carry softmax weights; the weight sums are not rescaled
@@ -836,8 +857,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     const int stage = c_stage;
                     if (!ready) wait(smem_u32(bars + stage), c_par);
                     peek_next(tl + G < n_tiles);
-                    score_tile(stages_u32 + stage * kWStageBytes + kWTileBytes, ring + stage * kWStageBytes + kWTileBytes, tl,
-                               okay ? cmask[tl] : 0u);
+                    float dt2[2][4];
+                    score_mma(stages_u32 + stage * kWStageBytes + kWTileBytes, dt2);
+                    score_write(dt2, ring + stage * kWStageBytes + kWTileBytes, tl, okay ? cmask[tl] : 0u);
                     release_and_refill();
                 }
             }
@@ -925,6 +947,8 @@ cudaError_t configure_wstep_kernel(const DevCtx &c)
     (void)c;
     cudaError_t e = cudaFuncSetAttribute(wstep_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     return e;
@@ -974,6 +998,9 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     if (warps <= 8) {
         if (fused) wstep_kernel<true, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
         else wstep_kernel<false, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+    } else if (warps <= 10) {   // 5 streams x 2 warps, the LlamaGen-XL shape: room for 204 registers per thread
+        if (fused) wstep_kernel<true, 10><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
+        else wstep_kernel<false, 10><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
     } else {
         if (fused) wstep_kernel<true, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
         else wstep_kernel<false, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
