@@ -264,6 +264,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 sc0[u] = in ? sc_g[slot] : 0.f;
             }
         }
+        uint32_t km0 = 0u;   // attention alone: this lane's first keep-mask word, requested with the other prologue loads
+        if constexpr (!FUSED) {
+            if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)local * c.mask_words + rk + lane * G];
+        }
         float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
         if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
@@ -635,7 +639,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         } else {
             const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {
-                uint32_t bits = gm[b];
+                uint32_t bits = b == rk + lane * G ? km0 : gm[b];
                 int valid = n - b * 32;
                 kmask[b] = valid >= 32 ? bits : (bits & ((1u << valid) - 1u));
             }
