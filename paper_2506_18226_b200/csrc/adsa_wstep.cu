@@ -200,6 +200,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         mbar_init_fence();
     }
     __syncthreads();   // the only CTA-wide barrier: every warp is still here
+    // Programmatic dependent launch: everything above touched no global memory, so it may run while the
+    // kernel launched before this one is still finishing; from here on its writes are needed.  The next
+    // kernel in the stream may then be scheduled onto SMs as this grid's CTAs leave them (it waits at the
+    // same place for this grid to complete).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     auto group_sync = [&]() {
         if (G == 1) __syncwarp();
         else asm volatile("bar.sync %0, %1;" ::"r"(1 + gi), "r"(32 * G) : "memory");
@@ -999,16 +1005,21 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
-    if (warps <= 8) {
-        if (fused) wstep_kernel<true, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-        else wstep_kernel<false, 8><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-    } else if (warps <= 10) {   // 5 streams x 2 warps, the LlamaGen-XL shape: room for 204 registers per thread
-        if (fused) wstep_kernel<true, 10><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-        else wstep_kernel<false, 10><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-    } else {
-        if (fused) wstep_kernel<true, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-        else wstep_kernel<false, 16><<<plan.grid, threads, plan.smem_bytes, st>>>(c, a, maps);
-    }
+    void (*kern)(DevCtx, WStepArgs, WStepMaps);
+    if (warps <= 8) kern = fused ? wstep_kernel<true, 8> : wstep_kernel<false, 8>;
+    else if (warps <= 10) kern = fused ? wstep_kernel<true, 10> : wstep_kernel<false, 10>;   // 5 streams x 2 warps, the LlamaGen-XL shape: room for 204 registers per thread
+    else kern = fused ? wstep_kernel<true, 16> : wstep_kernel<false, 16>;
+    // launched so that its set-up overlaps the tail of the kernel before it in the stream (the kernel
+    // itself waits for that kernel's completion before it reads or writes global memory)
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.grid); cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = plan.smem_bytes; cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, c, a, maps);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
