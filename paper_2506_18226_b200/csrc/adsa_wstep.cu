@@ -253,6 +253,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
         }
+        uint32_t qn = 0u, kn = 0u, vn = 0u;   // first warp: elements 2*lane, 2*lane + 1 of q and of the new row's K and V
+        if (rk == 0 && 2 * lane < c.d) {
+            qn = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d)[lane];
+            kn = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[lane];
+            vn = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[lane];
+        }
         constexpr int kRound = 10;   // 32-row blocks whose selection inputs are fetched together
         int ps0[kRound];
         float sc0[kRound];
@@ -486,6 +492,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
             unsigned long long my_key = 0ull;
             int my_slot = -1;
+            const bool same_cut = cut_next.lo == cut_now.lo;   // the local window does not move: candidates = previous region
             for (int b0 = rk; b0 < n_tiles; b0 += kRound * G) {   // kRound blocks per round: their loads overlap
                 int ps[kRound];
                 float sc[kRound];
@@ -505,26 +512,28 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     const bool live = slot < n;
                     const int reg = live ? region_by_cut(c, cut_now, ps[u]) : -1;
                     const bool is_prev = reg == kRegionPrevious;
-                    const bool is_cand = live && reg != kRegionInvalid && region_by_cut(c, cut_next, ps[u]) == kRegionPrevious;
                     if (live && reg == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
-                    unsigned long long key = ~0ull;
                     if (is_prev) {
-                        key = ((unsigned long long)orderable(sc[u]) << 32) | (uint32_t)ps[u];
+                        const unsigned long long key = ((unsigned long long)orderable(sc[u]) << 32) | (uint32_t)ps[u];
                         if (key > my_key) { my_key = key; my_slot = slot; }
                     }
-                    if (live) sm_keys[slot] = key;
-                    const unsigned bp = __ballot_sync(0xffffffffu, is_prev), bc = __ballot_sync(0xffffffffu, is_cand);
+                    const unsigned bp = __ballot_sync(0xffffffffu, is_prev);
+                    unsigned bc = bp;
+                    if (!same_cut)
+                        bc = __ballot_sync(0xffffffffu, live && reg != kRegionInvalid && region_by_cut(c, cut_next, ps[u]) == kRegionPrevious);
                     mine.p += __popc(bp);
                     mine.n_cand += __popc(bc);
                     mine.n_cand_not_prev += __popc(bc & ~bp);
                     if (lane == 0) { prevm[b] = bp; candm[b] = bc; }
                 }
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                unsigned long long ok = __shfl_xor_sync(0xffffffffu, my_key, o);
-                int os = __shfl_xor_sync(0xffffffffu, my_slot, o);
-                if (ok > my_key) { my_key = ok; my_slot = os; }
+            {   // the warp's largest key (keys are distinct: the low word is the position) and its slot
+                const uint32_t kh = (uint32_t)(my_key >> 32), kl = (uint32_t)my_key;
+                const uint32_t mh = __reduce_max_sync(0xffffffffu, kh);
+                const uint32_t ml = __reduce_max_sync(0xffffffffu, kh == mh ? kl : 0u);
+                const int src = __ffs(__ballot_sync(0xffffffffu, kh == mh && kl == ml)) - 1;
+                my_slot = __shfl_sync(0xffffffffu, my_slot, src);
+                my_key = ((unsigned long long)mh << 32) | ml;
             }
             mine.max_key = my_key; mine.max_slot = my_slot;
             if (lane == 0) sel_part[rk] = mine;
@@ -543,19 +552,34 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             n2 = n - n_evict + 1;
             wait(bar_meta, streams_done & 1);   // the inverse norms are in shared memory
             const bool general = K > 0 && K < p - 1;
+            single = a.have_svec && !general && n_evict <= 1 && n_cand_np == 0 && !new_cand;
+            uint32_t ve = 0u;      // single sweep: the evicted row's elements 2*lane, 2*lane + 1, requested as early as possible
+            float inv_e = 0.f;
             if (!general) {
                 if (K == p - 1 && p > 0) evict_slot = max_slot;
+                if (single && evict_slot >= 0) {
+                    ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
+                    inv_e = inv_s[evict_slot];
+                }
                 const bool drop_prev = K == 0 && p > 0;
-                for (int b = rk; b < n_tiles; b += G) {
+                for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {   // one block per lane
                     const int valid = n - b * 32;
                     uint32_t keep = valid >= 32 ? 0xffffffffu : ((1u << valid) - 1u);
                     if (drop_prev) keep &= ~prevm[b];
                     if (evict_slot >= 0 && (evict_slot >> 5) == b) keep &= ~(1u << (evict_slot & 31));
-                    if (lane == 0) { kmask[b] = keep; cmask[b] = candm[b] & keep; }
+                    kmask[b] = keep; cmask[b] = candm[b] & keep;
                 }
                 p_next = K >= p ? n_cand : drop_prev ? n_cand_np : n_cand - ((candm[evict_slot >> 5] >> (evict_slot & 31)) & 1u);
             } else {
-                // arbitrary K: radix select over all keys by the first warp, then every warp marks every block
+                // arbitrary K: the keys of all rows into shared memory (each warp its blocks), radix select
+                // over them by the first warp, then every warp marks every block
+                for (int b = rk; b < n_tiles; b += G) {
+                    const int slot = b * 32 + lane;
+                    if (slot < n)
+                        sm_keys[slot] = ((prevm[b] >> lane) & 1u)
+                                            ? ((unsigned long long)orderable(sc_g[slot]) << 32) | (uint32_t)pos_g[slot] : ~0ull;
+                }
+                group_sync();
                 if (rk == 0) {
                     unsigned long long mask = 0ull, thr = 0ull;
                     int k_rem = K;
@@ -615,19 +639,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             p_next += new_cand ? 1 : 0;
-            single = a.have_svec && !general && n_evict <= 1 && n_cand_np == 0 && !new_cand;
             if (!single) total = 2 * mt;
             rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;   // p' <= 1: every score is 0
-            if (single) {
-                float sp0 = st0, sp1 = st1;
-                if (evict_slot >= 0) {   // s' = s - u_e: the evicted row leaves the previous region
-                    const uint32_t ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
-                    const float inv_e = inv_s[evict_slot];
-                    sp0 = fmaf(-inv_e, bf16_lo(ve), sp0);
-                    sp1 = fmaf(-inv_e, bf16_hi(ve), sp1);
-                }
-                make_sb(sp0, sp1);
-            }
             __syncwarp();
             // w = 1/|v| for the retained rows the next step scores, as three bf16 parts (24 bits); they
             // take the place of the keys, which nobody reads any more
@@ -642,6 +655,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(md));
                 wsplit[slot] = h; wsplit[L.w_rows + slot] = md; wsplit[2 * L.w_rows + slot] = lo;
             }
+            if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
+                make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
         } else {
             const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {
@@ -658,31 +673,27 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         float m_run = -FLT_MAX, l_run = 0.f, o_run[4][4];
 #pragma unroll
         for (int md = 0; md < 4; ++md) { o_run[md][0] = o_run[md][1] = o_run[md][2] = o_run[md][3] = 0.f; }
+        float ss_new = 0.f, inv_row_new = 0.f;   // first warp: |v_new|^2 and 1 / max(|v_new|, eps)
         if (rk == 0) {
-            float s = 0.f, ss = 0.f;
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                int xx = 2 * lane + e;
-                float qf = xx < c.d ? __bfloat162float(a.q[(size_t)local * c.d + xx]) : 0.f;
-                float kf = xx < c.d ? __bfloat162float(a.k_new[(size_t)local * c.d + xx]) : 0.f;
-                float vf = xx < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + xx]) : 0.f;
-                s = fmaf(qf, kf, s);
-                ss = fmaf(vf, vf, ss);
-            }
+            float s = fmaf(bf16_hi(qn), bf16_hi(kn), fmaf(bf16_lo(qn), bf16_lo(kn), 0.f));
+            float ss = fmaf(bf16_hi(vn), bf16_hi(vn), fmaf(bf16_lo(vn), bf16_lo(vn), 0.f));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 s += __shfl_xor_sync(0xffffffffu, s, o);
                 ss += __shfl_xor_sync(0xffffffffu, ss, o);
             }
-            const float inv_new = new_cand ? 1.0f / fmaxf(sqrtf(ss), kNormEps) : 0.f;
+            ss_new = ss;
+            inv_row_new = 1.0f / fmaxf(sqrtf(ss), kNormEps);
+            const float inv_new = new_cand ? inv_row_new : 0.f;
             m_run = s * c.scale_log2e;
             l_run = g == 0 ? 1.f : 0.f;   // summed over the eight g lanes at the end
             const float wrole = t == 0 ? 1.f : t == 1 ? inv_new : 0.f;   // role 0 in lanes t = 0, role 2 in lanes t = 1
 #pragma unroll
             for (int md = 0; md < 4; ++md) {
-                int x0 = 16 * md + g, x1 = x0 + 8;
-                o_run[md][0] = wrole * (x0 < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + x0]) : 0.f);
-                o_run[md][2] = wrole * (x1 < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + x1]) : 0.f);
+                // elements 16*md + g and 16*md + g + 8 sit in lanes 8*md + g/2 and 8*md + g/2 + 4, half g & 1
+                const uint32_t w0 = __shfl_sync(0xffffffffu, vn, 8 * md + (g >> 1)), w1 = __shfl_sync(0xffffffffu, vn, 8 * md + (g >> 1) + 4);
+                o_run[md][0] = wrole * ((g & 1) ? bf16_hi(w0) : bf16_lo(w0));
+                o_run[md][2] = wrole * ((g & 1) ? bf16_hi(w1) : bf16_lo(w1));
             }
         }
 
@@ -890,24 +901,23 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     }
                 }
                 if (new_cand) {   // the new row's own score for the next step
-                    float dot = 0.f, ss = 0.f;
+                    float dot = fmaf(bf16_hi(vn), sv1, fmaf(bf16_lo(vn), sv0, 0.f));
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        int xx = 2 * lane + e;
-                        float vf = xx < c.d ? __bfloat162float(a.v_new[(size_t)local * c.d + xx]) : 0.f;
-                        dot = fmaf(vf, e == 0 ? sv0 : sv1, dot);
-                        ss = fmaf(vf, vf, ss);
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                        ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                    }
-                    float inv = 1.0f / fmaxf(sqrtf(ss), kNormEps);
-                    if (lane == 0) scores[last_hole] = (inv * dot - inv * inv * ss) * rden + 0.0f;
+                    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    if (lane == 0) scores[last_hole] = (inv_row_new * dot - inv_row_new * inv_row_new * ss_new) * rden + 0.0f;
                 }
-                write_row(c, pt, sid, last_hole, a.k_new + (size_t)local * c.d, a.v_new + (size_t)local * c.d, a.cur_pos);
+                {   // the new row, from the registers that hold it since the prologue (zero beyond d)
+                    if (need > have) {   // the page table grew: take the new entries
+                        for (int pg = have + lane; pg < need; pg += 32) pt_s[pg] = pt[pg];
+                        __syncwarp();
+                    }
+                    const size_t off = row_offset(c, pt_s, last_hole);
+                    *reinterpret_cast<uint32_t *>(c.k_pool + off + 2 * lane) = kn;
+                    *reinterpret_cast<uint32_t *>(c.v_pool + off + 2 * lane) = vn;
+                }
                 if (lane == 0) {
+                    c.pos[(size_t)sid * c.max_rows + last_hole] = a.cur_pos;
+                    c.inv_norm[(size_t)sid * c.max_rows + last_hole] = inv_row_new;
                     if (need < have) resize_pages(c, pt, have, need);
                     c.n_live[sid] = n2;
                 }
