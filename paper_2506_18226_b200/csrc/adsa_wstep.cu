@@ -199,6 +199,34 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         if (rk == 0) mbar_init(bar_meta, 1);
         mbar_init_fence();
     }
+    {
+        // The first stream's metadata is asked into L2 now.  A prefetch changes no state that a program can
+        // see, so it may run before the kernel launched ahead of this one has completed; the loads after
+        // the wait below then find their lines (and their address translations) close by.
+        const int local0 = gi * gridDim.x + blockIdx.x;
+        if (local0 < c.S && gi < a.n_groups) {
+            const int sid0 = a.layer * c.S + local0;
+            auto prefetch_span = [&](const void *ptr, size_t bytes) {
+                const char *b = reinterpret_cast<const char *>(ptr);
+                for (size_t off = (size_t)(rk * 32 + lane) * 128; off < bytes; off += (size_t)G * 32 * 128)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(b + off));
+            };
+            if (rk == 0 && lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.n_live + sid0));
+            prefetch_span(c.page_table + (size_t)sid0 * c.max_pages, (size_t)c.max_pages * 4);
+            if (rk == 0 && lane < 3) {
+                const __nv_bfloat16 *row = (lane == 0 ? a.q : lane == 1 ? a.k_new : a.v_new) + (size_t)local0 * c.d;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+            }
+            if constexpr (FUSED) {
+                prefetch_span(c.pos + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
+                prefetch_span(c.scores + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
+                prefetch_span(c.inv_norm + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
+                if (a.have_svec) prefetch_span(c.svec + (size_t)sid0 * 256, 256);
+            } else {
+                prefetch_span(c.keep_mask + (size_t)local0 * c.mask_words, (size_t)c.mask_words * 4);
+            }
+        }
+    }
     __syncthreads();   // the only CTA-wide barrier: every warp is still here
     // Programmatic dependent launch: everything above touched no global memory, so it may run while the
     // kernel launched before this one is still finishing; from here on its writes are needed.  The next
