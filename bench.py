@@ -60,6 +60,7 @@ def parse_args():
     ap.add_argument("--kernel-mode", type=int, default=1,
                     help="0 streaming, 1 automatic, 2 cluster, 3 persistent on CUDA cores, 4 persistent with MMA")
     ap.add_argument("--stream-warps", type=int, default=0, help="warps per stream of the tensor-core kernel (0 = automatic)")
+    ap.add_argument("--l2-ahead", type=int, default=-1, help="tiles per warp asked into L2 beyond the ring (-1 = automatic)")
     ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
@@ -177,6 +178,8 @@ def run_ours(args, rank, world, local_rank):
     eng.set_staged(args.kernel_mode)
     if args.ring_stages:
         eng.set_ring_stages(args.ring_stages)
+    if args.l2_ahead >= 0:
+        eng.set_l2_lookahead(args.l2_ahead)
     if args.stream_warps:
         eng.set_stream_warps(args.stream_warps)
     (q, k, v), (pk, pv), ring = make_inputs(w, HW, dev, args.seed + 1000 * rank)

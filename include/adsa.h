@@ -223,6 +223,12 @@ ADSA_API int adsa_set_single_sweep(adsa_ctx *ctx, int enabled);
  * max_stages stages (0 = as many as fit). */
 ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
 
+/* The tensor-core kernel asks the K/V tiles that come after the ones its ring holds into L2 while it is
+ * still selecting rows, so that HBM is busy before the attention sweep starts.  tiles = how many 32-row
+ * tiles per warp beyond the ring (0 = none, -1 = choose automatically, the default).  Results do not
+ * depend on it. */
+ADSA_API int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles);
+
 /* Override the rows per attention chunk (0 = choose automatically). */
 ADSA_API int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows);
 

@@ -93,6 +93,7 @@ struct adsa_ctx {
     WStepMaps maps;
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int stream_warps = 0;  // warps per stream of the warp-group kernel (0 = automatic)
+    int l2_ahead = -1;     // tiles per warp the tensor-core kernel asks into L2 ahead of its ring (-1 = automatic)
     int no_single_sweep = 0;  // 1: the fused tensor-core kernel always makes its second sweep (tests, comparisons)
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
@@ -174,6 +175,7 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     if (m == 0) return ch;
     if ((m == 1 || m == 4) && ctx->mma_ok) {
         ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages, ctx->stream_warps);
+        if (ctx->l2_ahead >= 0) ch.wp.l2_ahead = ctx->l2_ahead;
         if (ch.wp.n_groups) return ch;
     }
     if (m == 1 || m == 3) {
@@ -574,6 +576,13 @@ int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages)
 {
     if (!ctx || max_stages < 0) return ADSA_EINVAL;
     ctx->max_stages = max_stages;
+    return ADSA_OK;
+}
+
+int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles)
+{
+    if (!ctx || tiles < -1) return ADSA_EINVAL;
+    ctx->l2_ahead = tiles;
     return ADSA_OK;
 }
 

@@ -73,6 +73,7 @@ struct WStepPlan {
     int n_groups;       // streams a CTA serves at a time; 0 = not supported / does not fit
     int group_warps;    // warps that share a stream
     int depth;          // tiles in flight per warp
+    int l2_ahead;       // tiles asked into L2 beyond those in flight
     int grid;
     size_t smem_bytes;
 };

@@ -157,6 +157,7 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
 struct WStepArgs {
     int layer, cur_pos, budget_rows, depth;
     int group_warps, n_groups;   // warps per stream, groups per CTA
+    int l2_ahead;                // tiles per warp asked into L2 beyond the ring
     int have_svec;               // the sum of normalised rows of this step's previous region was carried in
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
@@ -385,6 +386,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 for (int i = rows * 8 + lane; i < kWTile * 8; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
             }
         };
+        // HBM is otherwise idle until the attention sweep starts (the ring holds `depth` tiles and the
+        // selection comes first), so the rows of the tiles after those are asked into L2 now, and one
+        // tile further with every tile consumed: the sweep then finds them in L2.
+        auto l2_ask = [&](int u) {   // this warp's u-th tile of pass 1, a row per lane
+            const int row = (rk + u * G) * kWTile + lane;
+            if (u < mt && row < n) {
+                const size_t off = row_offset(c, pt_s, row);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
+            }
+        };
         int next_issue = 0;
         for (; next_issue < total && next_issue < D; ++next_issue) {
             clear_tail(next_issue);
@@ -393,6 +405,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (lane == 0) issue(next_issue);
             i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
         }
+
+        if constexpr (FUSED) {
+            for (int u = D; u < D + a.l2_ahead; ++u) l2_ask(u);
+        }
         // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
         // (the reads are complete once their results have been used, which in-order issue guarantees
         // for this thread and __syncwarp for the others; a fence is needed only after the generic-proxy
@@ -400,6 +416,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
         const int partial_u = partial_tl >= 0 && (partial_tl - rk) % G == 0 && partial_tl >= rk ? (partial_tl - rk) / G : -1;
         auto release_and_refill = [&]() {
+            if (FUSED && a.l2_ahead > 0) l2_ask(next_issue + a.l2_ahead);
             if (next_issue < total) {
                 if (partial_u >= 0 && (next_issue == partial_u || next_issue == partial_u + mt)) {
                     clear_tail(next_issue);
@@ -1022,6 +1039,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
             if (depth >= 2 || (depth >= 1 && G == 1 && groups == 1)) {
                 WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, G, fused);
                 p.n_groups = groups; p.group_warps = G; p.depth = depth;
+                p.l2_ahead = fused ? 1 : 0;   // measured: with the ring this makes a three-deep pipeline; deeper is slower
                 p.smem_bytes = (size_t)L.per_group * groups;
                 p.grid = c.S < sm_count ? c.S : sm_count;   // spread the streams over every SM
                 return p;
@@ -1039,7 +1057,7 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     WStepArgs a;
     a.have_svec = have_svec ? 1 : 0;
     a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
-    a.group_warps = plan.group_warps; a.n_groups = plan.n_groups;
+    a.group_warps = plan.group_warps; a.n_groups = plan.n_groups; a.l2_ahead = plan.l2_ahead;
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
