@@ -226,6 +226,25 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             } else {
                 prefetch_span(c.keep_mask + (size_t)local0 * c.mask_words, (size_t)c.mask_words * 4);
             }
+            {
+                // The rows of the first tiles, too, located through a racy look at the row count and the
+                // page table (read past L1, used for nothing but these hints, and range-checked: a stale
+                // value costs a useless prefetch).
+                const int n0 = __ldcg(c.n_live + sid0);
+                const int32_t *pt0 = c.page_table + (size_t)sid0 * c.max_pages;
+                for (int u = 0; u < D + (FUSED ? a.l2_ahead : 0); ++u) {
+                    const int row = (rk + u * G) * kWTile + lane;
+                    if (row < n0 && row < c.max_rows) {
+                        const uint32_t pg = __umulhi((uint32_t)row, c.pr_magic);
+                        const int page = __ldcg(pt0 + pg);
+                        if (page >= 0 && page < c.n_pages) {
+                            const size_t off = ((size_t)page * c.page_rows + ((uint32_t)row - pg * (uint32_t)c.page_rows)) * (size_t)c.row_stride;
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
+                        }
+                    }
+                }
+            }
         }
     }
     __syncthreads();   // the only CTA-wide barrier: every warp is still here
