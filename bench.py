@@ -39,8 +39,8 @@ INPUT_RING_BYTES = 24 << 30   # q/k/v for all steps are kept in HBM up to this s
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/, keyed by workload; None where no capture of the current kernel exists.
-STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 104699904 + 4275456}    # profiles/step_kernel_cfg4_2layers.md
-ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94049024 + 4710144}     # profiles/attn_kernel_cfg4_2layers.md
+STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 98627584 + 3468544}    # profiles/step_kernel_cfg4_2layers.md
+ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94058240 + 3330176}     # profiles/attn_kernel_cfg4_2layers.md
 
 
 def parse_args():
@@ -337,8 +337,13 @@ def run_ours(args, rank, world, local_rank):
         "us_per_layer_step": ms * 1e3 / (K * L),
         "batch_rows_per_s": tokens / (ms * 1e-3) * (w.batch / prompts),
         "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_attn": roofline_attn,
+        # peak_bytes counts whole pool rows (row_stride elements: d rounded up to a 16-byte multiple);
+        # payload_bytes the d elements of each row, which is what dense_bytes counts
         "kv_pool": {"peak_bytes": peak_pool_bytes, "dense_bytes": w.dense_kv_bytes(),
-                    "ratio": peak_pool_bytes / w.dense_kv_bytes(), "budget_fraction": w.beta},
+                    "ratio": peak_pool_bytes / w.dense_kv_bytes(),
+                    "payload_bytes": peak_pool_bytes * w.head_dim // eng.cfg.row_stride,
+                    "payload_ratio": peak_pool_bytes * w.head_dim / eng.cfg.row_stride / w.dense_kv_bytes(),
+                    "row_stride": eng.cfg.row_stride, "budget_fraction": w.beta},
     }
     if e2e:
         line["e2e"] = e2e
