@@ -200,10 +200,12 @@ def test_repeat_runs_are_bit_identical(mode):
         assert np.array_equal(o[0], outs[0][0]) and np.array_equal(o[1], outs[0][1])
 
 
-@pytest.mark.parametrize("warps,depth", [(1, 2), (2, 2), (3, 3), (4, 2), (1, 8), (2, 0)])
-def test_tensor_core_kernel_group_sizes_and_ring_depths(warps, depth):
-    """The warp-group kernel with 1-4 warps per stream and several ring depths: a trajectory that grows,
-    fills up and evicts, on a grid whose rows are not a multiple of the 32-row tile."""
+@pytest.mark.parametrize("warps,depth,ahead", [(1, 2, -1), (2, 2, -1), (3, 3, -1), (4, 2, -1), (1, 8, -1), (2, 0, -1),
+                                               (2, 2, 0), (2, 2, 3), (1, 2, 5)])
+def test_tensor_core_kernel_group_sizes_and_ring_depths(warps, depth, ahead):
+    """The warp-group kernel with 1-4 warps per stream, several ring depths and several L2 look-ahead
+    distances: a trajectory that grows, fills up and evicts, on a grid whose rows are not a multiple of
+    the 32-row tile."""
     H = _harness()
     w = Workload("groups", 96, 1, 2, 3, 64, 40, 12, 11, 0.55, 1.0)
     C = w.capacity()
@@ -212,6 +214,7 @@ def test_tensor_core_kernel_group_sizes_and_ring_depths(warps, depth):
         eng.set_staged(4)
         eng.set_stream_warps(warps)
         eng.set_ring_stages(depth)
+        eng.set_l2_lookahead(ahead)
         lh = H.LayerHarness(eng, 0, oracle_cap=w.l_max + 1, fused=fused)
         k, v = prefix_kv(w, 4, 0)
         lh.prefill(k, v, 0)
