@@ -213,20 +213,29 @@ def run_ours(args, rank, world, local_rank):
         step_launches += eng.launch_count() - n0
     rows_step = int(eng._t["n_live"].max().item())
     attn_ms, attn_launches = 0.0, 0
+    call_ms = {"adsa_score": [], "adsa_select": [], "adsa_sparse_decode_attn": [], "adsa_kv_update": []}
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
     for g in range(HW - M, HW):
         cur, r = T0 + g, g % ring
+        ev[0].record()
         for l in range(L):
             eng.score(l, cur)
+        ev[1].record()
+        for l in range(L):
             eng.select(l, cur, C)
-        e0.record()
+        ev[2].record()
         for l in range(L):                          # L launches back to back, each reads a different layer's KV
             eng.sparse_decode_attn(l, cur, q[r, l], k[r, l], v[r, l], out[g & 1, l])
-        e1.record()
+        ev[3].record()
         for l in range(L):
             eng.kv_update(l, cur, k[r, l], v[r, l])
+        ev[4].record()
         torch.cuda.synchronize(dev)
-        attn_ms += e0.elapsed_time(e1)
+        attn_ms += ev[2].elapsed_time(ev[3])
         attn_launches += L
+        if g > HW - M:      # in the first of these cells the scores were left behind by the fused step: no score kernel runs
+            for i, name in enumerate(call_ms):
+                call_ms[name].append(ev[i].elapsed_time(ev[i + 1]) * 1e3 / L)
     status, _ = eng.get_status()
     assert status == 0, f"device status {status} after the warm-up generation"
     n_live = eng._t["n_live"]
@@ -251,12 +260,17 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.profiler.start()
     t0.record()
     g = first
+    cell_ev = []                                    # one event per cell: where in the generation the time goes
     for _ in range(K):
         if g == HW:                                 # K > H*W: start another generation inside the timed region
             start_generation()
             g = 0
         decode(g)
         g += 1
+        if K <= 4096:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record()
+            cell_ev.append((g - 1, e))
     t1.record()
     torch.cuda.synchronize(dev)
     if args.profiler_range:
@@ -299,6 +313,19 @@ def run_ours(args, rank, world, local_rank):
 
     if rank != 0:
         return
+    # per call (cache full, median over cells, per layer) and per cell of the timed generation
+    detail = {"per_call_us_cache_full": {n: float(np.median(v)) for n, v in call_ms.items() if v}}
+    if detail["per_call_us_cache_full"]:
+        detail["per_call_us_cache_full"]["four_call_sequence"] = float(sum(detail["per_call_us_cache_full"].values()))
+    if len(cell_ev) >= 48 and K == HW and first == 0:
+        prev, per_cell = t0, {}
+        for gcell, e in cell_ev:
+            per_cell[gcell] = prev.elapsed_time(e) * 1e3 / L
+            prev = e
+        span = lambda a: float(np.median([per_cell[i] for i in range(a, a + 16)]))
+        detail["fused_layer_step_us_by_cell"] = {"start_cells_0_15": span(0), "middle": span(HW // 2 - 8),
+                                                  "end_last_16": span(HW - 16),
+                                                  "rows_at": {"start": T0 + 1, "middle": min(C, T0 + HW // 2), "end": min(C, T0 + HW)}}
     # ---- rooflines, steady state (cache full, one eviction per step) ----------------------------
     # The dominant kernel is the fused layer-step (one launch per layer-step: select, attend, the next
     # step's scores, update).  Algorithmic bytes per stream: retained rows x (K + V) + 16 B of metadata per
@@ -337,6 +364,7 @@ def run_ours(args, rank, world, local_rank):
         "us_per_layer_step": ms * 1e3 / (K * L),
         "batch_rows_per_s": tokens / (ms * 1e-3) * (w.batch / prompts),
         "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_attn": roofline_attn,
+        "detail": detail,
         # peak_bytes counts whole pool rows (row_stride elements: d rounded up to a 16-byte multiple);
         # payload_bytes the d elements of each row, which is what dense_bytes counts
         "kv_pool": {"peak_bytes": peak_pool_bytes, "dense_bytes": w.dense_kv_bytes(),
