@@ -461,21 +461,21 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // 0, 1, 2 = its bf16 hi, mid, lo parts
         uint32_t sb0[4] = {0u, 0u, 0u, 0u}, sb1[4] = {0u, 0u, 0u, 0u};
         auto make_sb = [&](float s0, float s1) {
+            // each lane splits its own two elements (hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid)),
+            // packed in pairs; the fragments are then gathered with shuffles
+            const uint32_t ph = pack_bf16(s0, s1);
+            const float r0 = s0 - bf16_lo(ph), r1 = s1 - bf16_hi(ph);
+            const uint32_t pm = pack_bf16(r0, r1);
+            const uint32_t pl = pack_bf16(r0 - bf16_lo(pm), r1 - bf16_hi(pm));
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-                const int e0 = 16 * ks + 2 * t;   // elements e0, e0 + 1 live in lane e0 / 2; e0 + 8, e0 + 9 in lane e0 / 2 + 4
-                float v[4] = {__shfl_sync(0xffffffffu, s0, e0 >> 1), __shfl_sync(0xffffffffu, s1, e0 >> 1),
-                              __shfl_sync(0xffffffffu, s0, (e0 >> 1) + 4), __shfl_sync(0xffffffffu, s1, (e0 >> 1) + 4)};
-                float pr[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float h = __bfloat162float(__float2bfloat16_rn(v[i]));
-                    float md = __bfloat162float(__float2bfloat16_rn(v[i] - h));
-                    float lo = __bfloat162float(__float2bfloat16_rn(v[i] - h - md));
-                    pr[i] = g == 0 ? h : g == 1 ? md : g == 2 ? lo : 0.f;
-                }
-                sb0[ks] = pack_bf16(pr[0], pr[1]);
-                sb1[ks] = pack_bf16(pr[2], pr[3]);
+                const int src = 8 * ks + t;   // elements 16*ks + 2t, + 1 live in lane 8*ks + t; + 8, + 9 four lanes on
+                const uint32_t ah = __shfl_sync(0xffffffffu, ph, src), am = __shfl_sync(0xffffffffu, pm, src),
+                               al = __shfl_sync(0xffffffffu, pl, src);
+                const uint32_t bh = __shfl_sync(0xffffffffu, ph, src + 4), bm = __shfl_sync(0xffffffffu, pm, src + 4),
+                               bl = __shfl_sync(0xffffffffu, pl, src + 4);
+                sb0[ks] = g == 0 ? ah : g == 1 ? am : g == 2 ? al : 0u;
+                sb1[ks] = g == 0 ? bh : g == 1 ? bm : g == 2 ? bl : 0u;
             }
         };
         // Eq. 1-2 for the next step on one tile of V rows: dot_i = v_i . s by MMA,
@@ -709,15 +709,23 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // w = 1/|v| for the retained rows the next step scores, as three bf16 parts (24 bits); they
             // take the place of the keys, which nobody reads any more
             if (general) group_sync();
-            for (int b = rk; b < n_tiles; b += G) {
-                const int slot = b * 32 + lane;
-                const bool cand = (cmask[b] >> lane) & 1u;
-                float w = cand ? inv_s[slot] : 0.f;
-                __nv_bfloat16 h = __float2bfloat16_rn(w);
-                float r1 = w - __bfloat162float(h);
-                __nv_bfloat16 md = __float2bfloat16_rn(r1);
-                __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(md));
-                wsplit[slot] = h; wsplit[L.w_rows + slot] = md; wsplit[2 * L.w_rows + slot] = lo;
+            {
+                uint32_t *ws = reinterpret_cast<uint32_t *>(wsplit);
+                for (int i = 0; rk + i * G < n_tiles; i += 2) {   // two of the warp's blocks per trip, a pair of rows per lane
+                    const int b = rk + (i + (lane >> 4)) * G;
+                    if (b < n_tiles) {
+                        const int slot = b * 32 + 2 * (lane & 15);
+                        const uint32_t cm = cmask[b] >> (2 * (lane & 15));
+                        float w0 = 0.f, w1 = 0.f;
+                        if (cm & 1u) w0 = inv_s[slot];
+                        if (cm & 2u) w1 = inv_s[slot + 1];
+                        const uint32_t h = pack_bf16(w0, w1);
+                        const float r0 = w0 - bf16_lo(h), r1 = w1 - bf16_hi(h);
+                        const uint32_t md = pack_bf16(r0, r1);
+                        const uint32_t lo = pack_bf16(r0 - bf16_lo(md), r1 - bf16_hi(md));
+                        ws[slot >> 1] = h; ws[(L.w_rows + slot) >> 1] = md; ws[(2 * L.w_rows + slot) >> 1] = lo;
+                    }
+                }
             }
             if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
                 make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
