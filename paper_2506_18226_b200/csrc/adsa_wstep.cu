@@ -416,10 +416,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
             }
         };
+        const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
+        const int partial_u = partial_tl >= 0 && (partial_tl - rk) % G == 0 && partial_tl >= rk ? (partial_tl - rk) / G : -1;
         int next_issue = 0;
         for (; next_issue < total && next_issue < D; ++next_issue) {
-            clear_tail(next_issue);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (next_issue == partial_u) {   // generic-proxy stores into a stage are fenced before the copy that follows them
+                clear_tail(next_issue);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
             __syncwarp();
             if (lane == 0) issue(next_issue);
             i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
@@ -432,8 +436,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // (the reads are complete once their results have been used, which in-order issue guarantees
         // for this thread and __syncwarp for the others; a fence is needed only after the generic-proxy
         // stores of clear_tail)
-        const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
-        const int partial_u = partial_tl >= 0 && (partial_tl - rk) % G == 0 && partial_tl >= rk ? (partial_tl - rk) / G : -1;
         auto release_and_refill = [&]() {
             if (FUSED && a.l2_ahead > 0) l2_ask(next_issue + a.l2_ahead);
             if (next_issue < total) {
@@ -554,9 +556,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
             const float *sc_g = c.scores + (size_t)sid * c.max_rows;
             WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
-            unsigned long long my_key = 0ull;
+            uint32_t my_hi = 0u, my_lo = 0u;   // the lane's largest key so far: orderable score, position
             int my_slot = -1;
             const bool same_cut = cut_next.lo == cut_now.lo;   // the local window does not move: candidates = previous region
+            // previous region now: n_prefix <= pos < min(lo, cur); at the next step (for rows valid now): < min(lo', cur)
+            const uint32_t pre = (uint32_t)c.n_prefix;
+            const uint32_t span_now = (uint32_t)max(0, min(cut_now.lo, cut_now.cur) - c.n_prefix);
+            const uint32_t span_next = (uint32_t)max(0, min(cut_next.lo, cut_now.cur) - c.n_prefix);
             for (int b0 = rk; b0 < n_tiles; b0 += kRound * G) {   // kRound blocks per round: their loads overlap
                 int ps[kRound];
                 float sc[kRound];
@@ -574,25 +580,28 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     if (b >= n_tiles) break;
                     const int slot = b * 32 + lane;
                     const bool live = slot < n;
-                    const int reg = live ? region_by_cut(c, cut_now, ps[u]) : -1;
-                    const bool is_prev = reg == kRegionPrevious;
-                    if (live && reg == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
+                    const uint32_t pu = (uint32_t)ps[u];
+                    const bool is_prev = live && pu - pre < span_now;
+                    if (live && pu >= (uint32_t)cut_now.cur) set_status(c, ADSA_DEV_BAD_POSITION);   // negative, or not before the current position
                     if (is_prev) {
-                        const unsigned long long key = ((unsigned long long)orderable(sc[u]) << 32) | (uint32_t)ps[u];
-                        if (key > my_key) { my_key = key; my_slot = slot; }
+                        const uint32_t hi = orderable(sc[u]);
+                        if (hi > my_hi || (hi == my_hi && pu > my_lo)) { my_hi = hi; my_lo = pu; my_slot = slot; }
                     }
                     const unsigned bp = __ballot_sync(0xffffffffu, is_prev);
                     unsigned bc = bp;
-                    if (!same_cut)
-                        bc = __ballot_sync(0xffffffffu, live && reg != kRegionInvalid && region_by_cut(c, cut_next, ps[u]) == kRegionPrevious);
+                    if (!same_cut) {
+                        bc = __ballot_sync(0xffffffffu, live && pu < (uint32_t)cut_now.cur && pu - pre < span_next);
+                        mine.n_cand += __popc(bc);
+                        mine.n_cand_not_prev += __popc(bc & ~bp);
+                    }
                     mine.p += __popc(bp);
-                    mine.n_cand += __popc(bc);
-                    mine.n_cand_not_prev += __popc(bc & ~bp);
                     if (lane == 0) { prevm[b] = bp; candm[b] = bc; }
                 }
             }
+            if (same_cut) mine.n_cand = mine.p;
+            unsigned long long my_key;
             {   // the warp's largest key (keys are distinct: the low word is the position) and its slot
-                const uint32_t kh = (uint32_t)(my_key >> 32), kl = (uint32_t)my_key;
+                const uint32_t kh = my_hi, kl = my_lo;
                 const uint32_t mh = __reduce_max_sync(0xffffffffu, kh);
                 const uint32_t ml = __reduce_max_sync(0xffffffffu, kh == mh ? kl : 0u);
                 const int src = __ffs(__ballot_sync(0xffffffffu, kh == mh && kl == ml)) - 1;
