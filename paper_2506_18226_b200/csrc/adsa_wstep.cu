@@ -158,6 +158,7 @@ struct WStepArgs {
     int layer, cur_pos, budget_rows, depth;
     int group_warps, n_groups;   // warps per stream, groups per CTA
     int l2_ahead;                // tiles per warp asked into L2 beyond the ring
+    uint32_t g_magic;            // x / group_warps == __umulhi(x, g_magic) for the small x used here (group_warps > 1)
     int have_svec;               // the sum of normalised rows of this step's previous region was carried in
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
@@ -176,7 +177,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = a.group_warps, D = a.depth;
-    const int gi = warp / G, rk = warp - gi * G;      // group in the CTA, rank in the group
+    auto div_g = [&](int x) { return G == 1 ? x : (int)__umulhi((uint32_t)x, a.g_magic); };   // x / G without a division
+    const int gi = div_g(warp), rk = warp - gi * G;      // group in the CTA, rank in the group
     const WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, D, G, FUSED);
     unsigned char *smem = smem_all + (size_t)gi * L.per_group;
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + L.bars) + rk * kWMaxDepth;
@@ -332,7 +334,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
         const int n_tiles = (n + kWTile - 1) / kWTile;
-        const int mt = rk < n_tiles ? (n_tiles - rk + G - 1) / G : 0;   // this warp's tiles: rk, rk + G, ...
+        const int mt = rk < n_tiles ? div_g(n_tiles - rk + G - 1) : 0;   // this warp's tiles: rk, rk + G, ...
         int total = mt;   // pass 1 tiles; the fused kernel adds pass 2 tiles (V only) unless it can score during pass 1
         const float *inv_s = nullptr;
         if constexpr (FUSED) {
@@ -417,7 +419,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
         };
         const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
-        const int partial_u = partial_tl >= 0 && (partial_tl - rk) % G == 0 && partial_tl >= rk ? (partial_tl - rk) / G : -1;
+        const int partial_u = mt > 0 && rk + (mt - 1) * G == partial_tl ? mt - 1 : -1;   // it can only be the warp's last tile
         int next_issue = 0;
         for (; next_issue < total && next_issue < D; ++next_issue) {
             if (next_issue == partial_u) {   // generic-proxy stores into a stage are fenced before the copy that follows them
@@ -504,16 +506,18 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
             float sval[4], invv[4], dotv[4];
             bool want[4], rare = false;
+            const bool moves = n2 < n;   // more than one eviction: rows above the new length move down
+            const uint32_t cwg = t == 0 ? cw >> g : 0u;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int mbk = i >> 1, hh = i & 1;
                 const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
                 const int row = r0 + 16 * mbk + 8 * hh + g;
-                want[i] = t == 0 && ((cw >> (16 * mbk + 8 * hh + g)) & 1u);
-                invv[i] = inv_s[min(row, n - 1)];
+                want[i] = (cwg >> (16 * mbk + 8 * hh)) & 1u;
+                invv[i] = inv_s[row];   // past the last live row this reads whatever follows in shared memory: never wanted
                 dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
                 sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
-                rare |= want[i] && (invv[i] >= 1.0f / kNormEps || row >= n2);
+                rare |= want[i] && (invv[i] >= 1.0f / kNormEps || (moves && row >= n2));
             }
             if (!__any_sync(0xffffffffu, rare)) {
 #pragma unroll
@@ -894,7 +898,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             sv0 = 0.f; sv1 = 0.f;
             for (int w = 0; w < G; ++w) {
                 const float *ws = part + w * 132;
-                float wgt = exp2f(ws[128] - M);
+                float wgt = ex2(ws[128] - M);
                 Lb = fmaf(ws[129], wgt, Lb);
                 A0 = fmaf(ws[2 * lane], wgt, A0);
                 A1 = fmaf(ws[2 * lane + 1], wgt, A1);
@@ -903,7 +907,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             const int xx = 2 * lane;
             if (rk == 0 && xx < c.d) {
-                float o0 = A0 / Lb, o1 = A1 / Lb;
+                const float rl = 1.0f / Lb;
+                float o0 = A0 * rl, o1 = A1 * rl;
                 if (a.out_f32) {
                     a.out_f32[(size_t)local * c.d + xx] = o0;
                     if (xx + 1 < c.d) a.out_f32[(size_t)local * c.d + xx + 1] = o1;
@@ -941,7 +946,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 last_hole = nh > ns && nh > 0 ? holes[ns] : n;
             }
             list_ns = ns;
-            const int have = (n + c.page_rows - 1) / c.page_rows, need = (n2 + c.page_rows - 1) / c.page_rows;
+            // pages for n and for n2 rows (n2 beyond max_rows is refused below)
+            const int have = n > 0 ? (int)__umulhi((uint32_t)(n - 1), c.pr_magic) + 1 : 0;
+            const int need = (int)__umulhi((uint32_t)(min(n2, c.max_rows) - 1), c.pr_magic) + 1;
             int okay = 1;
             if (lane == 0) {
                 if (nh != ns + 1) { if (rk == 0) set_status(c, ADSA_DEV_BAD_EVICT); okay = 0; }
@@ -1094,6 +1101,7 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     a.have_svec = have_svec ? 1 : 0;
     a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
     a.group_warps = plan.group_warps; a.n_groups = plan.n_groups; a.l2_ahead = plan.l2_ahead;
+    a.g_magic = (uint32_t)((1ull << 32) / (uint32_t)plan.group_warps) + 1u;   // exact for x < 2^16 at least (group_warps <= 4)
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
