@@ -202,6 +202,23 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         if (rk == 0) mbar_init(bar_meta, 1);
         mbar_init_fence();
     }
+    // launch-wide constants (integer divisions among them) come before the dependency wait as well
+    auto group_sync = [&]() {
+        if (G == 1) __syncwarp();
+        else asm volatile("bar.sync %0, %1;" ::"r"(1 + gi), "r"(32 * G) : "memory");
+    };
+
+    const int g = lane >> 2, t = lane & 3;          // MMA fragment coordinates
+    const int mi = lane >> 3, lr = lane & 7;        // ldmatrix: matrix index, row within the matrix
+    const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
+    // ldmatrix row addresses inside a tile.  Tile rows used by a lane are (multiple of 8) + lr, so the
+    // swizzle term is (chunk ^ lr) << 4 and every address is a per-lane base xor a small constant:
+    //   rows of K or V as the A operand, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
+    const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
+    //   V^T (transposing loads), rows 16*a + 8*(mi>>1) + lr, chunk 2*b + (mi&1):   a*2048 + (vt_off ^ (b << 5))
+    const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
+    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
+    const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     {
         // The first stream's metadata is asked into L2 now.  A prefetch changes no state that a program can
         // see, so it may run before the kernel launched ahead of this one has completed; the loads after
@@ -256,22 +273,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     // same place for this grid to complete).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    auto group_sync = [&]() {
-        if (G == 1) __syncwarp();
-        else asm volatile("bar.sync %0, %1;" ::"r"(1 + gi), "r"(32 * G) : "memory");
-    };
-
-    const int g = lane >> 2, t = lane & 3;          // MMA fragment coordinates
-    const int mi = lane >> 3, lr = lane & 7;        // ldmatrix: matrix index, row within the matrix
-    const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
-    // ldmatrix row addresses inside a tile.  Tile rows used by a lane are (multiple of 8) + lr, so the
-    // swizzle term is (chunk ^ lr) << 4 and every address is a per-lane base xor a small constant:
-    //   rows of K or V as the A operand, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
-    const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
-    //   V^T (transposing loads), rows 16*a + 8*(mi>>1) + lr, chunk 2*b + (mi&1):   a*2048 + (vt_off ^ (b << 5))
-    const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
-    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
-    const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     int spin_limit = kCopySpinLimit;
     auto wait = [&](uint32_t bar, uint32_t parity) {
         if (!mbar_wait_sleepy(bar, parity, spin_limit)) {
