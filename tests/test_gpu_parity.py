@@ -97,6 +97,20 @@ def test_budget_covering_context_is_dense_attention(mode):
     assert int(eng._t["n_live"].max().item()) == w.l_max
 
 
+@pytest.mark.parametrize("preset", ["window", "window+prefix"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused", "cores-fused"])
+def test_ablation_presets_without_global_tokens(preset, mode):
+    """The comparison settings of Fig. 3 are corner cases of the same calls: a budget below prefix + window
+    makes K = 0 at every step, so the cache keeps the local window alone (no prefix configured) or the
+    prefix and the window, and nothing of the previous region."""
+    w = Workload("tiny-presets", 96, 1, 1, 4, 64, 10, 9, 7, 0.5, 1.0)
+    n_prefix = 0 if preset == "window" else w.n_text
+    lh, eng = _run_trajectory(w, 0, 4, lambda cur: 1, n_prefix=n_prefix, page_rows=8, mode=mode)
+    assert lh.stats.steps == w.n_cells
+    # after the last cell: the prefix, the grid row above, the last grid row (the new row included)
+    assert int(eng._t["n_live"].min().item()) == int(eng._t["n_live"].max().item()) == n_prefix + 2 * w.grid_w
+
+
 # ---------------------------------------------------------------------------
 # the benchmark configurations
 # ---------------------------------------------------------------------------
