@@ -38,13 +38,22 @@
 //   Each tile's product starts from zero and is folded into fp32 running sums with
 //   round-to-nearest FMAs, so tensor-core accumulation rounding never compounds
 //   beyond 32 rows.
-// Pass 2 (fused), per tile of V rows again (they come out of L2):  dot_i = v_i . s
-//   with s split into three bf16 parts as B columns 0-2;
-//   S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), Eq. 1-2 for the next step (u_i.u_i = 1
-//   unless |v_i| was clamped, in which case it is computed from the row).
+// Next step's scores (fused).  Eq. 1-2 for the next step, S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1) with
+//   dot_i = v_i . s, s = the sum of the normalised rows of the next step's previous region
+//   (u_i.u_i = 1 unless |v_i| was clamped, in which case it is computed from the row).  s itself is
+//   carried from step to step.  In the steady state the next previous region is this one minus the
+//   evicted row, so s' = s - u_e is known once the selection has named e, and every pass-1 tile also
+//   yields the scores of its rows: 4 more MMAs per 16 rows, s' split into three bf16 parts as B
+//   columns 0-2 (single sweep).  Otherwise (nothing carried in, rows leaving the local window, more
+//   than one eviction) a second sweep over V, which comes out of L2, uses the s just accumulated.
 // Then the Section 4.2 update.  All rows of a stream are copied, retained or not
 // (one row per step is not); the rows of a partial last tile that the copy does not
 // write are cleared first, so that a zero weight never meets a NaN pattern.
+//
+// Launch overlap.  The kernel is launched with programmatic stream serialization.  What touches no
+// global state (barrier set-up, launch-wide constants, L2 prefetch hints for the first stream's
+// metadata and first tiles) runs ahead of griddepcontrol.wait, i.e. under the tail of the kernel
+// before it in the stream; every load and store whose value matters comes after the wait.
 //
 // Every wait on a copy is bounded: if it runs out the warp raises
 // ADSA_DEV_COPY_TIMEOUT, shortens its later waits and runs to the end (all accesses
