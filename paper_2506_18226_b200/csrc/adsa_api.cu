@@ -95,6 +95,10 @@ struct adsa_ctx {
     int stream_warps = 0;  // warps per stream of the warp-group kernel (0 = automatic)
     int l2_ahead = -1;     // tiles per warp the tensor-core kernel asks into L2 ahead of its ring (-1 = automatic)
     int no_single_sweep = 0;  // 1: the fused tensor-core kernel always makes its second sweep (tests, comparisons)
+    // What the kernel launched last through this context may still be writing when the next one starts its
+    // set-up (launches overlap by programmatic dependent launch): the layer it served (-1 = several or
+    // unknown) and whether it writes the cache proper (rows, pages, positions, norms) / the carried scores.
+    int prev_layer = -1, prev_writes_cache = 1, prev_writes_scores = 1;
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -186,13 +190,29 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     return ch;
 }
 
+void note_launch(adsa_ctx *ctx, int layer, bool writes_cache, bool writes_scores)
+{
+    ctx->prev_layer = layer;
+    ctx->prev_writes_cache = writes_cache ? 1 : 0;
+    ctx->prev_writes_scores = writes_scores ? 1 : 0;
+}
+
+// May the kernel about to be launched read `layer`'s cache state (and, for the fused step, its carried
+// scores) before the kernel ahead of it has completed?
+bool state_is_quiet(const adsa_ctx *ctx, int layer, bool needs_scores)
+{
+    if (ctx->prev_layer < 0) return false;
+    if (ctx->prev_layer != layer) return true;
+    return !ctx->prev_writes_cache && !(needs_scores && ctx->prev_writes_scores);
+}
+
 cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fused, int layer, int cur_pos,
                           int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                           float *out_f32, cudaStream_t st, bool have_svec = false)
 {
     if (ch.wp.n_groups)
         return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st,
-                            have_svec && !ctx->no_single_sweep);
+                            have_svec && !ctx->no_single_sweep, state_is_quiet(ctx, layer, fused));
     if (ch.pp.n_stages)
         return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
     return launch_step(ctx->dev, ch.sp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
@@ -308,6 +328,7 @@ int adsa_reset(adsa_ctx *ctx, adsa_stream_t stream)
     if (!ctx) return ADSA_EINVAL;
     if (ctx->cuda_error) return ADSA_ECUDA;
     for (auto &l : ctx->layers) l = LayerState();
+    note_launch(ctx, -1, true, true);
     ++ctx->launches;
     return cuda_fail(ctx, launch_reset(ctx->dev, ctx->cfg.n_layers * ctx->dev.S, (cudaStream_t)stream));
 }
@@ -325,6 +346,7 @@ int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, co
     L.rows_hi += n_rows;
     L.scores_pos = -1;
     L.svec_pos = -1;
+    note_launch(ctx, layer, true, true);
     ++ctx->launches;
     return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
 }
@@ -345,6 +367,7 @@ int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, 
     L.scores_pos = -1;
     L.svec_pos = -1;
     int sid = (layer * ctx->cfg.batch + b) * ctx->cfg.n_heads + h;
+    note_launch(ctx, layer, true, true);
     ++ctx->launches;
     return cuda_fail(ctx, launch_set_rows(ctx->dev, sid, k, v, pos, n_rows, (cudaStream_t)stream));
 }
@@ -360,11 +383,13 @@ int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_st
     L.cur_pos = cur_pos;
     if (L.scores_pos == cur_pos) {   // carried in from the previous fused step: nothing to compute
         if (!scores_out) return ADSA_OK;
+        note_launch(ctx, layer, false, false);
         ++ctx->launches;
         return cuda_fail(ctx, launch_scores_copy(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
     }
     L.scores_pos = cur_pos;
     L.svec_pos = -1;   // the stand-alone score kernel does not leave the sum behind
+    note_launch(ctx, layer, false, true);
     ++ctx->launches;
     return cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
 }
@@ -385,6 +410,7 @@ int adsa_select(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, int32_t 
     if (!pool_can_hold(ctx, layer, after > L.rows_hi ? after : L.rows_hi)) return ADSA_ENOMEM;
     L.phase = kSelected;
     L.budget = budget_rows;
+    note_launch(ctx, layer, false, false);
     ++ctx->launches;
     return cuda_fail(ctx, launch_select(ctx->dev, layer, cur_pos, budget_rows, sel_slots, sel_pos, evict_pos, counts,
                                         (cudaStream_t)stream));
@@ -401,12 +427,15 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
     L.phase = kAttended;
     ++ctx->launches;
     StagedChoice ch = choose_staged(ctx, L.rows_hi, false);
-    if (ch.any())
-        return cuda_fail(ctx, launch_staged(ctx, ch, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32,
-                                            (cudaStream_t)stream));
-    AttnPlan plan = plan_attn(ctx, L.rows_hi);
-    return cuda_fail(ctx, launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32,
-                                      (cudaStream_t)stream));
+    cudaError_t e;
+    if (ch.any()) {
+        e = launch_staged(ctx, ch, false, layer, cur_pos, 0, q, k_new, v_new, out_bf16, out_f32, (cudaStream_t)stream);
+    } else {
+        AttnPlan plan = plan_attn(ctx, L.rows_hi);
+        e = launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32, (cudaStream_t)stream);
+    }
+    note_launch(ctx, layer, false, false);   // attention reads the cache and writes the output only
+    return cuda_fail(ctx, e);
 }
 
 int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, const void *v_new, adsa_stream_t stream)
@@ -422,6 +451,7 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
     L.phase = kIdle;
     L.scores_pos = -1;   // rows move and the scores of the next step were not computed
     L.svec_pos = -1;
+    note_launch(ctx, layer, true, false);
     ++ctx->launches;
     return cuda_fail(ctx, launch_kv_update(ctx->dev, layer, cur_pos, k_new, v_new, (cudaStream_t)stream));
 }
@@ -455,6 +485,7 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (L.phase == kIdle && L.scores_pos != cur_pos) {   // no scores carried in (first step, or the cache was rewritten)
         ++ctx->launches;
         L.svec_pos = -1;
+        note_launch(ctx, layer, false, true);
         rc = cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, nullptr, (cudaStream_t)stream));
         if (rc) return rc;
     }
@@ -462,6 +493,7 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     ++ctx->launches;
     rc = cuda_fail(ctx, launch_staged(ctx, ch, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
                                       (cudaStream_t)stream, have_svec));
+    note_launch(ctx, layer, true, true);
     L.rows_hi = after;
     L.phase = kIdle;
     L.cur_pos = cur_pos;

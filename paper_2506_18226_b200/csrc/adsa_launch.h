@@ -82,7 +82,7 @@ int build_wstep_maps(const DevCtx &c, WStepMaps *out);   // 0 on success
 WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps);
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                         float *out_f32, cudaStream_t st, bool have_svec);
+                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state);
 cudaError_t configure_wstep_kernel(const DevCtx &c);
 
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).

@@ -169,6 +169,7 @@ struct WStepArgs {
     int l2_ahead;                // tiles per warp asked into L2 beyond the ring
     uint32_t g_magic;            // x / group_warps == __umulhi(x, g_magic) for the small x used here (group_warps > 1)
     int have_svec;               // the sum of normalised rows of this step's previous region was carried in
+    int early_state;             // the cache state of this layer is not being written by the kernel ahead in the stream
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
     float *out_f32;
@@ -240,12 +241,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 for (size_t off = (size_t)(rk * 32 + lane) * 128; off < bytes; off += (size_t)G * 32 * 128)
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(b + off));
             };
-            if (rk == 0 && lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.n_live + sid0));
-            prefetch_span(c.page_table + (size_t)sid0 * c.max_pages, (size_t)c.max_pages * 4);
             if (rk == 0 && lane < 3) {
                 const __nv_bfloat16 *row = (lane == 0 ? a.q : lane == 1 ? a.k_new : a.v_new) + (size_t)local0 * c.d;
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
             }
+            if (a.early_state) {
+                // the state is read for real right away (see dep_wait below): only the inputs need hints
+                if constexpr (!FUSED) prefetch_span(c.keep_mask + (size_t)local0 * c.mask_words, (size_t)c.mask_words * 4);
+            } else {
+            if (rk == 0 && lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.n_live + sid0));
+            prefetch_span(c.page_table + (size_t)sid0 * c.max_pages, (size_t)c.max_pages * 4);
             if constexpr (FUSED) {
                 prefetch_span(c.pos + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
                 prefetch_span(c.scores + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
@@ -273,15 +278,27 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     }
                 }
             }
+            }
         }
     }
     __syncthreads();   // the only CTA-wide barrier: every warp is still here
-    // Programmatic dependent launch: everything above touched no global memory, so it may run while the
-    // kernel launched before this one is still finishing; from here on its writes are needed.  The next
-    // kernel in the stream may then be scheduled onto SMs as this grid's CTAs leave them (it waits at the
-    // same place for this grid to complete).
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Programmatic dependent launch: everything above read no value from global memory, so it may run
+    // while the kernel launched before this one is still finishing.  That kernel's writes are needed from
+    // dep_wait() on.  Normally that is here.  When the host knows that the kernel ahead does not write this
+    // layer's cache state (it served another layer; only the kernel directly ahead can still be running,
+    // because every kernel of this library waits for its predecessor before it lets its successor start),
+    // the state is read, the first tiles are requested and the rows are classified first, and the wait
+    // comes just before the caller's inputs (q, the new row, the keep mask) are touched.  After its own
+    // wait a grid lets the next kernel in the stream be scheduled onto the SMs its CTAs leave.
+    bool waited = false;
+    auto dep_wait = [&]() {
+        if (!waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            waited = true;
+        }
+    };
+    if (!a.early_state) dep_wait();
     int spin_limit = kCopySpinLimit;
     auto wait = [&](uint32_t bar, uint32_t parity) {
         if (!mbar_wait_sleepy(bar, parity, spin_limit)) {
@@ -303,8 +320,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // ---- everything that only needs addresses is requested first --------------------------------
         int n = c.n_live[sid];
         for (int pg = lane; pg < c.max_pages; pg += 32) pt_s[pg] = pt[pg];   // every warp of the group writes the same values
-        uint32_t qa0[4], qa2[4];   // q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements
-        {
+        // the caller's inputs: q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements; for the
+        // first warp elements 2*lane, 2*lane + 1 of q and of the new row's K and V; attention alone: this lane's
+        // first keep-mask word.  Requested with the other prologue loads when the dependency wait is behind us.
+        uint32_t qa0[4] = {0u, 0u, 0u, 0u}, qa2[4] = {0u, 0u, 0u, 0u};
+        uint32_t qn = 0u, kn = 0u, vn = 0u, km0 = 0u;
+        auto load_inputs = [&]() {
             const uint32_t *q2 = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d);   // c.d is even
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
@@ -312,13 +333,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 qa0[ks] = e0 < c.d ? q2[e0 >> 1] : 0u;
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
-        }
-        uint32_t qn = 0u, kn = 0u, vn = 0u;   // first warp: elements 2*lane, 2*lane + 1 of q and of the new row's K and V
-        if (rk == 0 && 2 * lane < c.d) {
-            qn = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d)[lane];
-            kn = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[lane];
-            vn = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[lane];
-        }
+            if (rk == 0 && 2 * lane < c.d) {
+                qn = q2[lane];
+                kn = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[lane];
+                vn = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[lane];
+            }
+            if constexpr (!FUSED) {
+                if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)local * c.mask_words + rk + lane * G];
+            }
+        };
+        if (waited) load_inputs();
         constexpr int kRound = 10;   // 32-row blocks whose selection inputs are fetched together
         int ps0[kRound];
         float sc0[kRound];
@@ -335,10 +359,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 ps0[u] = in ? pos_g[slot] : -1;
                 sc0[u] = in ? sc_g[slot] : 0.f;
             }
-        }
-        uint32_t km0 = 0u;   // attention alone: this lane's first keep-mask word, requested with the other prologue loads
-        if constexpr (!FUSED) {
-            if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)local * c.mask_words + rk + lane * G];
         }
         float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
         if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
@@ -613,6 +633,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             if (same_cut) mine.n_cand = mine.p;
+            if (!waited) { dep_wait(); load_inputs(); }   // the inputs arrive while the selection is completed
             unsigned long long my_key;
             {   // the warp's largest key (keys are distinct: the low word is the position) and its slot
                 const uint32_t kh = my_hi, kl = my_lo;
@@ -753,6 +774,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
                 make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
         } else {
+            if (!waited) { dep_wait(); load_inputs(); }
             const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {
                 uint32_t bits = b == rk + lane * G ? km0 : gm[b];
@@ -1105,10 +1127,11 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                         float *out_f32, cudaStream_t st, bool have_svec)
+                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state)
 {
     WStepArgs a;
     a.have_svec = have_svec ? 1 : 0;
+    a.early_state = early_state ? 1 : 0;
     a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
     a.group_warps = plan.group_warps; a.n_groups = plan.n_groups; a.l2_ahead = plan.l2_ahead;
     a.g_magic = (uint32_t)((1ull << 32) / (uint32_t)plan.group_warps) + 1u;   // exact for x < 2^16 at least (group_warps <= 4)

@@ -273,6 +273,56 @@ def test_layer_step_and_host_variant_match_separate_calls():
     assert engs[0].launch_count() - 2 == 4 * 100 and engs[1].launch_count() - 2 == 100 + 1
 
 
+def test_back_to_back_layers_match_serialised_launches():
+    """Launches of consecutive layers overlap (the next kernel's set-up, and, when the kernel ahead serves
+    another layer, its reading and selection of the cache run under the previous kernel's tail).  The
+    results must be bit-identical to the same steps with the device synchronised after every launch, for
+    the fused step and for the four separate calls, over a trajectory that fills up and evicts."""
+    H = _harness()
+    w = Workload("layers", 95, 3, 2, 3, 64, 24, 10, 9, 0.5, 1.0)
+    C, L, S, T = w.capacity(), w.n_layers, w.streams_per_layer, w.n_cells
+    qs, ks, vs = [], [], []
+    for g in range(T):
+        per = [layer_step_qkv(w, 5, l, g) for l in range(L)]
+        qs.append(torch.stack([H.dev_bf16(x[0]) for x in per]))
+        ks.append(torch.stack([H.dev_bf16(x[1]) for x in per]))
+        vs.append(torch.stack([H.dev_bf16(x[2]) for x in per]))
+    results = []
+    for variant in ("fused-free", "fused-synced", "calls-free", "calls-synced"):
+        eng = H.engine_for(w, capacity=C, page_rows=16)
+        for l in range(L):
+            k, v = prefix_kv(w, 5, l)
+            eng.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
+        outs = torch.zeros((T, L, S, w.head_dim), dtype=torch.bfloat16, device="cuda:0")
+        synced = variant.endswith("synced")
+        for g in range(T):
+            cur = w.n_text + g
+            if variant.startswith("fused"):
+                if synced:
+                    for l in range(L):
+                        eng.layer_step(l, cur, C, qs[g][l], ks[g][l], vs[g][l], outs[g, l])
+                        torch.cuda.synchronize()
+                else:
+                    eng.token_step(cur, C, qs[g], ks[g], vs[g], outs[g].view(L, w.batch, w.n_heads, w.head_dim))
+            else:
+                for l in range(L):
+                    eng.score(l, cur)
+                    eng.select(l, cur, C)
+                for l in range(L):      # attention launches of consecutive layers back to back
+                    eng.sparse_decode_attn(l, cur, qs[g][l], ks[g][l], vs[g][l], outs[g, l])
+                    if synced:
+                        torch.cuda.synchronize()
+                for l in range(L):
+                    eng.kv_update(l, cur, ks[g][l], vs[g][l])
+        assert eng.get_status()[0] == 0
+        n_live = eng._t["n_live"].cpu().numpy()
+        pos = np.sort(eng._t["pos"][:, :C].cpu().numpy(), axis=1)
+        results.append((outs.cpu(), n_live, pos))
+    for a, b in ((0, 1), (2, 3)):
+        assert torch.equal(results[a][0], results[b][0])
+        assert np.array_equal(results[a][1], results[b][1]) and np.array_equal(results[a][2], results[b][2])
+
+
 def test_error_paths_return_status_and_launch_nothing():
     import paper_2506_18226_b200 as A
     H = _harness()
