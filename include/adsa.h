@@ -32,6 +32,18 @@
  *     position at or after cur_pos) set bits of a status word, skip the
  *     offending access and never trap; read it with adsa_get_status.
  *   - A context is not thread-safe: use it from one host thread at a time.
+ *   - Launches overlap.  The attention and layer-step kernels are launched with
+ *     programmatic stream serialization: their set-up runs while the kernel
+ *     ahead of them in the stream drains, and when the context's previous call
+ *     served another layer they also read this layer's cache state (rows, page
+ *     table, positions, norms, carried scores) before that kernel has finished.
+ *     Two rules follow.  The buffers of adsa_buffers belong to the library between
+ *     calls: nothing else may write them while work of this context is in flight.
+ *     And the calls of one context that touch the same layer must reach the device
+ *     in order (one stream, or streams ordered by events), as they would have to
+ *     anyway.  q, k_new, v_new and the keep mask are read only after the kernel
+ *     ahead has completed, so producing them in the kernel launched just before
+ *     the call is fine.
  *   - bf16 tensors are dense, row-major, innermost dimension head_dim
  *     ([batch][n_heads][head_dim] unless stated); all arithmetic is fp32.
  */

@@ -249,7 +249,7 @@ def _run_steps(T0, H, W, d, budget_fn, n_prefix, seed, score_variant=0, n_stream
 
 
 def test_budget_covering_the_context_is_dense_attention():
-    # "behaves identically to the baseline when the cache is not full" (Section 4.2)
+    # Section 4.2: as long as the cache has room nothing is evicted, so the method is plain dense attention
     T0, H, W, d = 6, 4, 5, 16
     st, hk, hv, log = _run_steps(T0, H, W, d, lambda cur: 10_000, T0, seed=8)
     for cur, q, before, res, n_live in log:
