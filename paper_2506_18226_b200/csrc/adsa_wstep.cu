@@ -395,20 +395,21 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             cur_in = tl * kWTile - cur_pg * c.page_rows;
         };
         seek(rk);
-        auto issue = [&](int u) {   // lane 0 only: this warp's u-th tile of the stream into the next free stage
+        auto issue = [&](int u) {   // all lanes (the copies themselves by lanes 0 and 1): this warp's u-th tile of the stream into the next free stage
             const int stage = i_stage;
             const int pass = u >= mt ? 1 : 0, tl = rk + (pass ? u - mt : u) * G;
             if (u == mt) seek(rk);
             const int r0 = tl * kWTile, r1 = min(n, r0 + kWTile);
             const uint32_t kdst = stages_u32 + stage * kWStageBytes, vdst = kdst + kWTileBytes;
             const uint32_t bar = smem_u32(bars + stage);
-            mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
+            __syncwarp();
             if (r1 - r0 == kWTile && cur_in + kWTile <= c.page_rows) {
-                // the common case: a whole tile inside one page is one box per pool
+                // the common case: a whole tile inside one page is one box per pool; lane 0 copies K, lane 1 copies V
                 const int y = pt_s[cur_pg] * c.page_rows + cur_in;
-                if (pass == 0) tma_2d(kdst, &maps.k[5], 0, y, bar);
-                tma_2d(vdst, &maps.v[5], 0, y, bar);
-            } else {
+                if (lane == 1 || (lane == 0 && pass == 0))
+                    tma_2d(lane ? vdst : kdst, lane ? &maps.v[5] : &maps.k[5], 0, y, bar);
+            } else if (lane == 0) {
                 int r = r0, pg = cur_pg, in = cur_in;
                 while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
                     int cnt = min(r1 - r, c.page_rows - in);
@@ -457,7 +458,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             __syncwarp();
-            if (lane == 0) issue(next_issue);
+            issue(next_issue);
             i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
         }
 
@@ -476,7 +477,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
                 __syncwarp();
-                if (lane == 0) issue(next_issue);
+                issue(next_issue);
                 ++next_issue;
                 i_stage = i_stage + 1 == D ? 0 : i_stage + 1;
             }
