@@ -634,7 +634,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             if (same_cut) mine.n_cand = mine.p;
-            if (!waited) { dep_wait(); load_inputs(); }   // the inputs arrive while the selection is completed
             unsigned long long my_key;
             {   // the warp's largest key (keys are distinct: the low word is the position) and its slot
                 const uint32_t kh = my_hi, kl = my_lo;
@@ -645,7 +644,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 my_key = ((unsigned long long)mh << 32) | ml;
             }
             mine.max_key = my_key; mine.max_slot = my_slot;
-            if (lane == 0) sel_part[rk] = mine;
+            if (lane == 0) {
+                sel_part[rk] = mine;
+                // the row this warp would evict is one of the group's candidates: a hint now makes the load of
+                // the chosen one, after the group has met, a short one
+                if (my_slot >= 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + row_offset(c, pt_s, my_slot)));
+            }
+            if (!waited) { dep_wait(); load_inputs(); }   // the inputs arrive while the selection is completed
             group_sync();
             int p = 0, n_cand = 0, n_cand_np = 0;
             unsigned long long max_key = 0ull;
