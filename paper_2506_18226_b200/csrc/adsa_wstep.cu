@@ -1010,7 +1010,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     release_and_refill();
                 }
             }
-            group_sync();   // every warp's copies of this stream have landed before rows move or pages are freed
+            // every warp's copies of this stream have landed before rows move or pages are freed (after a single
+            // sweep the group has met since its last copy landed: at the merge of the partial states)
+            if (!single) group_sync();
 
             // ---- the update itself, by the first warp ---------------------------------------------------
             if (okay && rk == 0) {
@@ -1049,7 +1051,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
         }
-        group_sync();   // the stream's shared buffers are free for the next one
+        if (local + stride < c.S) group_sync();   // the stream's shared buffers are free for the next one
     }
 }
 
