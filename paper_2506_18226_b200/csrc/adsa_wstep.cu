@@ -287,8 +287,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     // dep_wait() on.  Normally that is here.  When the host knows that the kernel ahead does not write this
     // layer's cache state (it served another layer; only the kernel directly ahead can still be running,
     // because every kernel of this library waits for its predecessor before it lets its successor start),
-    // the state is read, the first tiles are requested and the rows are classified first, and the wait
-    // comes just before the caller's inputs (q, the new row, the keep mask) are touched.  After its own
+    // the state is read, the first tiles are requested and the whole selection is made first (all of it
+    // shared-memory work on the cache state; nothing is written to global memory), and the wait comes
+    // just before the caller's inputs (q, the new row, the keep mask) are touched.  After its own
     // wait a grid lets the next kernel in the stream be scheduled onto the SMs its CTAs leave.
     bool waited = false;
     auto dep_wait = [&]() {
@@ -650,7 +651,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 // the chosen one, after the group has met, a short one
                 if (my_slot >= 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + row_offset(c, pt_s, my_slot)));
             }
-            if (!waited) { dep_wait(); load_inputs(); }   // the inputs arrive while the selection is completed
             group_sync();
             int p = 0, n_cand = 0, n_cand_np = 0;
             unsigned long long max_key = 0ull;
@@ -790,6 +790,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
         __syncwarp();
 
+        if (FUSED && !waited) { dep_wait(); load_inputs(); }   // the whole selection came first: it reads the cache state only
         // ---- the running state; the first warp starts from the new row: weight 1 for role 0, its 1/|v| for role 2 ----
         // o_run[md][0..3]: dimension 16*md + g (0, 1) and 16*md + g + 8 (2, 3), roles 2t (0, 2) and 2t + 1 (1, 3), where
         // role 0/1 = softmax.V through P_hi / P_lo and roles 2/3/4 = s through w_hi / w_mid / w_lo.
