@@ -517,6 +517,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // Eq. 1-2 for the next step on one tile of V rows: dot_i = v_i . s by MMA,
         // S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), written at the row's new slot
         int list_ns = 0, n2 = n;   // survivors of the general compaction; live rows after the update
+        bool warp_rare = false;
         float rden = 0.f;
         // (two halves, so that the products can be issued early and their results used later)
         auto score_mma = [&](uint32_t vb, float (&dt)[2][4]) {
@@ -537,8 +538,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const int r0 = tl * kWTile;
             // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
             float sval[4], invv[4], dotv[4];
-            bool want[4], rare = false;
-            const bool moves = n2 < n;   // more than one eviction: rows above the new length move down
+            bool want[4];
             const uint32_t cwg = t == 0 ? cw >> g : 0u;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -549,9 +549,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 invv[i] = inv_s[row];   // past the last live row this reads whatever follows in shared memory: never wanted
                 dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
                 sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
-                rare |= want[i] && (invv[i] >= 1.0f / kNormEps || (moves && row >= n2));
             }
-            if (!__any_sync(0xffffffffu, rare)) {
+            // warp_rare (set when the row weights were made): one of this warp's scored rows has a clamped
+            // norm, or rows move down in the update; otherwise every row is written where it stands
+            if (!warp_rare) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
@@ -761,6 +762,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (general) group_sync();
             {
                 uint32_t *ws = reinterpret_cast<uint32_t *>(wsplit);
+                float w_big = 0.f;   // the largest 1/|v| among the rows this warp will score
                 for (int i = 0; rk + i * G < n_tiles; i += 2) {   // two of the warp's blocks per trip, a pair of rows per lane
                     const int b = rk + (i + (lane >> 4)) * G;
                     if (b < n_tiles) {
@@ -769,6 +771,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         float w0 = 0.f, w1 = 0.f;
                         if (cm & 1u) w0 = inv_s[slot];
                         if (cm & 2u) w1 = inv_s[slot + 1];
+                        w_big = fmaxf(w_big, fmaxf(w0, w1));
                         const uint32_t h = pack_bf16(w0, w1);
                         const float r0 = w0 - bf16_lo(h), r1 = w1 - bf16_hi(h);
                         const uint32_t md = pack_bf16(r0, r1);
@@ -776,6 +779,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         ws[slot >> 1] = h; ws[(L.w_rows + slot) >> 1] = md; ws[(2 * L.w_rows + slot) >> 1] = lo;
                     }
                 }
+                warp_rare = __any_sync(0xffffffffu, w_big >= 1.0f / kNormEps) || n2 < n;
             }
             if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
                 make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
