@@ -445,7 +445,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         auto l2_ask = [&](int u) {   // this warp's u-th tile of pass 1, a row per lane
             const int row = (rk + u * G) * kWTile + lane;
             if (u < mt && row < n) {
-                const size_t off = row_offset(c, pt_s, row);
+                const size_t off = c.max_pages == 1 ? ((size_t)pt_s[0] * c.page_rows + row) * (size_t)c.row_stride
+                                                    : row_offset(c, pt_s, row);
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
             }
