@@ -39,8 +39,8 @@ INPUT_RING_BYTES = 24 << 30   # q/k/v for all steps are kept in HBM up to this s
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/, keyed by workload; None where no capture of the current kernel exists.
-STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 98625152 + 3501568}    # profiles/step_kernel_cfg4_2layers.md
-ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94054656 + 3007872}     # profiles/attn_kernel_cfg4_2layers.md
+STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 98622720 + 3850112}    # profiles/step_kernel_cfg4_2layers.md
+ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94057600 + 3473536}     # profiles/attn_kernel_cfg4_2layers.md
 
 
 def parse_args():
