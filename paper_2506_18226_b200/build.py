@@ -26,7 +26,9 @@ def build_lib(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc, *NVCC_FLAGS, "-shared", "-o", tmp, *[os.path.join(CSRC, s) for s in SOURCES]]
+    # --threads: the sources are independent translation units, compiled side by side
+    cmd = [nvcc, "--threads", str(min(len(SOURCES), os.cpu_count() or 1)), *NVCC_FLAGS, "-shared", "-o", tmp,
+           *[os.path.join(CSRC, s) for s in SOURCES]]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)
