@@ -312,7 +312,8 @@ def run_ours(args, rank, world, local_rank):
         per = int(np.prod(shape)) * 2
         e2e = {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 3 * per,
                "d2h_bytes_per_step": per, "steps": Ke, "ms_per_step": e2e_ms / Ke,
-               "api": "adsa_token_step_host (pinned host q/k/v in, host output out, one sync per token)"}
+               "api": "adsa_token_step_host (pinned host q/k/v in, host output out, copies in chunks of layers under the "
+                      "compute, one sync per token)"}
 
     if rank != 0:
         return

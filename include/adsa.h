@@ -198,9 +198,13 @@ ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int bud
 ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 
-/* adsa_token_step with HOST tensors of the same shapes: one host-to-device copy
- * per input, all layers, one device-to-host copy of the outputs, then the
- * stream is synchronised.  Uses the staging part of the workspace. */
+/* adsa_token_step with HOST tensors of the same shapes (pinned memory, or the
+ * copies do not overlap anything).  Inputs and outputs travel in up to six
+ * chunks of layers on two copy streams that the context creates on its first
+ * call here, so that later layers' inputs and earlier layers' outputs cross the
+ * bus while the layers in between compute; the kernels run on `stream`.  When
+ * the call returns every layer has run and the outputs are on the host.  Uses
+ * the staging part of the workspace; results are those of adsa_token_step. */
 ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host,
                                   const void *k_new_host, const void *v_new_host, void *out_host,
                                   adsa_stream_t stream);

@@ -102,6 +102,11 @@ struct adsa_ctx {
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
+    // adsa_token_step_host moves its tensors in chunks of layers on two copy streams of its own, so that the
+    // copies of later layers travel while earlier layers compute (created on first use, host-side objects only)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_done;
 };
 
 namespace {
@@ -319,6 +324,13 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
 
 int adsa_destroy(adsa_ctx *ctx)
 {
+    if (ctx) {
+        for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
+        for (cudaEvent_t e : ctx->ev_done) cudaEventDestroy(e);
+        if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+        if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+        if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    }
     delete ctx;
     return ADSA_OK;
 }
@@ -544,15 +556,75 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
     if (ctx->cuda_error) return ADSA_ECUDA;
     if (!q_host || !k_new_host || !v_new_host || !out_host) return ADSA_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
-    size_t bytes = (size_t)ctx->dev.S * ctx->cfg.n_layers * ctx->cfg.head_dim * sizeof(__nv_bfloat16);
-    cudaError_t e = cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_k, k_new_host, bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stage_v, v_new_host, bytes, cudaMemcpyHostToDevice, st);
+    const int L = ctx->cfg.n_layers;
+    // chunk boundaries: a first chunk of one layer, so that computing starts after a short copy, then up to five
+    // equal ones
+    int bound[7], n_chunks = 0;
+    bound[0] = 0;
+    if (L <= 6) {
+        for (int l = 1; l <= L; ++l) bound[l] = l;
+        n_chunks = L;
+    } else {
+        bound[1] = 1;
+        const int rest = L - 1, per = (rest + 4) / 5;
+        n_chunks = 1;
+        for (int l = 1; l < L; l += per) { bound[n_chunks + 1] = l + per < L ? l + per : L; ++n_chunks; }
+    }
+    cudaError_t e = cudaSuccess;
+    if (!ctx->copy_in) {   // first use on this context
+        e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming);
+        for (int c = 0; c < 6 && e == cudaSuccess; ++c) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            e = cudaEventCreateWithFlags(&a, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b, cudaEventDisableTiming);
+            if (a) ctx->ev_in.push_back(a);
+            if (b) ctx->ev_done.push_back(b);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    const size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;   // elements
+    const char *qh = (const char *)q_host, *kh = (const char *)k_new_host, *vh = (const char *)v_new_host;
+    char *oh = (char *)out_host;
+    auto copy_in_chunk = [&](int c) -> cudaError_t {   // inputs of chunk c, on the inbound copy stream
+        const size_t off = (size_t)bound[c] * per_layer, bytes = (size_t)(bound[c + 1] - bound[c]) * per_layer * sizeof(__nv_bfloat16);
+        cudaError_t r = cudaMemcpyAsync(ctx->stage_q + off, qh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+        if (r == cudaSuccess) r = cudaMemcpyAsync(ctx->stage_k + off, kh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+        if (r == cudaSuccess) r = cudaMemcpyAsync(ctx->stage_v + off, vh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+        if (r == cudaSuccess) r = cudaEventRecord(ctx->ev_in[c], ctx->copy_in);
+        return r;
+    };
+    // the copies start when the work already queued on the caller's stream is done (it may still read the staging buffers)
+    e = cudaEventRecord(ctx->ev_start, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_in, ctx->ev_start, 0);
+    // copies are queued two chunks ahead of the launches, so that the first kernel is queued early
+    for (int c = 0; c < 2 && c < n_chunks && e == cudaSuccess; ++c) e = copy_in_chunk(c);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    int rc = adsa_token_step(ctx, cur_pos, budget_rows, ctx->stage_q, ctx->stage_k, ctx->stage_v, ctx->stage_o, stream);
-    if (rc) return rc;
-    e = cudaMemcpyAsync(out_host, ctx->stage_o, bytes, cudaMemcpyDeviceToHost, st);
+    for (int c = 0; c < n_chunks; ++c) {
+        const int l0 = bound[c], l1 = bound[c + 1];
+        const size_t off = (size_t)l0 * per_layer, bytes = (size_t)(l1 - l0) * per_layer * sizeof(__nv_bfloat16);
+        e = cudaStreamWaitEvent(st, ctx->ev_in[c], 0);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        for (int l = l0; l < l1; ++l) {
+            int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, ctx->stage_q + l * per_layer, ctx->stage_k + l * per_layer,
+                                     ctx->stage_v + l * per_layer, ctx->stage_o + l * per_layer, stream);
+            if (rc) {   // nothing may be left running on the private streams when the call returns
+                cudaStreamSynchronize(ctx->copy_in);
+                cudaStreamSynchronize(ctx->copy_out);
+                cudaStreamSynchronize(st);
+                return rc;
+            }
+        }
+        e = cudaEventRecord(ctx->ev_done[c], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[c], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(oh + off * 2, ctx->stage_o + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
+        if (e == cudaSuccess && c + 2 < n_chunks) e = copy_in_chunk(c + 2);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    e = cudaStreamSynchronize(ctx->copy_out);   // the last output chunk is on the host: every layer has run
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->copy_in);
     return cuda_fail(ctx, e);
 }
 

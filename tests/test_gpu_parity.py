@@ -323,6 +323,37 @@ def test_back_to_back_layers_match_serialised_launches():
         assert np.array_equal(results[a][1], results[b][1]) and np.array_equal(results[a][2], results[b][2])
 
 
+@pytest.mark.parametrize("n_layers", [1, 4, 8])
+def test_token_step_host_matches_device_call(n_layers):
+    """adsa_token_step_host (inputs and outputs in pinned host memory, moved in chunks of layers while other
+    layers compute) gives bit for bit what adsa_token_step gives on device tensors, and leaves the same cache."""
+    H = _harness()
+    w = Workload("host", 94, n_layers, 2, 2, 64, 16, 8, 7, 0.5, 1.0)
+    C, L, T = w.capacity(), w.n_layers, w.n_cells
+    engs = [H.engine_for(w, capacity=C, page_rows=16) for _ in range(2)]
+    for e in engs:
+        for l in range(L):
+            k, v = prefix_kv(w, 6, l)
+            e.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
+    shape = (L, w.batch, w.n_heads, w.head_dim)
+    out_d = torch.zeros(shape, dtype=torch.bfloat16, device="cuda:0")
+    out_h = torch.zeros(shape, dtype=torch.bfloat16).pin_memory()
+    for g in range(T):
+        per = [layer_step_qkv(w, 6, l, g) for l in range(L)]
+        bits = [np.stack([x[i] for x in per]).reshape(shape) for i in range(3)]
+        dev = [H.dev_bf16(b) for b in bits]
+        host = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory() for b in bits]
+        cur = w.n_text + g
+        engs[0].token_step(cur, C, dev[0], dev[1], dev[2], out_d)
+        engs[1].token_step_host(cur, C, host[0], host[1], host[2], out_h)
+        assert torch.equal(out_d.cpu(), out_h), f"cell {g}"
+    for e in engs:
+        assert e.get_status()[0] == 0
+    assert torch.equal(engs[0]._t["n_live"].cpu(), engs[1]._t["n_live"].cpu())
+    pos = [np.sort(e._t["pos"][:, :C].cpu().numpy(), axis=1) for e in engs]
+    assert np.array_equal(pos[0], pos[1])
+
+
 def test_error_paths_return_status_and_launch_nothing():
     import paper_2506_18226_b200 as A
     H = _harness()
