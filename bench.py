@@ -212,9 +212,8 @@ def run_ours(args, rank, world, local_rank):
         step_ms += e0.elapsed_time(e1)
         step_launches += eng.launch_count() - n0
     rows_step = int(eng._t["n_live"].max().item())
-    # (the workspace holds one layer's keep mask and evict list, so with the calls grouped like this every layer's
-    # attention and update use the last layer's selection: same rows kept and evicted per launch, i.e. the same work,
-    # but the outputs of these cells mean nothing and the timed generation below starts from a reset)
+    # (the keep mask and counts are stored per layer, so grouping the calls like this is a valid trajectory: every
+    # layer attends and evicts by its own selection; the timed generation below starts from a reset all the same)
     attn_ms, attn_launches = 0.0, 0
     call_ms = {"adsa_score": [], "adsa_select": [], "adsa_sparse_decode_attn": [], "adsa_kv_update": []}
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]

@@ -34,16 +34,21 @@
  *   - A context is not thread-safe: use it from one host thread at a time.
  *   - Launches overlap.  The attention and layer-step kernels are launched with
  *     programmatic stream serialization: their set-up runs while the kernel
- *     ahead of them in the stream drains, and when the context's previous call
- *     served another layer they also read this layer's cache state (rows, page
- *     table, positions, norms, carried scores) before that kernel has finished.
- *     Two rules follow.  The buffers of adsa_buffers belong to the library between
+ *     ahead of them in the stream drains, and when that kernel is this context's
+ *     previous launch, went to the same stream and served another layer (or does
+ *     not write what is about to be read), they also read this layer's cache state
+ *     (rows, page table, positions, norms, carried scores) before it has finished.
+ *     Three rules follow.  The buffers of adsa_buffers belong to the library between
  *     calls: nothing else may write them while work of this context is in flight.
- *     And the calls of one context that touch the same layer must reach the device
- *     in order (one stream, or streams ordered by events), as they would have to
- *     anyway.  q, k_new, v_new and the keep mask are read only after the kernel
- *     ahead has completed, so producing them in the kernel launched just before
- *     the call is fine.
+ *     The calls of one context must reach the device in the order they are made:
+ *     use one stream, or order the streams with events (work on a second stream
+ *     that is not ordered after the first races on the shared scratch and on the
+ *     cache state).  And a kernel of the caller's own that is put between two
+ *     calls on the same stream must not itself start early under programmatic
+ *     stream serialization, or must wait for its predecessor before it lets its
+ *     successor start.  q, k_new, v_new and the keep mask are read only after the
+ *     kernel ahead has completed, so producing them in the kernel launched just
+ *     before the call is fine.
  *   - bf16 tensors are dense, row-major, innermost dimension head_dim
  *     ([batch][n_heads][head_dim] unless stated); all arithmetic is fp32.
  */
@@ -109,8 +114,9 @@ typedef struct {
 } adsa_buffers;
 /* n_streams = n_layers * batch * n_heads.  All buffers are initialised by adsa_reset. */
 
-/* Scratch size the configuration needs (scores, keep masks, evict lists, split
- * partials, staging for the *_host call).  No CUDA call is made. */
+/* Scratch size the configuration needs (per layer: scores, carried sums, keep
+ * masks, counts, staging for the *_host calls; once: split partials, status
+ * word).  No CUDA call is made. */
 ADSA_API int adsa_workspace_bytes(const adsa_config *cfg, size_t *out_bytes);
 
 /* Validate cfg and buffers and build the host-side context.  Queries the
@@ -142,7 +148,11 @@ ADSA_API int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const 
  * cur_pos is the context position of the token being decoded (its row is "the
  * new row").  Section 4.1 partitions each stream's live rows by position into
  * prefix (pos < n_prefix), local (image cells before the current one, in the
- * current grid row or the R rows above) and previous (the rest). */
+ * current grid row or the R rows above) and previous (the rest).
+ * The order is kept per layer (ADSA_ESTATE otherwise).  What one call leaves for
+ * the next (scores, keep mask, counts) is stored per layer, so the steps of
+ * different layers may be interleaved in any way: score and select for every
+ * layer, then every layer's attention, then every update, is a valid sequence. */
 
 /* Eq. 1-2.  For every row i of the previous region of every stream of `layer`:
  * S_i = (1/(p-1)) sum_{j != i} cos(v_i, v_j), j over the same region (p rows);
@@ -276,7 +286,7 @@ ADSA_API int64_t adsa_launch_count(const adsa_ctx *ctx);
  * The scratch of the split reduction is a fixed 4 MiB array inside the library image: every GPU that
  * loads the library holds it until the process exits.  Limits: n_streams <= 4096, max_rows <= 2^20
  * (ADSA_ENOMEM beyond them; fewer chunks per stream are used when the partial states of more would
- * not fit).  No cudaMalloc, cudaFree or allocating routine is called; the call only enqueues a
+ * not fit, down to a single chunk, which needs no partial state at all).  No cudaMalloc, cudaFree or allocating routine is called; the call only enqueues a
  * counter clear and one kernel on `stream`.
  * The first call on each device looks up the array's device address (that device must be current);
  * make that first call before any stream capture begins.  All calls share the array and it keeps

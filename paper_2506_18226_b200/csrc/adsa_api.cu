@@ -24,12 +24,14 @@ struct LayerState {
     int rows_hi = 0;   // upper bound of n_live over the layer's streams
     int scores_pos = -1;  // the carried scores (DevCtx::scores) are Eq. 2 for a step at this position; -1 = stale
     int svec_pos = -1;    // the carried sum of normalised rows (DevCtx::svec) belongs to that position too; -1 = none
+    bool launched = false;            // some kernel of this layer has been launched since the reset
+    cudaStream_t last_stream = nullptr;   // ... the latest of them on this stream
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, evict_slots, counts, partials, tickets, svec, status, staging, total;
+    size_t scores, keep_mask, counts, partials, tickets, svec, status, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -40,9 +42,8 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     WorkspaceLayout w;
     size_t off = 0;
     w.scores = off;      off = align_up(off + S * (size_t)cfg.n_layers * R * sizeof(float), 256);
-    w.keep_mask = off;   off = align_up(off + S * mask_words_of(cfg) * sizeof(uint32_t), 256);
-    w.evict_slots = off; off = align_up(off + S * R * sizeof(int32_t), 256);
-    w.counts = off;      off = align_up(off + S * 4 * sizeof(int32_t), 256);
+    w.keep_mask = off;   off = align_up(off + S * (size_t)cfg.n_layers * mask_words_of(cfg) * sizeof(uint32_t), 256);
+    w.counts = off;      off = align_up(off + S * (size_t)cfg.n_layers * 4 * sizeof(int32_t), 256);
     w.partials = off;    off = align_up(off + S * kMaxSplits * (size_t)(cfg.row_stride + 2) * sizeof(float), 256);
     w.tickets = off;     off = align_up(off + S * sizeof(int32_t), 256);
     w.svec = off;        off = align_up(off + S * (size_t)cfg.n_layers * 256 * sizeof(float), 256);
@@ -99,6 +100,7 @@ struct adsa_ctx {
     // set-up (launches overlap by programmatic dependent launch): the layer it served (-1 = several or
     // unknown) and whether it writes the cache proper (rows, pages, positions, norms) / the carried scores.
     int prev_layer = -1, prev_writes_cache = 1, prev_writes_scores = 1;
+    cudaStream_t prev_stream = nullptr;   // the stream that launch went to: only a launch on the same stream is its successor
     int cuda_error = 0;  // sticky
     int64_t launches = 0;
     __nv_bfloat16 *stage_q, *stage_k, *stage_v, *stage_o;
@@ -195,18 +197,25 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     return ch;
 }
 
-void note_launch(adsa_ctx *ctx, int layer, bool writes_cache, bool writes_scores)
+void note_launch(adsa_ctx *ctx, int layer, bool writes_cache, bool writes_scores, adsa_stream_t stream)
 {
+    ctx->prev_stream = (cudaStream_t)stream;
+    if (layer >= 0) { ctx->layers[layer].launched = true; ctx->layers[layer].last_stream = (cudaStream_t)stream; }
     ctx->prev_layer = layer;
     ctx->prev_writes_cache = writes_cache ? 1 : 0;
     ctx->prev_writes_scores = writes_scores ? 1 : 0;
 }
 
-// May the kernel about to be launched read `layer`'s cache state (and, for the fused step, its carried
-// scores) before the kernel ahead of it has completed?
-bool state_is_quiet(const adsa_ctx *ctx, int layer, bool needs_scores)
+// May the kernel about to be launched on `stream` read `layer`'s cache state (and, for the fused step, its
+// carried scores) before the kernel ahead of it in that stream has completed?  Only when that kernel is the
+// context's previous launch (same stream), so that what it writes is known.
+bool state_is_quiet(const adsa_ctx *ctx, int layer, bool needs_scores, cudaStream_t stream)
 {
-    if (ctx->prev_layer < 0) return false;
+    if (ctx->prev_layer < 0 || ctx->prev_stream != stream) return false;
+    // the layer's own earlier kernels are known to be complete only if they went to this stream too: every
+    // kernel of the library lets its successor in the stream start only after its own dependency wait
+    const LayerState &L = ctx->layers[layer];
+    if (L.launched && L.last_stream != stream) return false;
     if (ctx->prev_layer != layer) return true;
     return !ctx->prev_writes_cache && !(needs_scores && ctx->prev_writes_scores);
 }
@@ -217,7 +226,7 @@ cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fuse
 {
     if (ch.wp.n_groups)
         return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st,
-                            have_svec && !ctx->no_single_sweep, state_is_quiet(ctx, layer, fused));
+                            have_svec && !ctx->no_single_sweep, state_is_quiet(ctx, layer, fused, st));
     if (ch.pp.n_stages)
         return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
     return launch_step(ctx->dev, ch.sp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
@@ -277,7 +286,6 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.free_state = buf->free_state;
     d.scores = (float *)(w + ws.scores);
     d.keep_mask = (uint32_t *)(w + ws.keep_mask);
-    d.evict_slots = (int32_t *)(w + ws.evict_slots);
     d.counts = (int32_t *)(w + ws.counts);
     d.partials = (float *)(w + ws.partials);
     d.tickets = (int32_t *)(w + ws.tickets);
@@ -339,8 +347,12 @@ int adsa_reset(adsa_ctx *ctx, adsa_stream_t stream)
 {
     if (!ctx) return ADSA_EINVAL;
     if (ctx->cuda_error) return ADSA_ECUDA;
-    for (auto &l : ctx->layers) l = LayerState();
-    note_launch(ctx, -1, true, true);
+    for (auto &l : ctx->layers) {
+        l = LayerState();
+        l.launched = true;   // the reset kernel writes every layer's state
+        l.last_stream = (cudaStream_t)stream;
+    }
+    note_launch(ctx, -1, true, true, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_reset(ctx->dev, ctx->cfg.n_layers * ctx->dev.S, (cudaStream_t)stream));
 }
@@ -358,7 +370,7 @@ int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, co
     L.rows_hi += n_rows;
     L.scores_pos = -1;
     L.svec_pos = -1;
-    note_launch(ctx, layer, true, true);
+    note_launch(ctx, layer, true, true, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
 }
@@ -379,7 +391,7 @@ int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, 
     L.scores_pos = -1;
     L.svec_pos = -1;
     int sid = (layer * ctx->cfg.batch + b) * ctx->cfg.n_heads + h;
-    note_launch(ctx, layer, true, true);
+    note_launch(ctx, layer, true, true, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_set_rows(ctx->dev, sid, k, v, pos, n_rows, (cudaStream_t)stream));
 }
@@ -395,13 +407,13 @@ int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_st
     L.cur_pos = cur_pos;
     if (L.scores_pos == cur_pos) {   // carried in from the previous fused step: nothing to compute
         if (!scores_out) return ADSA_OK;
-        note_launch(ctx, layer, false, false);
+        note_launch(ctx, layer, false, false, stream);
         ++ctx->launches;
         return cuda_fail(ctx, launch_scores_copy(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
     }
     L.scores_pos = cur_pos;
     L.svec_pos = -1;   // the stand-alone score kernel does not leave the sum behind
-    note_launch(ctx, layer, false, true);
+    note_launch(ctx, layer, false, true, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
 }
@@ -422,7 +434,7 @@ int adsa_select(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, int32_t 
     if (!pool_can_hold(ctx, layer, after > L.rows_hi ? after : L.rows_hi)) return ADSA_ENOMEM;
     L.phase = kSelected;
     L.budget = budget_rows;
-    note_launch(ctx, layer, false, false);
+    note_launch(ctx, layer, false, false, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_select(ctx->dev, layer, cur_pos, budget_rows, sel_slots, sel_pos, evict_pos, counts,
                                         (cudaStream_t)stream));
@@ -446,7 +458,7 @@ int adsa_sparse_decode_attn(adsa_ctx *ctx, int layer, int cur_pos, const void *q
         AttnPlan plan = plan_attn(ctx, L.rows_hi);
         e = launch_attn(ctx->dev, plan, layer, cur_pos, q, k_new, v_new, out_bf16, out_f32, (cudaStream_t)stream);
     }
-    note_launch(ctx, layer, false, false);   // attention reads the cache and writes the output only
+    note_launch(ctx, layer, false, false, stream);   // attention reads the cache and writes the output only
     return cuda_fail(ctx, e);
 }
 
@@ -463,7 +475,7 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
     L.phase = kIdle;
     L.scores_pos = -1;   // rows move and the scores of the next step were not computed
     L.svec_pos = -1;
-    note_launch(ctx, layer, true, false);
+    note_launch(ctx, layer, true, false, stream);
     ++ctx->launches;
     return cuda_fail(ctx, launch_kv_update(ctx->dev, layer, cur_pos, k_new, v_new, (cudaStream_t)stream));
 }
@@ -497,7 +509,7 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     if (L.phase == kIdle && L.scores_pos != cur_pos) {   // no scores carried in (first step, or the cache was rewritten)
         ++ctx->launches;
         L.svec_pos = -1;
-        note_launch(ctx, layer, false, true);
+        note_launch(ctx, layer, false, true, stream);
         rc = cuda_fail(ctx, launch_score(ctx->dev, layer, cur_pos, nullptr, (cudaStream_t)stream));
         if (rc) return rc;
     }
@@ -505,7 +517,7 @@ int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, cons
     ++ctx->launches;
     rc = cuda_fail(ctx, launch_staged(ctx, ch, true, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
                                       (cudaStream_t)stream, have_svec));
-    note_launch(ctx, layer, true, true);
+    note_launch(ctx, layer, true, true, stream);
     L.rows_hi = after;
     L.phase = kIdle;
     L.cur_pos = cur_pos;
@@ -537,6 +549,7 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
                     const void *v_new, void *out_bf16, adsa_stream_t stream)
 {
     if (!ctx || !q || !k_new || !v_new || !out_bf16) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
     size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k_new,
                         *vb = (const __nv_bfloat16 *)v_new;
@@ -600,31 +613,27 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
     if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_in, ctx->ev_start, 0);
     // copies are queued two chunks ahead of the launches, so that the first kernel is queued early
     for (int c = 0; c < 2 && c < n_chunks && e == cudaSuccess; ++c) e = copy_in_chunk(c);
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
-    for (int c = 0; c < n_chunks; ++c) {
+    int rc = ADSA_OK;
+    for (int c = 0; c < n_chunks && e == cudaSuccess && rc == ADSA_OK; ++c) {
         const int l0 = bound[c], l1 = bound[c + 1];
         const size_t off = (size_t)l0 * per_layer, bytes = (size_t)(l1 - l0) * per_layer * sizeof(__nv_bfloat16);
         e = cudaStreamWaitEvent(st, ctx->ev_in[c], 0);
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
-        for (int l = l0; l < l1; ++l) {
-            int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, ctx->stage_q + l * per_layer, ctx->stage_k + l * per_layer,
-                                     ctx->stage_v + l * per_layer, ctx->stage_o + l * per_layer, stream);
-            if (rc) {   // nothing may be left running on the private streams when the call returns
-                cudaStreamSynchronize(ctx->copy_in);
-                cudaStreamSynchronize(ctx->copy_out);
-                cudaStreamSynchronize(st);
-                return rc;
-            }
-        }
+        for (int l = l0; l < l1 && e == cudaSuccess && rc == ADSA_OK; ++l)
+            rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, ctx->stage_q + l * per_layer, ctx->stage_k + l * per_layer,
+                                 ctx->stage_v + l * per_layer, ctx->stage_o + l * per_layer, stream);
+        if (e != cudaSuccess || rc != ADSA_OK) break;
         e = cudaEventRecord(ctx->ev_done[c], st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[c], 0);
         if (e == cudaSuccess) e = cudaMemcpyAsync(oh + off * 2, ctx->stage_o + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
         if (e == cudaSuccess && c + 2 < n_chunks) e = copy_in_chunk(c + 2);
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
-    e = cudaStreamSynchronize(ctx->copy_out);   // the last output chunk is on the host: every layer has run
-    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->copy_in);
+    // One way out, whatever happened: nothing of this call may still be running on the private streams, or
+    // reading and writing the caller's host buffers, when it returns.  On success the last output chunk is
+    // then on the host and every layer has run.
+    const cudaError_t s_out = cudaStreamSynchronize(ctx->copy_out), s_st = cudaStreamSynchronize(st),
+                      s_in = cudaStreamSynchronize(ctx->copy_in);
+    if (rc != ADSA_OK) return rc;
+    if (e == cudaSuccess) e = s_out != cudaSuccess ? s_out : s_st != cudaSuccess ? s_st : s_in;
     return cuda_fail(ctx, e);
 }
 

@@ -44,7 +44,7 @@ attn_kernel(DevCtx c, int layer, int chunk_rows, int n_splits, const __nv_bfloat
 
     const int split = blockIdx.x, local = blockIdx.y, sid = layer * c.S + local;
     const int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
-    const uint32_t *mask = c.keep_mask + (size_t)local * c.mask_words;
+    const uint32_t *mask = c.keep_mask + (size_t)sid * c.mask_words;
     const int n = c.n_live[sid];
     const int c0 = split * chunk_rows, c1 = min(n, c0 + chunk_rows);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -262,7 +262,7 @@ extern "C" int adsa_decode_attn_static(const void *q, const void *k, const void 
     const size_t ticket_bytes = (size_t)kStaticMaxStreams * sizeof(int32_t);
     const size_t per_split = (size_t)n_streams * (row_stride + 2) * sizeof(float);
     int fit = (int)((kStaticScratchBytes - ticket_bytes) / per_split);
-    if (fit < 1) return ADSA_ENOMEM;
+    if (fit < 1) fit = 1;   // a single chunk per stream writes its output directly: no partial state, no counter
     int rows = max_rows < 1 ? 1 : max_rows;
     int splits = (sd->sm_count * 8 + n_streams - 1) / n_streams;
     splits = splits < 1 ? 1 : splits > kMaxSplits ? kMaxSplits : splits;

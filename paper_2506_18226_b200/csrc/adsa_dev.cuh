@@ -25,11 +25,12 @@ struct DevCtx {
     int32_t *page_table, *pos, *n_live;
     float *inv_norm;
     int32_t *free_ring, *free_state;
-    // workspace (one layer's worth, reused by every layer)
+    // workspace; S = streams per layer.  What one layer-step hands from call to call (scores, keep mask,
+    // counts) exists per layer, so that the steps of several layers may be in flight between their calls;
+    // the split partials are scratch of one attention launch and are shared by all layers
     float *scores;          // [n_layers * S][max_rows]  Eq. 2 scores by slot; carried from one step to the next
-    uint32_t *keep_mask;    // [S][mask_words]   bit s = slot s is retained
-    int32_t *evict_slots;   // [S][max_rows]     ascending
-    int32_t *counts;        // [S][4]            p, evicted, retained, K
+    uint32_t *keep_mask;    // [n_layers * S][mask_words]   bit s = slot s is retained
+    int32_t *counts;        // [n_layers * S][4]            p, evicted, retained, K
     float *partials;        // [S][kMaxSplits][partial_stride]
     int32_t *tickets;       // [S]
     float *svec;            // [n_layers * S][256]  s = sum of the normalised V rows the next step scores (carried with the scores)

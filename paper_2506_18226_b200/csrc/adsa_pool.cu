@@ -83,9 +83,9 @@ kv_update_kernel(DevCtx c, int layer, int cur_pos, const __nv_bfloat16 *k_new, c
     __shared__ int warp_cnt[2][kUpdateThreads / 32];
     int local = blockIdx.x, sid = layer * c.S + local;
     int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
-    const uint32_t *mask = c.keep_mask + (size_t)local * c.mask_words;
+    const uint32_t *mask = c.keep_mask + (size_t)sid * c.mask_words;
     int32_t *holes = sm_lists, *surv = sm_lists + c.max_rows + 1;
-    int n = c.n_live[sid], e = c.counts[local * 4 + 1];
+    int n = c.n_live[sid], e = c.counts[(size_t)sid * 4 + 1];
     int n2 = n - e + 1;
     int have = (n + c.page_rows - 1) / c.page_rows, need = (n2 + c.page_rows - 1) / c.page_rows;
     if (threadIdx.x == 0) {

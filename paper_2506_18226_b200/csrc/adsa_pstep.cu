@@ -159,7 +159,7 @@ pstep_kernel(DevCtx c, PStepArgs a)
                     }
                 }
             } else {
-                const uint32_t *g = c.keep_mask + (size_t)local * c.mask_words;
+                const uint32_t *g = c.keep_mask + (size_t)sid * c.mask_words;
                 uint32_t *d = reinterpret_cast<uint32_t *>(meta);
                 for (int w = lane; w * 32 < n; w += 32) d[w] = g[w];
             }

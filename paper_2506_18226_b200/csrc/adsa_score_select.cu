@@ -139,8 +139,7 @@ select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_sl
     const int p = sel.p, K = sel.K;
 
     // retained / evicted lists in ascending slot order, keep mask, counts
-    uint32_t *keep_mask = c.keep_mask + (size_t)local * c.mask_words;
-    int32_t *ev_slots = c.evict_slots + (size_t)local * c.max_rows;
+    uint32_t *keep_mask = c.keep_mask + (size_t)sid * c.mask_words;
     const size_t ob = (size_t)local * c.max_rows;
     for (int base = 0; base < n; base += kSSThreads) {
         int slot = base + threadIdx.x;
@@ -163,7 +162,6 @@ select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_sl
             if (sel_pos) sel_pos[ob + i] = pos[slot];
         } else if (live) {
             int i = oe + __popc(be & below);
-            ev_slots[i] = slot;
             if (evict_pos) evict_pos[ob + i] = pos[slot];
         }
         __syncthreads();
@@ -173,7 +171,7 @@ select_kernel(DevCtx c, int layer, int cur_pos, int budget_rows, int32_t *sel_sl
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        int32_t *cn = c.counts + local * 4;
+        int32_t *cn = c.counts + (size_t)sid * 4;
         cn[0] = p; cn[1] = s_be; cn[2] = s_bk; cn[3] = K;
         if (counts_out) { counts_out[local * 4 + 0] = p; counts_out[local * 4 + 1] = s_be;
                           counts_out[local * 4 + 2] = s_bk; counts_out[local * 4 + 3] = K; }

@@ -173,7 +173,7 @@ step_kernel(DevCtx c, StepArgs a)
         __syncthreads();
         p_next = s_pnext + (new_cand ? 1 : 0);
     } else {
-        const uint32_t *gmask = c.keep_mask + (size_t)local * c.mask_words;
+        const uint32_t *gmask = c.keep_mask + (size_t)sid * c.mask_words;
         for (int w = tid; w * 32 < n; w += kStepThreads) kmask[w] = gmask[w];
         __syncthreads();
     }

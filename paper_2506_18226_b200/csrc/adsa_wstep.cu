@@ -247,7 +247,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             if (a.early_state) {
                 // the state is read for real right away (see dep_wait below): only the inputs need hints
-                if constexpr (!FUSED) prefetch_span(c.keep_mask + (size_t)local0 * c.mask_words, (size_t)c.mask_words * 4);
+                if constexpr (!FUSED) prefetch_span(c.keep_mask + (size_t)sid0 * c.mask_words, (size_t)c.mask_words * 4);
             } else {
             if (rk == 0 && lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.n_live + sid0));
             prefetch_span(c.page_table + (size_t)sid0 * c.max_pages, (size_t)c.max_pages * 4);
@@ -257,7 +257,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 prefetch_span(c.inv_norm + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
                 if (a.have_svec) prefetch_span(c.svec + (size_t)sid0 * 256, 256);
             } else {
-                prefetch_span(c.keep_mask + (size_t)local0 * c.mask_words, (size_t)c.mask_words * 4);
+                prefetch_span(c.keep_mask + (size_t)sid0 * c.mask_words, (size_t)c.mask_words * 4);
             }
             {
                 // The rows of the first tiles, too, located through a racy look at the row count and the
@@ -340,7 +340,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 vn = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[lane];
             }
             if constexpr (!FUSED) {
-                if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)local * c.mask_words + rk + lane * G];
+                if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)sid * c.mask_words + rk + lane * G];
             }
         };
         if (waited) load_inputs();
@@ -786,7 +786,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
         } else {
             if (!waited) { dep_wait(); load_inputs(); }
-            const uint32_t *gm = c.keep_mask + (size_t)local * c.mask_words;
+            const uint32_t *gm = c.keep_mask + (size_t)sid * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {
                 uint32_t bits = b == rk + lane * G ? km0 : gm[b];
                 int valid = n - b * 32;

@@ -124,6 +124,25 @@ def test_call_order_and_capacity_are_checked_before_any_launch():
     lib.adsa_destroy(ctx)
 
 
+def test_every_layer_has_its_own_selection_scratch():
+    """What one call of a layer-step leaves for the next (scores, keep mask, counts) is stored per layer, so
+    the steps of several layers may be interleaved.  Seen from the host: each extra layer adds at least
+    its scores, its carried sum, its keep mask and its counts to the workspace."""
+    base = dict(batch=3, n_heads=5, max_rows_per_stream=700)
+    S, R = 15, 700
+    per_layer = S * (R * 4 + 256 * 4 + (R + 31) // 32 * 4 + 16)
+    sizes = [A.workspace_bytes(_cfg(n_layers=n, **base)) for n in (1, 2, 5)]
+    assert sizes[1] - sizes[0] >= per_layer and sizes[2] - sizes[1] >= 3 * per_layer
+    # the step order is kept per layer: another layer being mid-step changes nothing for this one
+    lib = A.load()
+    rc, ctx = _fake_ctx(_cfg(n_pages=4000))
+    assert rc == 0
+    null, ptr = C.c_void_p(None), C.c_void_p(0x30000000)
+    assert lib.adsa_select(ctx, 1, 130, 100, null, null, null, null, null) == B.ESTATE
+    assert lib.adsa_kv_update(ctx, 1, 130, ptr, ptr, null) == B.ESTATE
+    lib.adsa_destroy(ctx)
+
+
 def test_page_division_by_multiplication_is_exact():
     # the kernels compute slot // page_rows as umulhi(slot, floor(2^32 / page_rows) + 1)
     for pr in list(range(2, 130)) + [255, 256, 1000, 4096]:

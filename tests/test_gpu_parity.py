@@ -143,40 +143,105 @@ def test_config2_full_trajectory(layer, mode):
     assert lh.stats.steps == 256
 
 
-@pytest.mark.parametrize("cfg,beta,n_sample,steps", [
-    (3, 0.5, 32, 3),
-    (4, 0.5, 32, 3),
-    (5, 0.25, 12, 2),
-    (5, 0.5, 8, 2),
-    (5, 0.75, 6, 2),
-])
-@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused", "cluster-fused"])
-def test_full_size_layer_steps(cfg, beta, n_sample, steps, mode):
-    """One layer at the full size of configs 3-5, in the launch configuration the benchmark
-    times, from a seeded late-generation state (cache full); the oracle follows a sample of streams."""
+def _bench_page_rows(C):
+    """The page size bench.py times: the largest divisor of the capacity up to 1024 rows (one page per
+    stream for the LlamaGen shapes)."""
+    return pick_page_rows(C, hi=1024)
+
+
+def _full_size_harness(w, C, page_rows, mode, n_sample, seed, n_rows, cur0, extra_rows=0):
+    """One layer of workload `w` at full size, loaded with a seeded late-generation state of n_rows rows
+    per stream as of position cur0; the oracle follows a seeded sample of the streams."""
     H = _harness()
-    w = get_workload(cfg, beta)
-    C = w.capacity()
-    rng = np.random.default_rng(cfg * 100 + int(beta * 100))
-    eng = H.engine_for(w, n_layers=1, capacity=C, page_rows=pick_page_rows(C, hi=128))
+    rng = np.random.default_rng(seed)
+    eng = H.engine_for(w, n_layers=1, capacity=C, page_rows=page_rows, extra_rows=extra_rows)
     sample = sorted(rng.choice(w.streams_per_layer, size=n_sample, replace=False).tolist())
     lh = H.LayerHarness(eng, 0, oracle_cap=C + 4, sample=sample, fused=_apply_mode(eng, mode))
+    pos, k, v = late_state(w, seed=seed, n_rows=n_rows, cur_pos=cur0)
+    lh.prefill(k.reshape(w.batch, w.n_heads, n_rows, w.head_dim), v.reshape(w.batch, w.n_heads, n_rows, w.head_dim), 0, pos)
+    lh.check_state()
+    return eng, lh
+
+
+def _pages_in_use(eng):
+    st, fs = eng.get_status()
+    assert st == 0
+    return eng.cfg.n_pages - fs[2]
+
+
+@pytest.mark.parametrize("cfg,beta,n_sample,steps,pages", [
+    (3, 0.5, 32, 3, "paged"), (3, 0.5, 32, 3, "bench"),
+    (4, 0.5, 32, 3, "paged"), (4, 0.5, 32, 3, "bench"),
+    (5, 0.25, 12, 2, "bench"),
+    (5, 0.5, 8, 2, "bench"),
+    (5, 0.75, 6, 2, "bench"),
+])
+@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused", "cluster-fused"])
+def test_full_size_layer_steps(cfg, beta, n_sample, steps, pages, mode):
+    """One layer at the full size of configs 3-5 from a seeded late-generation state (cache one row short
+    of full, then full), mid-row near the end of the grid; the oracle follows a sample of streams.
+    pages = "bench": the page size the benchmark times (one page per stream where the capacity allows);
+    "paged": pages of at most 128 rows, several per stream."""
+    w = get_workload(cfg, beta)
+    C = w.capacity()
+    pr = _bench_page_rows(C) if pages == "bench" else pick_page_rows(C, hi=128)
     g0 = w.n_cells - steps - w.grid_w // 2          # mid-row, near the end of the grid
     cur0 = w.n_text + g0
-    pos, k, v = late_state(w, seed=cfg, n_rows=C - 1, cur_pos=cur0)
-    lh.prefill(k.reshape(w.batch, w.n_heads, C - 1, w.head_dim), v.reshape(w.batch, w.n_heads, C - 1, w.head_dim), 0, pos)
-    lh.check_state()
+    eng, lh = _full_size_harness(w, C, pr, mode, n_sample, cfg * 100 + int(beta * 100), C - 1, cur0)
     for t in range(steps):
         q, kn, vn = layer_step_qkv(w, 0, 0, g0 + t)
         lh.step(q, kn, vn, cur0 + t, C)
-    st, fs = eng.get_status()
-    assert st == 0
     assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
     n_live = eng._t["n_live"].cpu().numpy()
     assert (n_live == C).all()
     # every page in use is accounted for, none leaked
-    pr = eng.cfg.page_rows
-    assert eng.cfg.n_pages - fs[2] == w.streams_per_layer * -(-C // pr)
+    assert _pages_in_use(eng) == w.streams_per_layer * -(-C // pr)
+
+
+@pytest.mark.parametrize("cfg,pages", [(3, "bench"), (3, "paged"), (4, "bench"), (4, "paged")])
+@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused"])
+def test_full_size_steps_that_change_the_code_path(cfg, pages, mode):
+    """Configs 3 and 4 at full size, in the launch configuration the benchmark times ("bench" pages) and
+    with several pages per stream, on the steps where the kernels take another branch: the step at which
+    the cache fills up, the step that ends a grid row and the one that starts the next (rows leave the
+    local window: the carried sum cannot be updated in closed form and the next scores come from a second
+    sweep), a step whose budget is smaller than the one before (several evictions at once: the general
+    selection, survivors moving into holes, pages returned), the steady steps after it, and the last two
+    cells of the grid."""
+    w = get_workload(cfg)
+    C, W, T0 = w.capacity(), w.grid_w, w.n_text
+    pr = _bench_page_rows(C) if pages == "bench" else pick_page_rows(C, hi=128)
+    S = w.streams_per_layer
+
+    # (a) two rows short of full, three cells before the end of a grid row: grow, fill up, first eviction
+    #     on the row's last cell, then the first two cells of the next row
+    g0 = (w.grid_h - 3) * W + W - 3
+    eng, lh = _full_size_harness(w, C, pr, mode, 32, cfg * 10 + 1, C - 2, T0 + g0)
+    want_rows = [C - 1, C, C, C, C]
+    for t in range(5):
+        q, kn, vn = layer_step_qkv(w, 1, 0, g0 + t)
+        lh.step(q, kn, vn, T0 + g0 + t, C)
+        assert (eng._t["n_live"].cpu().numpy() == want_rows[t]).all()
+    assert _pages_in_use(eng) == S * -(-C // pr)
+    # (b) the budget drops by 37 rows (general K: many rows go at once, survivors move down), stays there
+    #     for a step (one eviction), then is lifted again (the cache regrows without eviction)
+    g1 = g0 + 5
+    for t, budget in enumerate([C - 37, C - 37, C, C]):
+        q, kn, vn = layer_step_qkv(w, 1, 0, g1 + t)
+        lh.step(q, kn, vn, T0 + g1 + t, budget)
+    assert (eng._t["n_live"].cpu().numpy() == C - 35).all()
+    assert _pages_in_use(eng) == S * -(-(C - 35) // pr)
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+
+    # (c) the last two cells of the grid, cache full
+    g2 = w.n_cells - 2
+    eng, lh = _full_size_harness(w, C, pr, mode, 32, cfg * 10 + 2, C, T0 + g2)
+    for t in range(2):
+        q, kn, vn = layer_step_qkv(w, 2, 0, g2 + t)
+        lh.step(q, kn, vn, T0 + g2 + t, C)
+    assert (eng._t["n_live"].cpu().numpy() == C).all()
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+    assert _pages_in_use(eng) == S * -(-C // pr)
 
 
 # ---------------------------------------------------------------------------
@@ -277,27 +342,55 @@ def test_back_to_back_layers_match_serialised_launches():
     """Launches of consecutive layers overlap (the next kernel's set-up, and, when the kernel ahead serves
     another layer, its reading and selection of the cache run under the previous kernel's tail).  The
     results must be bit-identical to the same steps with the device synchronised after every launch, for
-    the fused step and for the four separate calls, over a trajectory that fills up and evicts."""
+    the fused step and for the four separate calls with the layers interleaved (score and select for every
+    layer, then every layer's attention back to back, then every update: what each call leaves for the next
+    is stored per layer), over a trajectory that fills up and evicts.  A third way of issuing the fused
+    steps alternates two streams ordered by events.  The free-running fused and four-call runs are also
+    compared with the oracle following every stream of every layer."""
     H = _harness()
+    from oracle import adsa_oracle as orc
+    from adsa_workloads import bf16_bits_to_f32
     w = Workload("layers", 95, 3, 2, 3, 64, 24, 10, 9, 0.5, 1.0)
-    C, L, S, T = w.capacity(), w.n_layers, w.streams_per_layer, w.n_cells
-    qs, ks, vs = [], [], []
+    C, L, S, T, d = w.capacity(), w.n_layers, w.streams_per_layer, w.n_cells, w.head_dim
+    bits, qs, ks, vs = [], [], [], []
     for g in range(T):
         per = [layer_step_qkv(w, 5, l, g) for l in range(L)]
+        bits.append([np.stack([x[i] for x in per]).reshape(L * S, d) for i in range(3)])
         qs.append(torch.stack([H.dev_bf16(x[0]) for x in per]))
         ks.append(torch.stack([H.dev_bf16(x[1]) for x in per]))
         vs.append(torch.stack([H.dev_bf16(x[2]) for x in per]))
-    results = []
-    for variant in ("fused-free", "fused-synced", "calls-free", "calls-synced"):
+    # the oracle: all L * S streams side by side (stream index = layer * S + stream within the layer)
+    ost = orc.OracleStreams(L * S, d, w.l_max + 1, w.n_text, w.grid_w, w.n_text)
+    pk = np.concatenate([bf16_bits_to_f32(prefix_kv(w, 5, l)[0]).reshape(S, w.n_text, d) for l in range(L)])
+    pv = np.concatenate([bf16_bits_to_f32(prefix_kv(w, 5, l)[1]).reshape(S, w.n_text, d) for l in range(L)])
+    ost.append_rows(pk, pv, 0)
+    want = np.zeros((T, L * S, d))
+    for g in range(T):
+        res = ost.step(*(bf16_bits_to_f32(b) for b in bits[g]), w.n_text + g, C)
+        want[g] = res.out
+    want_pos = np.sort(ost.pos[:, :C], axis=1)
+
+    side = torch.cuda.Stream()
+    results = {}
+    for variant in ("fused-free", "fused-synced", "fused-two-streams", "calls-free", "calls-synced"):
         eng = H.engine_for(w, capacity=C, page_rows=16)
         for l in range(L):
             k, v = prefix_kv(w, 5, l)
             eng.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
         outs = torch.zeros((T, L, S, w.head_dim), dtype=torch.bfloat16, device="cuda:0")
         synced = variant.endswith("synced")
+        main = torch.cuda.current_stream()
         for g in range(T):
             cur = w.n_text + g
-            if variant.startswith("fused"):
+            if variant == "fused-two-streams":
+                for l in range(L):                  # odd layers on the side stream, each launch ordered after the one before
+                    st = side if l & 1 else main
+                    other = main if l & 1 else side
+                    st.wait_stream(other)
+                    with torch.cuda.stream(st):
+                        eng.layer_step(l, cur, C, qs[g][l], ks[g][l], vs[g][l], outs[g, l])
+                main.wait_stream(side)
+            elif variant.startswith("fused"):
                 if synced:
                     for l in range(L):
                         eng.layer_step(l, cur, C, qs[g][l], ks[g][l], vs[g][l], outs[g, l])
@@ -314,13 +407,69 @@ def test_back_to_back_layers_match_serialised_launches():
                         torch.cuda.synchronize()
                 for l in range(L):
                     eng.kv_update(l, cur, ks[g][l], vs[g][l])
+        torch.cuda.synchronize()
         assert eng.get_status()[0] == 0
         n_live = eng._t["n_live"].cpu().numpy()
         pos = np.sort(eng._t["pos"][:, :C].cpu().numpy(), axis=1)
-        results.append((outs.cpu(), n_live, pos))
-    for a, b in ((0, 1), (2, 3)):
-        assert torch.equal(results[a][0], results[b][0])
-        assert np.array_equal(results[a][1], results[b][1]) and np.array_equal(results[a][2], results[b][2])
+        results[variant] = (outs.cpu(), n_live, pos)
+    for a, b in (("fused-free", "fused-synced"), ("fused-free", "fused-two-streams"), ("calls-free", "calls-synced")):
+        assert torch.equal(results[a][0], results[b][0]), (a, b)
+        assert np.array_equal(results[a][1], results[b][1]) and np.array_equal(results[a][2], results[b][2]), (a, b)
+    for a in ("fused-free", "calls-free"):
+        got = results[a][0].float().numpy().reshape(T, L * S, d)
+        err = np.abs(got - want)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3, (a, err.max(), err.mean())
+        assert (results[a][1] == C).all() and np.array_equal(results[a][2], want_pos), a
+
+
+def test_interleaved_layers_keep_their_own_selection():
+    """score/select of two layers, then both attentions, then both updates: each layer attends and evicts by
+    its own keep mask.  The layers get different budgets, so a mix-up changes the row counts."""
+    H = _harness()
+    w = Workload("layers2", 93, 2, 1, 4, 64, 12, 6, 6, 0.5, 1.0)
+    S, d = w.streams_per_layer, w.head_dim
+    eng = H.engine_for(w, capacity=w.l_max, page_rows=16)
+    for l in range(2):
+        k, v = prefix_kv(w, 7, l)
+        eng.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
+    out = torch.zeros((2, S, d), dtype=torch.bfloat16, device="cuda:0")
+    for g in range(20):                                  # grow both layers without eviction
+        for l in range(2):
+            q, kn, vn = (H.dev_bf16(x) for x in layer_step_qkv(w, 7, l, g))
+            eng.layer_step(l, w.n_text + g, w.l_max, q, kn, vn, out[l])
+    cur = w.n_text + 20
+    budgets = (32, 25)                                   # 32 live rows each; layer 0 evicts 1, layer 1 evicts 8
+    counts = torch.zeros((2, S, 4), dtype=torch.int32, device="cuda:0")
+    qkv = [[H.dev_bf16(x) for x in layer_step_qkv(w, 7, l, 20)] for l in range(2)]
+    for l in range(2):
+        eng.score(l, cur)
+        eng.select(l, cur, budgets[l], counts=counts[l])
+    for l in range(2):
+        eng.sparse_decode_attn(l, cur, *qkv[l], out[l])
+    for l in range(2):
+        eng.kv_update(l, cur, qkv[l][1], qkv[l][2])
+    assert eng.get_status()[0] == 0
+    n_live = eng._t["n_live"].cpu().numpy().reshape(2, S)
+    assert (n_live[0] == 32).all() and (n_live[1] == 25).all()
+    c = counts.cpu().numpy()
+    assert (c[0, :, 1] == 1).all() and (c[1, :, 1] == 8).all()
+    # and each layer's output is what the same layer gives when stepped on its own
+    ref = H.engine_for(w, capacity=w.l_max, page_rows=16)
+    for l in range(2):
+        k, v = prefix_kv(w, 7, l)
+        ref.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
+    o2 = torch.zeros((2, S, d), dtype=torch.bfloat16, device="cuda:0")
+    for g in range(20):
+        for l in range(2):
+            q, kn, vn = (H.dev_bf16(x) for x in layer_step_qkv(w, 7, l, g))
+            ref.layer_step(l, w.n_text + g, w.l_max, q, kn, vn, o2[l])
+    for l in range(2):
+        ref.score(l, cur)
+        ref.select(l, cur, budgets[l])
+        ref.sparse_decode_attn(l, cur, *qkv[l], o2[l])
+        ref.kv_update(l, cur, qkv[l][1], qkv[l][2])
+    assert torch.equal(out.cpu(), o2.cpu())
+    assert np.array_equal(np.sort(eng._t["pos"].cpu().numpy(), axis=1), np.sort(ref._t["pos"].cpu().numpy(), axis=1))
 
 
 @pytest.mark.parametrize("n_layers", [1, 4, 8])

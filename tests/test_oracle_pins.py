@@ -311,6 +311,53 @@ def test_update_invariants(n_prefix_kind):
         np.testing.assert_array_equal(v, hv[s, pos])
 
 
+def test_step_scores_the_value_rows_and_not_the_keys():
+    """Section 4.1 (the sentence before Eq. 1) takes the similarity between V rows, because rotary position
+    embedding sits on Q and K; Section 4.2 evicts the row most similar to the others.  A hand case the step
+    must get right: eight cached rows, all in the previous region, whose V rows are mutually orthogonal
+    except that the row at position 5 is a positive multiple of the row at position 2 (cosine 1); the K rows
+    are unrelated, with their own duplicate pair at positions 1 and 6.  With a budget of one row less than
+    cache + new row exactly one row goes: of the two V duplicates (equal scores 1/(p-1), all others 0) the
+    higher position, 5.  Scoring the keys instead would evict 6."""
+    d, W = 16, 4
+    rng = np.random.default_rng(21)
+    v = np.zeros((8, d), np.float32)
+    for i in range(8):
+        v[i, i] = 2.0
+    v[5] = 3.0 * v[2]
+    k = _randn(rng, 8, d)
+    k[6] = k[1]
+    cur = 5 * W + 1                      # grid row 5: the local window is rows 4-5, positions 0..7 are "previous"
+    for order in (np.arange(8), rng.permutation(8)):        # the physical order of the cache must not matter
+        st = orc.OracleStreams(1, d, 16, 0, W, 0)
+        st.load(0, np.arange(8)[order], k[order], v[order])
+        res = st.step(_randn(rng, 1, d), _randn(rng, 1, d), _randn(rng, 1, d), cur, budget=8)
+        assert res.evict_pos[0].tolist() == [5]
+        assert sorted(res.kept_pos[0].tolist()) == [0, 1, 2, 3, 4, 6, 7]
+        sc = dict(zip(res.cand_pos[0].tolist(), res.cand_score[0].tolist()))
+        assert sc[2] == sc[5] == pytest.approx(1.0 / 7.0, abs=1e-7)
+        assert all(abs(sc[p_]) < 1e-7 for p_ in (0, 1, 3, 4, 6, 7))
+
+
+def test_step_scores_equal_eq_1_2_on_the_cached_value_rows():
+    """Over whole trajectories with independent K and V draws: the scores the step reports for its
+    candidates are Eq. 1-2 of exactly those positions' V rows (taken from the full history, which the
+    step never sees), and they are not what the K rows would give."""
+    T0, H, W, d = 6, 6, 5, 8
+    C = (T0 + H * W) // 2
+    st, hk, hv, log = _run_steps(T0, H, W, d, lambda cur: C, T0, seed=22)
+    differs = 0
+    for cur, q, before, res, n_live in log:
+        for s in range(2):
+            cp = res.cand_pos[s]
+            if len(cp) == 0:
+                continue
+            np.testing.assert_array_equal(res.cand_score[s], orc.score_definition(hv[s, cp]))
+            if len(cp) >= 3 and np.abs(res.cand_score[s] - orc.score_definition(hk[s, cp])).max() > 1e-3:
+                differs += 1
+    assert differs >= 20
+
+
 def _golden_rows():
     rows = []
     with open(GOLDEN) as f:
