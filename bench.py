@@ -61,6 +61,9 @@ def parse_args():
                     help="0 streaming, 1 automatic, 2 cluster, 3 persistent on CUDA cores, 4 persistent with MMA")
     ap.add_argument("--stream-warps", type=int, default=0, help="warps per stream of the tensor-core kernel (0 = automatic)")
     ap.add_argument("--l2-ahead", type=int, default=-1, help="tiles per warp asked into L2 beyond the ring (-1 = automatic)")
+    ap.add_argument("--sweep-mode", type=int, default=2, help="adsa_set_single_sweep: 0 two sweeps, 1 single sweep, 2 single sweep + carried evictee")
+    ap.add_argument("--token-launch", type=int, default=1, help="adsa_set_token_launch: 1 one launch per token, 0 one launch per layer")
+    ap.add_argument("--next-tiles", type=int, default=-1, help="adsa_set_next_layer_hint (-1 = the library's default)")
     ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
@@ -176,6 +179,11 @@ def run_ours(args, rank, world, local_rank):
     if args.chunk_rows:
         eng.set_attn_chunk_rows(args.chunk_rows)
     eng.set_staged(args.kernel_mode)
+    if args.sweep_mode != 2:
+        eng.set_single_sweep(args.sweep_mode)
+    eng.set_token_launch(args.token_launch)
+    if args.next_tiles >= 0:
+        eng.set_next_layer_hint(args.next_tiles)
     if args.ring_stages:
         eng.set_ring_stages(args.ring_stages)
     if args.l2_ahead >= 0:

@@ -202,9 +202,13 @@ ADSA_API int adsa_layer_step(adsa_ctx *ctx, int layer, int cur_pos, int budget_r
 ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows, const void *q_host,
                          const void *k_new_host, const void *v_new_host, void *out_host, adsa_stream_t stream);
 
-/* One decoded token through every layer of an attention stack: adsa_layer_step
- * for layer 0 .. n_layers-1 with the same cur_pos and budget.  q, k_new, v_new,
- * out_bf16: [device] bf16 [n_layers][batch][n_heads][head_dim]. */
+/* One decoded token through every layer of an attention stack: what adsa_layer_step
+ * does, for layer 0 .. n_layers-1 with the same cur_pos and budget.  q, k_new, v_new,
+ * out_bf16: [device] bf16 [n_layers][batch][n_heads][head_dim].  Because every layer's
+ * inputs are given at once, no layer has to wait for another: when the tensor-core
+ * kernel serves the configuration and every layer is between steps, ONE launch walks
+ * the streams of all layers (adsa_set_token_launch); otherwise the layers are
+ * launched one after the other.  Results are those of adsa_layer_step layer by layer. */
 ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 
@@ -239,11 +243,16 @@ ADSA_API int adsa_set_staged(adsa_ctx *ctx, int mode);
  * streams per SM and the shared memory the configuration needs. */
 ADSA_API int adsa_set_stream_warps(adsa_ctx *ctx, int warps);
 
-/* 1 (default): the fused tensor-core kernel scores the next step's rows during its attention sweep
- * whenever the sum of normalised rows carried in from the previous step can be updated in closed form
- * (no eviction, or one; no rows leaving the local window); 0: it always makes a second sweep over V.
- * Same results up to rounding of the carried sum. */
-ADSA_API int adsa_set_single_sweep(adsa_ctx *ctx, int enabled);
+/* How much the fused tensor-core kernel takes over from the step before (same results up to rounding of
+ * the carried sum of normalised rows):
+ *   0  nothing but the scores: it always makes a second sweep over V for the next step's scores;
+ *   1  it scores the next step's rows during its attention sweep whenever the sum of normalised rows
+ *      carried in from the previous step can be updated in closed form (no eviction, or one; no rows
+ *      leaving the local window);
+ *   2  (default) as 1, and when the cache is exactly full it evicts the row the previous step noted as
+ *      the highest-scoring of this step's previous region instead of classifying and comparing the rows
+ *      again (the previous step leaves no note when two rows tie for the highest score or rows moved). */
+ADSA_API int adsa_set_single_sweep(adsa_ctx *ctx, int mode);
 
 /* Cap the tile ring (per CTA of the persistent kernel, per warp of the tensor-core kernel) at
  * max_stages stages (0 = as many as fit). */
@@ -254,6 +263,18 @@ ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
  * tiles per warp beyond the ring (0 = none, -1 = choose automatically, the default).  Results do not
  * depend on it. */
 ADSA_API int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles);
+
+/* adsa_token_step: 1 (default) = one launch serves every layer when it can, 0 = one launch per layer
+ * (what a decoder whose layers feed each other has to do, through adsa_layer_step). */
+ADSA_API int adsa_set_token_launch(adsa_ctx *ctx, int mode);
+
+/* Between the end of a launch's sweep and the moment the next launch has located its first rows HBM is
+ * idle.  A decoder runs its layers in order, so when a launch of the tensor-core kernel has fetched its
+ * last tile it asks the first `tiles` 32-row tiles per warp of the same streams of layer (layer + 1) mod
+ * n_layers into L2 (the 126 MB L2 holds them until that launch reads them).  A hint only: if another layer
+ * comes next the prefetch is wasted, nothing else.  In a launch that serves several layers the hint is
+ * for the stream the same warps serve next.  0 = off (default: measured, it did not pay). */
+ADSA_API int adsa_set_next_layer_hint(adsa_ctx *ctx, int tiles);
 
 /* Override the rows per attention chunk (0 = choose automatically). */
 ADSA_API int adsa_set_attn_chunk_rows(adsa_ctx *ctx, int chunk_rows);

@@ -31,7 +31,7 @@ struct LayerState {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, counts, partials, tickets, svec, status, staging, total;
+    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, status, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -47,6 +47,8 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.partials = off;    off = align_up(off + S * kMaxSplits * (size_t)(cfg.row_stride + 2) * sizeof(float), 256);
     w.tickets = off;     off = align_up(off + S * sizeof(int32_t), 256);
     w.svec = off;        off = align_up(off + S * (size_t)cfg.n_layers * 256 * sizeof(float), 256);
+    w.carry = off;       off = align_up(off + S * (size_t)cfg.n_layers * 4 * sizeof(int32_t), 256);
+    w.cand_mask = off;   off = align_up(off + S * (size_t)cfg.n_layers * mask_words_of(cfg) * sizeof(uint32_t), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
     w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
@@ -95,7 +97,11 @@ struct adsa_ctx {
     int max_stages = 0;    // cap on the persistent kernel's ring (0 = as many as fit)
     int stream_warps = 0;  // warps per stream of the warp-group kernel (0 = automatic)
     int l2_ahead = -1;     // tiles per warp the tensor-core kernel asks into L2 ahead of its ring (-1 = automatic)
-    int no_single_sweep = 0;  // 1: the fused tensor-core kernel always makes its second sweep (tests, comparisons)
+    int next_tiles = 0;    // tiles per warp of the stream served next (the next layer's, in one-layer launches) a launch asks
+                           // into L2 when its own sweep is over
+    int token_launch = 1;  // adsa_token_step: 1 = one launch of the tensor-core kernel serves every layer, 0 = one launch per layer
+    int sweep_mode = 2;    // adsa_set_single_sweep: 0 the fused tensor-core kernel always makes its second sweep, 1 it scores
+                           // during the attention sweep when it can, 2 it also takes the evicted row from the previous step's note
     // What the kernel launched last through this context may still be writing when the next one starts its
     // set-up (launches overlap by programmatic dependent launch): the layer it served (-1 = several or
     // unknown) and whether it writes the cache proper (rows, pages, positions, norms) / the carried scores.
@@ -226,7 +232,8 @@ cudaError_t launch_staged(const adsa_ctx *ctx, const StagedChoice &ch, bool fuse
 {
     if (ch.wp.n_groups)
         return launch_wstep(ctx->dev, ch.wp, ctx->maps, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st,
-                            have_svec && !ctx->no_single_sweep, state_is_quiet(ctx, layer, fused, st));
+                            have_svec && ctx->sweep_mode >= 1, state_is_quiet(ctx, layer, fused, st), ctx->sweep_mode >= 2,
+                            ctx->next_tiles > 0 ? (layer + 1) % ctx->cfg.n_layers : -1, ctx->next_tiles);
     if (ch.pp.n_stages)
         return launch_pstep(ctx->dev, ch.pp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
     return launch_step(ctx->dev, ch.sp, fused, layer, cur_pos, budget_rows, q, k_new, v_new, out_bf16, out_f32, st);
@@ -290,6 +297,8 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.partials = (float *)(w + ws.partials);
     d.tickets = (int32_t *)(w + ws.tickets);
     d.svec = (float *)(w + ws.svec);
+    d.carry = (int32_t *)(w + ws.carry);
+    d.cand_mask = (uint32_t *)(w + ws.cand_mask);
     d.status = (uint32_t *)(w + ws.status);
     d.d = cfg->head_dim;
     d.row_stride = cfg->row_stride;
@@ -550,16 +559,80 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
 {
     if (!ctx || !q || !k_new || !v_new || !out_bf16) return ADSA_EINVAL;
     if (ctx->cuda_error) return ADSA_ECUDA;
+    if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
+    const int NL = ctx->cfg.n_layers;
     size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k_new,
                         *vb = (const __nv_bfloat16 *)v_new;
     __nv_bfloat16 *ob = (__nv_bfloat16 *)out_bf16;
-    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
-        int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
-                                 vb + l * per_layer, ob + l * per_layer, stream);
-        if (rc) return rc;
+
+    // One launch for the whole stack: the caller hands over every layer's q, k_new and v_new at once, so no
+    // layer has to wait for another, and the tensor-core kernel walks the streams of all layers as one list.
+    // The warps of a multiprocessor then sit in different phases of different streams (locating rows,
+    // sweeping, updating) instead of all starting and all draining together once per layer.  Taken when
+    // every layer is between steps and in the same carried state; otherwise layer by layer.
+    bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok;
+    if (one_launch) {
+        const LayerState &L0 = ctx->layers[0];
+        for (int l = 0; l < NL && one_launch; ++l) {
+            const LayerState &L = ctx->layers[l];
+            one_launch = L.phase == kIdle && (L.scores_pos == cur_pos) == (L0.scores_pos == cur_pos) &&
+                         (L.svec_pos == cur_pos) == (L0.svec_pos == cur_pos);
+        }
     }
-    return ADSA_OK;
+    WStepPlan wp = {};
+    if (one_launch) {
+        wp = plan_wstep(ctx->dev, true, ctx->sm_count, ctx->max_stages, ctx->stream_warps, NL);
+        if (ctx->l2_ahead >= 0) wp.l2_ahead = ctx->l2_ahead;
+        one_launch = wp.n_groups > 0;
+    }
+    if (!one_launch) {
+        for (int l = 0; l < NL; ++l) {
+            int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
+                                     vb + l * per_layer, ob + l * per_layer, stream);
+            if (rc) return rc;
+        }
+        return ADSA_OK;
+    }
+    // capacity checks of adsa_select for every layer, before anything is launched
+    const int mand = mandatory_rows_bound(ctx, cur_pos) + 1;
+    const int cap = budget_rows > mand ? budget_rows : mand;
+    std::vector<int> after(NL);
+    {
+        long long need = 0;
+        for (int l = 0; l < NL; ++l) {
+            const int hi = ctx->layers[l].rows_hi;
+            after[l] = hi + 1 < cap ? hi + 1 : cap;
+            if (after[l] > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+            need += (long long)ctx->dev.S * pages_for(ctx, after[l] > hi ? after[l] : hi);
+        }
+        if (need > ctx->cfg.n_pages) return ADSA_ENOMEM;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (ctx->layers[0].scores_pos != cur_pos) {   // nothing carried in (first step, or the caches were rewritten)
+        for (int l = 0; l < NL; ++l) {
+            ++ctx->launches;
+            ctx->layers[l].svec_pos = -1;
+            note_launch(ctx, l, false, true, stream);
+            int rc = cuda_fail(ctx, launch_score(ctx->dev, l, cur_pos, nullptr, st));
+            if (rc) return rc;
+        }
+    }
+    const bool have_svec = ctx->layers[0].svec_pos == cur_pos;
+    ++ctx->launches;
+    int rc = cuda_fail(ctx, launch_wstep(ctx->dev, wp, ctx->maps, true, 0, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
+                                         st, have_svec && ctx->sweep_mode >= 1, false, ctx->sweep_mode >= 2, -1, ctx->next_tiles, NL));
+    for (int l = 0; l < NL; ++l) {
+        LayerState &L = ctx->layers[l];
+        L.rows_hi = after[l];
+        L.cur_pos = cur_pos;
+        L.scores_pos = cur_pos + 1;
+        L.svec_pos = cur_pos + 1;
+        L.launched = true;
+        L.last_stream = st;
+    }
+    note_launch(ctx, -1, true, true, stream);
+    return rc;
 }
 
 int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host, const void *k_new_host,
@@ -678,10 +751,10 @@ int adsa_set_stream_warps(adsa_ctx *ctx, int warps)
     return ADSA_OK;
 }
 
-int adsa_set_single_sweep(adsa_ctx *ctx, int enabled)
+int adsa_set_single_sweep(adsa_ctx *ctx, int mode)
 {
-    if (!ctx) return ADSA_EINVAL;
-    ctx->no_single_sweep = enabled ? 0 : 1;
+    if (!ctx || mode < 0 || mode > 2) return ADSA_EINVAL;
+    ctx->sweep_mode = mode;
     return ADSA_OK;
 }
 
@@ -696,6 +769,20 @@ int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles)
 {
     if (!ctx || tiles < -1) return ADSA_EINVAL;
     ctx->l2_ahead = tiles;
+    return ADSA_OK;
+}
+
+int adsa_set_token_launch(adsa_ctx *ctx, int mode)
+{
+    if (!ctx || mode < 0 || mode > 1) return ADSA_EINVAL;
+    ctx->token_launch = mode;
+    return ADSA_OK;
+}
+
+int adsa_set_next_layer_hint(adsa_ctx *ctx, int tiles)
+{
+    if (!ctx || tiles < 0 || tiles > 64) return ADSA_EINVAL;
+    ctx->next_tiles = tiles;
     return ADSA_OK;
 }
 

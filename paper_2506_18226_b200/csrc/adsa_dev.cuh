@@ -34,6 +34,10 @@ struct DevCtx {
     float *partials;        // [S][kMaxSplits][partial_stride]
     int32_t *tickets;       // [S]
     float *svec;            // [n_layers * S][256]  s = sum of the normalised V rows the next step scores (carried with the scores)
+    int32_t *carry;         // [n_layers * S][4]    left by a fused step for the next one: slot of the row it will evict (the
+                            //                      highest-scoring row of its previous region; -1 = not known), number of rows
+                            //                      in that region, bit 0 = some cached V row has a clamped norm, spare
+    uint32_t *cand_mask;    // [n_layers * S][mask_words]  bit s = slot s lies in the previous region of the next step
     uint32_t *status;       // [1]
     int d, row_stride, page_rows, n_pages, max_rows, max_pages, mask_words, S;
     int partial_stride;     // floats per split partial: row_stride + 2 (m, l)

@@ -79,10 +79,11 @@ struct WStepPlan {
 };
 bool wstep_supported(const DevCtx &c);
 int build_wstep_maps(const DevCtx &c, WStepMaps *out);   // 0 on success
-WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps);
+WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps, int n_run = 1);
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state);
+                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state, bool use_note,
+                         int next_layer, int next_tiles, int n_run = 1);
 cudaError_t configure_wstep_kernel(const DevCtx &c);
 
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).

@@ -75,6 +75,7 @@ constexpr int kWTileBytes = kWTile * kWRowBytes;  // one K (or V) tile
 constexpr int kWStageBytes = 2 * kWTileBytes;
 constexpr int kWMaxDepth = 8;                     // stages per warp
 constexpr int kWMaxGroupWarps = 4;                // warps that may share a stream
+constexpr int kWPart = 136;                       // floats of one warp's partial state: acc[64] | s[64] | m, l | flags
 
 // ---- PTX wrappers ---------------------------------------------------------
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
@@ -137,7 +138,7 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     WLayout L;
     uint32_t off = 0;
     L.bars = off;   off += (kWMaxGroupWarps * kWMaxDepth + 2) * 8;       // tile barriers per warp, then the metadata barrier
-    L.hdr = off;    off += kWMaxGroupWarps * 32 + 32;                     // per-warp selection partials, then the threshold
+    L.hdr = off;    off += kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16 + kWMaxGroupWarps * 8;   // per-warp selection partials, the threshold, per-warp highest carried scores, per-warp look at the next launch's stream
     L.pt = off;     off += w_align(max_pages * 4, 16);
     L.inv_words = w_align(max_rows + 8, 4);
     L.inv = off;    off += fused ? L.inv_words * 4 : 0;                   // inverse norms by slot
@@ -154,7 +155,7 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     L.candm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows in the previous region of the next step
     L.kmask = off;  off += w_align(L.mwords * 4, 16);                     // retained rows
     L.cmask = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // retained rows the next step scores
-    L.part = off;   off += kWMaxGroupWarps * 132 * 4;                     // per warp: acc[64] | s[64] | m, l
+    L.part = off;   off += kWMaxGroupWarps * kWPart * 4;                  // per warp: acc[64] | s[64] | m, l | flags
     L.hist = L.part;                                                      // radix histogram: used before any partial state exists
     off = w_align(off, 1024);                                             // the swizzle pattern repeats every 1024 bytes
     L.rings = off;
@@ -165,11 +166,16 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
 
 struct WStepArgs {
     int layer, cur_pos, budget_rows, depth;
+    int n_run;                   // consecutive layers served by this launch, starting at `layer` (q, k_new, v_new, out: [n_run][S][d])
     int group_warps, n_groups;   // warps per stream, groups per CTA
     int l2_ahead;                // tiles per warp asked into L2 beyond the ring
     uint32_t g_magic;            // x / group_warps == __umulhi(x, g_magic) for the small x used here (group_warps > 1)
     int have_svec;               // the sum of normalised rows of this step's previous region was carried in
+    int use_note;                // ... and with it the previous fused step's note (DevCtx::carry, cand_mask): which
+                                 // slots hold this step's previous region and how many; it may stand in for the classification
     int early_state;             // the cache state of this layer is not being written by the kernel ahead in the stream
+    int next_layer, next_tiles;  // the layer the next launch is expected to serve (-1 = unknown) and how many of its first
+                                 // 32-row tiles per warp this launch asks into L2 once its own sweep is over
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
     float *out_f32;
@@ -229,12 +235,15 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
     const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
+    // the local window does not move between this step and the next, and the new row stays inside it: the next
+    // step's previous region is this one's minus whatever is evicted
+    const bool steady_cut = FUSED && cut_next.lo == cut_now.lo && !new_cand;
     {
         // The first stream's metadata is asked into L2 now.  A prefetch changes no state that a program can
         // see, so it may run before the kernel launched ahead of this one has completed; the loads after
         // the wait below then find their lines (and their address translations) close by.
         const int local0 = gi * gridDim.x + blockIdx.x;
-        if (local0 < c.S && gi < a.n_groups) {
+        if (local0 < c.S * a.n_run && gi < a.n_groups) {
             const int sid0 = a.layer * c.S + local0;
             auto prefetch_span = [&](const void *ptr, size_t bytes) {
                 const char *b = reinterpret_cast<const char *>(ptr);
@@ -255,7 +264,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 prefetch_span(c.pos + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
                 prefetch_span(c.scores + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
                 prefetch_span(c.inv_norm + (size_t)sid0 * c.max_rows, (size_t)c.max_rows * 4);
-                if (a.have_svec) prefetch_span(c.svec + (size_t)sid0 * 256, 256);
+                if (a.have_svec) prefetch_span(c.svec + (size_t)sid0 * 256 + (a.cur_pos & 1) * 128, 256);
             } else {
                 prefetch_span(c.keep_mask + (size_t)sid0 * c.mask_words, (size_t)c.mask_words * 4);
             }
@@ -313,14 +322,35 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     int i_stage = 0, c_stage = 0;
     uint32_t c_par = 0;
     int streams_done = 0;
-    const int stride = gridDim.x * a.n_groups;
-    for (int local = gi * gridDim.x + blockIdx.x; local < c.S; local += stride, ++streams_done) {
+    // `local` counts the streams of this launch: those of layer a.layer first, then of the layers after it
+    // (the caller's tensors and the per-stream state are laid out in that order)
+    const int stride = gridDim.x * a.n_groups, n_local = c.S * a.n_run;
+    for (int local = gi * gridDim.x + blockIdx.x; local < n_local; local += stride, ++streams_done) {
         const int sid = a.layer * c.S + local;
         int32_t *pt = c.page_table + (size_t)sid * c.max_pages;
         const float *inv_g = c.inv_norm + (size_t)sid * c.max_rows;
         // ---- everything that only needs addresses is requested first --------------------------------
         int n = c.n_live[sid];
+        // the previous fused step's note for this one: {valid, rows in the previous region, flags}, and this lane's
+        // word of the mask of those rows by slot (32-row block rk + lane * G)
+        int4 note = make_int4(0, 0, 0, 0);
+        uint32_t cand_w = 0u;
+        const bool try_fast = FUSED && a.use_note && steady_cut;
+        if (try_fast) {
+            note = *reinterpret_cast<const int4 *>(c.carry + (size_t)sid * 4);
+            if (rk + lane * G < c.mask_words) cand_w = c.cand_mask[(size_t)sid * c.mask_words + rk + lane * G];
+        }
         for (int pg = lane; pg < c.max_pages; pg += 32) pt_s[pg] = pt[pg];   // every warp of the group writes the same values
+        // A look at the same stream of the layer the next launch will serve (its row count and first page): used for
+        // nothing but L2 hints after the sweep, range-checked, so a stale value costs a useless prefetch.
+        int *const nxt = reinterpret_cast<int *>(smem + L.hdr + kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16) + 2 * rk;
+        // (one layer per launch: the same stream of the next layer; several: the stream this group serves next)
+        const int sid2 = a.n_run == 1 ? (a.next_layer >= 0 ? a.next_layer * c.S + local : -1)
+                                      : (local + stride < n_local ? sid + stride : -1);
+        if (sid2 >= 0 && a.next_tiles > 0 && lane == 0) {
+            nxt[0] = __ldcg(c.n_live + sid2);
+            nxt[1] = __ldcg(c.page_table + (size_t)sid2 * c.max_pages);
+        }
         // the caller's inputs: q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements; for the
         // first warp elements 2*lane, 2*lane + 1 of q and of the new row's K and V; attention alone: this lane's
         // first keep-mask word.  Requested with the other prologue loads when the dependency wait is behind us.
@@ -347,6 +377,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         constexpr int kRound = 10;   // 32-row blocks whose selection inputs are fetched together
         int ps0[kRound];
         float sc0[kRound];
+        // (the positions not when the previous step's note is expected to stand in for the classification)
         if constexpr (FUSED) {
             // positions and carried scores of this warp's first blocks: requested before n is known (the
             // arrays hold max_rows entries per stream, whatever n is), so that one memory latency covers
@@ -357,12 +388,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             for (int u = 0; u < kRound; ++u) {
                 const int slot = (rk + u * G) * 32 + lane;
                 const bool in = slot < c.max_rows;
-                ps0[u] = in ? pos_g[slot] : -1;
+                ps0[u] = in && !try_fast ? pos_g[slot] : -1;
                 sc0[u] = in ? sc_g[slot] : 0.f;
             }
         }
         float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
-        if (FUSED && a.have_svec) { st0 = c.svec[(size_t)sid * 256 + 2 * lane]; st1 = c.svec[(size_t)sid * 256 + 2 * lane + 1]; }
+        // (the two halves of a stream's 256 floats take turns: a step reads one and writes the other)
+        float *const svec_in = c.svec + (size_t)sid * 256 + (a.cur_pos & 1) * 128, *const svec_out = c.svec + (size_t)sid * 256 + ((a.cur_pos + 1) & 1) * 128;
+        if (FUSED && a.have_svec) { st0 = svec_in[2 * lane]; st1 = svec_in[2 * lane + 1]; }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
         const int n_tiles = (n + kWTile - 1) / kWTile;
         const int mt = rk < n_tiles ? div_g(n_tiles - rk + G - 1) : 0;   // this warp's tiles: rk, rk + G, ...
@@ -518,7 +551,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // Eq. 1-2 for the next step on one tile of V rows: dot_i = v_i . s by MMA,
         // S_i = (dot_i/|v_i| - u_i.u_i) / (p' - 1), written at the row's new slot
         int list_ns = 0, n2 = n;   // survivors of the general compaction; live rows after the update
-        bool warp_rare = false;
+        bool warp_rare = false, warp_clamped = false;   // warp_clamped: one of the rows this warp scores has a clamped norm
         float rden = 0.f;
         // (two halves, so that the products can be issued early and their results used later)
         auto score_mma = [&](uint32_t vb, float (&dt)[2][4]) {
@@ -590,7 +623,76 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // row leaves the local window, at most one eviction), its sum of normalised rows is the carried
         // sum minus that row, known before the sweep, and the next scores are taken during pass 1.
         bool single = false;
-        if constexpr (FUSED) {
+        // The short way.  The previous fused step has scored this step's previous region and left a mask of its
+        // slots and its size; if the cache is exactly full (n = budget: K = p - 1, one row goes) and the next
+        // step's previous region is this one's minus that row, nothing has to be classified: the evicted row is
+        // the highest carried score under the mask (two equal highest scores: positions decide, the long way
+        // looks at them), all other rows are kept, the rows to score are the mask minus that row, and
+        // s' = s - u_e.  The sum of normalised rows is not summed again: s' is carried on (it is summed afresh
+        // whenever the long way runs, at least once per grid row).
+        bool fast = false;
+        if (try_fast && n == a.budget_rows && note.x == 1 && note.y >= 1) {   // the same decision in every warp of the group
+            const float *sc_g = c.scores + (size_t)sid * c.max_rows;
+            float best = -INFINITY;
+            int best_slot = -1;
+            bool tie = false;
+            for (int b0 = rk, idx0 = 0; b0 < n_tiles; b0 += kRound * G, idx0 += kRound) {
+#pragma unroll
+                for (int u = 0; u < kRound; ++u) {
+                    const int b = b0 + u * G;
+                    if (b >= n_tiles) break;
+                    const int slot = b * 32 + lane;
+                    const float sc = b0 == rk ? sc0[u] : (slot < n ? sc_g[slot] : 0.f);
+                    const uint32_t w = idx0 + u < 32 ? __shfl_sync(0xffffffffu, cand_w, idx0 + u)
+                                                     : c.cand_mask[(size_t)sid * c.mask_words + b];
+                    if (((w >> lane) & 1u) && slot < n) {
+                        if (sc > best) { best = sc; best_slot = slot; tie = false; }
+                        else if (sc == best) tie = true;
+                    }
+                }
+            }
+            float v = best;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+            const bool mine = best_slot >= 0 && best == v;
+            const unsigned who = __ballot_sync(0xffffffffu, mine);
+            tie = __any_sync(0xffffffffu, mine && tie) || __popc(who) > 1;
+            const int wslot = who ? __shfl_sync(0xffffffffu, best_slot, __ffs(who) - 1) : -1;
+            float *tops = reinterpret_cast<float *>(smem + L.hdr + kWMaxGroupWarps * 32 + 32);
+            if (lane == 0) { tops[rk * 4] = v; reinterpret_cast<int *>(tops)[rk * 4 + 1] = tie ? -1 : wslot; }
+            group_sync();
+            float gbest = -INFINITY;
+            int gslot = -1;
+            bool gtie = false;
+            for (int w = 0; w < G; ++w) {
+                const float wv = tops[w * 4];
+                const int ws = reinterpret_cast<const int *>(tops)[w * 4 + 1];
+                if (wv > gbest) { gbest = wv; gslot = ws; gtie = false; }
+                else if (wv == gbest && wv > -INFINITY) gtie = true;
+            }
+            fast = gslot >= 0 && !gtie;
+            if (fast) evict_slot = gslot;
+        }
+        if (fast) {
+            n_evict = 1; n2 = n; single = true;
+            p_next = note.y - 1;
+            rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;
+            warp_clamped = (note.z & 1) != 0;   // known for the stream as a whole
+            warp_rare = warp_clamped;
+            const uint32_t ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
+            const uint32_t *cm_g = c.cand_mask + (size_t)sid * c.mask_words;
+            for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {   // one block per lane
+                const int valid = n - b * 32;
+                uint32_t keep = valid >= 32 ? 0xffffffffu : ((1u << valid) - 1u);
+                if ((evict_slot >> 5) == b) keep &= ~(1u << (evict_slot & 31));
+                kmask[b] = keep; cmask[b] = (b == rk + lane * G ? cand_w : cm_g[b]) & keep;
+            }
+            wait(bar_meta, streams_done & 1);   // the inverse norms are in shared memory
+            const float inv_e = inv_s[evict_slot];
+            const float sp0 = fmaf(-inv_e, bf16_lo(ve), st0), sp1 = fmaf(-inv_e, bf16_hi(ve), st1);
+            make_sb(sp0, sp1);
+            if (rk == 0) { svec_out[2 * lane] = sp0; svec_out[2 * lane + 1] = sp1; }   // s' is what the next step starts from
+        } else if constexpr (FUSED) {
             const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
             const float *sc_g = c.scores + (size_t)sid * c.max_rows;
             WSelPartial mine = {0ull, -1, 0, 0, 0, 0, 0};
@@ -606,7 +708,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 float sc[kRound];
 #pragma unroll
                 for (int u = 0; u < kRound; ++u) {
-                    if (b0 == rk) { ps[u] = ps0[u]; sc[u] = sc0[u]; continue; }   // the first round came with the prologue
+                    if (b0 == rk && !try_fast) { ps[u] = ps0[u]; sc[u] = sc0[u]; continue; }   // the first round came with the prologue
                     const int slot = (b0 + u * G) * 32 + lane;
                     const bool live = b0 + u * G < n_tiles && slot < n;
                     ps[u] = live ? pos_g[slot] : -1;
@@ -780,7 +882,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         ws[slot >> 1] = h; ws[(L.w_rows + slot) >> 1] = md; ws[(2 * L.w_rows + slot) >> 1] = lo;
                     }
                 }
-                warp_rare = __any_sync(0xffffffffu, w_big >= 1.0f / kNormEps) || n2 < n;
+                warp_clamped = __any_sync(0xffffffffu, w_big >= 1.0f / kNormEps);
+                warp_rare = warp_clamped || n2 < n;
             }
             if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
                 make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
@@ -885,7 +988,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 uint32_t l0 = pack_bf16(p00 - bf16_lo(h0), p01 - bf16_hi(h0));
                 uint32_t l2 = pack_bf16(p10 - bf16_lo(h2), p11 - bf16_hi(h2));
                 uint32_t w0 = 0u, w2 = 0u;
-                if constexpr (FUSED) {
+                if (FUSED && !fast) {   // the short way carries s' on instead of summing it again: no row weights
                     w0 = w_role[(r0 + 16 * ks + 2 * t) >> 1];
                     w2 = w_role[(r0 + 16 * ks + 8 + 2 * t) >> 1];
                 }
@@ -918,12 +1021,39 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
         }
 
+        // ---- HBM has nothing more to do for this stream: the first tiles the next launch will ask for go into L2 now,
+        //      while this launch merges, updates and drains and the next one starts up ----
+        if (sid2 >= 0 && a.next_tiles > 0) {
+            const int nn = __shfl_sync(0xffffffffu, lane == 0 ? nxt[0] : 0, 0), pg0 = __shfl_sync(0xffffffffu, lane == 0 ? nxt[1] : 0, 0);
+            if (nn > 0 && nn <= c.max_rows && pg0 >= 0 && pg0 < c.n_pages) {
+                const int32_t *pt2 = c.page_table + (size_t)sid2 * c.max_pages;
+                for (int u = 0; u < a.next_tiles; ++u) {
+                    const int r0 = (rk + u * G) * kWTile, rows = min(nn, r0 + kWTile) - r0;
+                    if (rows <= 0) break;
+                    if (r0 + rows <= c.page_rows) {   // inside the first page: one bulk hint per pool
+                        if (lane < 2) {
+                            const __nv_bfloat16 *src = (lane ? c.v_pool : c.k_pool) + ((size_t)pg0 * c.page_rows + r0) * (size_t)c.row_stride;
+                            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * kWRowBytes) : "memory");
+                        }
+                    } else if (lane < rows) {         // a row per lane, located through the next stream's page table
+                        const int row = r0 + lane;
+                        const uint32_t pg = __umulhi((uint32_t)row, c.pr_magic);
+                        const int page = __ldcg(pt2 + pg);
+                        if (page >= 0 && page < c.n_pages) {
+                            const size_t off = ((size_t)page * c.page_rows + ((uint32_t)row - pg * (uint32_t)c.page_rows)) * (size_t)c.row_stride;
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
+                        }
+                    }
+                }
+            }
+        }
         // ---- this warp's state: softmax.V = roles 0 + 1, s = roles 2 + 3 + 4; then the warps of the group ----
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 4);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 8);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
         {
-            float *w = part + rk * 132;
+            float *w = part + rk * kWPart;
 #pragma unroll
             for (int md = 0; md < 4; ++md) {
                 const float lo0 = __shfl_down_sync(0xffffffffu, o_run[md][0], 1), lo2 = __shfl_down_sync(0xffffffffu, o_run[md][2], 1);
@@ -931,17 +1061,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 if (t == 0) { w[x0] = o_run[md][0] + o_run[md][1]; w[x1] = o_run[md][2] + o_run[md][3]; }
                 if (t == 1) { w[64 + x0] = (o_run[md][0] + o_run[md][1]) + lo0; w[64 + x1] = (o_run[md][2] + o_run[md][3]) + lo2; }
             }
-            if (lane == 0) { w[128] = m_run; w[129] = l_run; }
+            if (lane == 0) { w[128] = m_run; w[129] = l_run; reinterpret_cast<int *>(w)[130] = warp_clamped ? 1 : 0; }
         }
         group_sync();
         float sv0, sv1;   // s[2*lane], s[2*lane + 1]
         {
             float M = -FLT_MAX;
-            for (int w = 0; w < G; ++w) M = fmaxf(M, part[w * 132 + 128]);
+            for (int w = 0; w < G; ++w) M = fmaxf(M, part[w * kWPart + 128]);
             float Lb = 0.f, A0 = 0.f, A1 = 0.f;
             sv0 = 0.f; sv1 = 0.f;
             for (int w = 0; w < G; ++w) {
-                const float *ws = part + w * 132;
+                const float *ws = part + w * kWPart;
                 float wgt = ex2(ws[128] - M);
                 Lb = fmaf(ws[129], wgt, Lb);
                 A0 = fmaf(ws[2 * lane], wgt, A0);
@@ -963,9 +1093,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
 
         if constexpr (FUSED) {
-            if (rk == 0) {   // carried to the next step together with the scores
-                c.svec[(size_t)sid * 256 + 2 * lane] = sv0;
-                c.svec[(size_t)sid * 256 + 2 * lane + 1] = sv1;
+            if (rk == 0 && !fast) {   // carried to the next step together with the scores (the short way has written s' already)
+                svec_out[2 * lane] = sv0;
+                svec_out[2 * lane + 1] = sv1;
             }
             // ---- Section 4.2 bookkeeping: holes below the new length, survivors above it ----------
             int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;   // keys are dead now
@@ -1020,6 +1150,29 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // sweep the group has met since its last copy landed: at the merge of the partial states)
             if (!single) group_sync();
 
+            // ---- the note for the next step: its previous region by slot and by size, clamped-norm flag ----
+            if (okay) {
+                uint32_t *cm_g = c.cand_mask + (size_t)sid * c.mask_words;
+                const uint32_t new_bit = new_cand ? 1u << (last_hole & 31) : 0u;
+                if (fast) {   // one word changes: the evicted row's slot now holds the new row, which is local
+                    const int b = evict_slot >> 5;
+                    if (lane == 0 && b - div_g(b) * G == rk) cm_g[b] = cmask[b];
+                } else {
+                    for (int b = rk + lane * G; b * 32 < n2; b += 32 * G) {
+                        uint32_t word = b < n_tiles ? cmask[b] : 0u;
+                        if (b * 32 + 32 > n2) word &= (1u << (n2 - b * 32)) - 1u;   // bits of slots the update vacates
+                        if ((last_hole >> 5) == b) word |= new_bit;
+                        cm_g[b] = word;
+                    }
+                }
+            }
+            if (rk == 0 && lane == 0) {
+                int clamped = 0;
+                for (int w = 0; w < G; ++w) clamped |= reinterpret_cast<const int *>(part + w * kWPart)[130];
+                // rows that moved were scored at their new slots, but the mask above is by old slot: no note then
+                *reinterpret_cast<int4 *>(c.carry + (size_t)sid * 4) = make_int4(okay && ns == 0 ? 1 : 0, p_next, clamped, 0);
+            }
+
             // ---- the update itself, by the first warp ---------------------------------------------------
             if (okay && rk == 0) {
                 for (int i = 0; i < ns; ++i) {   // survivors move down: 8 + 8 pieces of 16 bytes
@@ -1057,7 +1210,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
         }
-        if (local + stride < c.S) group_sync();   // the stream's shared buffers are free for the next one
+        if (local + stride < n_local) group_sync();   // the stream's shared buffers are free for the next one
     }
 }
 
@@ -1111,13 +1264,29 @@ cudaError_t configure_wstep_kernel(const DevCtx &c)
 // Groups per CTA, warps per group and ring depth per warp.  As many groups as the SM has streams to
 // serve (at most 8), then as many warps per group as shared memory and the 16 warps of a CTA allow
 // with a ring of at least two tiles each.  group_warps > 0 fixes the group size.
-WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps)
+WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps, int n_run)
 {
     WStepPlan p = {};
     if (!wstep_supported(c)) return p;
-    int groups = (c.S + sm_count - 1) / sm_count;
+    const int n_streams = c.S * (n_run < 1 ? 1 : n_run);   // streams one launch serves
+    int groups = (n_streams + sm_count - 1) / sm_count;
     groups = groups < 1 ? 1 : groups > 8 ? 8 : groups;
     const int cap = max_depth > 0 && max_depth < kWMaxDepth ? max_depth : kWMaxDepth;
+    if (n_run > 1 && group_warps <= 0) {
+        // A launch over several layers has more streams than any grouping can hold at once, so the SM's time is
+        // what counts: as many warps as shared memory allows with rings of two tiles (measured on the XL shape:
+        // 5 streams x 2 warps beat 8 x 1), and among equals more streams in flight.
+        int best_groups = 0, best_g = 0;
+        for (int gr = groups; gr >= 1; --gr)
+            for (int G = kWMaxGroupWarps; G >= 1; --G) {
+                if (gr * G > 16) continue;
+                const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused).per_group;
+                const long long room = (long long)kWSmemLimit / gr - fixed;
+                if (room < 2ll * G * kWStageBytes) continue;
+                if (gr * G > best_groups * best_g) { best_groups = gr; best_g = G; }
+            }
+        if (best_groups) { groups = best_groups; group_warps = best_g; }
+    }
     for (; groups >= 1; --groups) {
         for (int G = group_warps > 0 ? group_warps : kWMaxGroupWarps; G >= 1; --G) {
             if (G > kWMaxGroupWarps || groups * G > 16) { if (group_warps > 0) break; continue; }
@@ -1130,7 +1299,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
                 p.n_groups = groups; p.group_warps = G; p.depth = depth;
                 p.l2_ahead = fused ? 1 : 0;   // measured: with the ring this makes a three-deep pipeline; deeper is slower
                 p.smem_bytes = (size_t)L.per_group * groups;
-                p.grid = c.S < sm_count ? c.S : sm_count;   // spread the streams over every SM
+                p.grid = n_streams < sm_count ? n_streams : sm_count;   // spread the streams over every SM
                 return p;
             }
             if (group_warps > 0) break;
@@ -1141,10 +1310,14 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
-                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state)
+                         float *out_f32, cudaStream_t st, bool have_svec, bool early_state, bool use_note, int next_layer, int next_tiles,
+                         int n_run)
 {
     WStepArgs a;
+    a.n_run = n_run < 1 ? 1 : n_run;
+    a.next_layer = next_layer; a.next_tiles = next_tiles;
     a.have_svec = have_svec ? 1 : 0;
+    a.use_note = have_svec && use_note ? 1 : 0;
     a.early_state = early_state ? 1 : 0;
     a.layer = layer; a.cur_pos = cur_pos; a.budget_rows = budget_rows; a.depth = plan.depth;
     a.group_warps = plan.group_warps; a.n_groups = plan.n_groups; a.l2_ahead = plan.l2_ahead;

@@ -15,12 +15,14 @@ def _harness():
     return harness
 
 
-MODES = ["calls", "fused", "two-sweep-fused", "streaming", "cluster-calls", "cluster-fused", "cores-calls", "cores-fused"]
+MODES = ["calls", "fused", "two-sweep-fused", "reselect-fused", "streaming", "cluster-calls", "cluster-fused", "cores-calls", "cores-fused"]
 # calls: the four C-ABI calls one by one (attention by the persistent pipelined kernel, tensor-core
 #        arithmetic where the pool rows are 64 elements wide);
 # fused: adsa_layer_step, one persistent kernel per layer-step, scores carried from step to step;
 # two-sweep-fused: the fused kernel always scoring in a second sweep over V (by default it scores during the
 #        attention sweep whenever the carried sum of normalised rows can be updated in closed form);
+# reselect-fused: the fused kernel making the full selection at every step (by default, when the cache is
+#        exactly full, it evicts the row the previous step noted as the highest-scoring one);
 # streaming: the four calls with the staged kernels switched off (the register-streaming attention);
 # cluster-*: the same two ways of calling, with the one-cluster-per-stream kernel;
 # cores-*: the same, with the persistent kernel forced onto the CUDA cores.
@@ -34,7 +36,9 @@ def _apply_mode(eng, mode):
     elif mode.startswith("cores"):
         eng.set_staged(3)
     elif mode.startswith("two-sweep"):
-        eng.set_single_sweep(False)
+        eng.set_single_sweep(0)
+    elif mode.startswith("reselect"):
+        eng.set_single_sweep(1)
     return mode.endswith("fused")
 
 
