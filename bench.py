@@ -11,15 +11,19 @@ no trained weights); the default is the XL shape (36 layers, batch 32 = 16 promp
   python bench.py --impl reference ...      # times the CPU oracle instead (a deliberately slow program)
 
 The timed region is the LAST K grid cells of a generation (cache full: the most expensive
-cells); the cells before them are decoded untimed first, which is also the warm-up.  With
-the default K = H*W the whole generation is timed and a full untimed generation precedes it.
-One JSON line is printed by rank 0.
+cells).  With K below H*W the cache is loaded with a seeded late-generation state (text rows, the
+two most recent grid rows, a random subset of older cells per stream), W cells are decoded untimed
+and K cells timed; this is repeated until about half a second has been timed and the median
+region is reported.  With the default K = H*W a whole generation is timed after a whole untimed one.
+One JSON line is printed by rank 0; besides the headline workload it carries short measurements of
+the other configurations (`detail.all_configs`) and a memory-against-batch table (`detail.memory_vs_batch`).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -35,45 +39,48 @@ import torch  # noqa: E402
 from adsa_workloads import get_workload, late_state, pick_page_rows  # noqa: E402
 
 METRIC, UNIT = "image_tokens_per_s", "image-tokens/s"
-INPUT_RING_BYTES = 24 << 30   # q/k/v for all steps are kept in HBM up to this size, else a ring of steps is cycled
-
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
-# under profiles/, keyed by workload; None where no capture of the current kernel exists.
-STEP_DRAM_TRAFFIC_BYTES = {"cfg4": 98622720 + 3850112}    # profiles/step_kernel_cfg4_2layers.md
-ATTN_DRAM_TRAFFIC_BYTES = {"cfg4": 94057600 + 3473536}     # profiles/attn_kernel_cfg4_2layers.md
+INPUT_RING_BYTES = 12 << 30   # q/k/v of the decoded cells are kept in HBM up to this size, else a ring of cells is cycled
+TIMED_SECONDS = 0.5           # repeats of the timed region add up to about this much device time
+LLAMAGEN_XL_PARAM_BYTES = 775_000_000 * 2   # bf16 weights of the 775 M-parameter XL decoder (context for the memory table)
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "selftest"])
+    ap.add_argument("--workload", default="cfg4", help="cfg1 .. cfg5: the headline workload of the JSON line")
     ap.add_argument("--beta", type=float, default=None)
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-all-configs", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--no-memory-sweep", action="store_true", help="skip the memory-against-batch table")
+    ap.add_argument("--no-detail", action="store_true",
+                    help="headline region only: no per-call, attention-alone or per-layer-launch timing")
     ap.add_argument("--chunk-rows", type=int, default=0, help="override rows per attention chunk (0 = automatic)")
-    ap.add_argument("--page-rows", type=int, default=0, help="rows per pool page (0 = the largest divisor of the capacity up to 128)")
+    ap.add_argument("--page-rows", type=int, default=0, help="rows per pool page (0 = the largest divisor of the capacity up to 1024)")
     ap.add_argument("--kernel-mode", type=int, default=1,
                     help="0 streaming, 1 automatic, 2 cluster, 3 persistent on CUDA cores, 4 persistent with MMA")
     ap.add_argument("--stream-warps", type=int, default=0, help="warps per stream of the tensor-core kernel (0 = automatic)")
     ap.add_argument("--l2-ahead", type=int, default=-1, help="tiles per warp asked into L2 beyond the ring (-1 = automatic)")
-    ap.add_argument("--sweep-mode", type=int, default=2, help="adsa_set_single_sweep: 0 two sweeps, 1 single sweep, 2 single sweep + carried evictee")
+    ap.add_argument("--sweep-mode", type=int, default=2,
+                    help="adsa_set_single_sweep: 0 two sweeps, 1 single sweep, 2 single sweep + carried evictee")
     ap.add_argument("--token-launch", type=int, default=1, help="adsa_set_token_launch: 1 one launch per token, 0 one launch per layer")
     ap.add_argument("--next-tiles", type=int, default=-1, help="adsa_set_next_layer_hint (-1 = the library's default)")
     ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
-                    help="bracket the timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`)")
-    return ap.parse_args()
+                    help="bracket ONE timed region with cudaProfilerStart/Stop (for `ncu --profile-from-start off`); no repeats")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend when several ranks run")
+    return ap.parse_args(argv)
 
 
-def _workload(args):
+def _workload(args, name=None, beta=None):
     from dataclasses import replace
-    w = get_workload(int(args.workload.replace("cfg", "")), args.beta)
-    return w if args.layers is None else replace(w, n_layers=args.layers, name=f"{w.name}-{args.layers}layers")
+    w = get_workload(int((name or args.workload).replace("cfg", "")), beta if name else args.beta)
+    return w if args.layers is None or name else replace(w, n_layers=args.layers, name=f"{w.name}-{args.layers}layers")
 
 
 def peaks():
@@ -82,6 +89,20 @@ def peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def dram_traffic(kind, workload, page_rows, launch):
+    """DRAM bytes (read + written) per layer-step from the ncu captures summarised under profiles/, or None
+    when no capture matches the kernel configuration that was timed."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            for e in json.load(f)["entries"]:
+                if (e["kind"], e["workload"], e["page_rows"], e["launch"]) == (kind, workload, page_rows, launch):
+                    return e["dram_bytes_per_layer_step"]
+    except (OSError, KeyError, ValueError):
+        pass
+    return None
 
 
 # --------------------------------------------------------------------------------------
@@ -98,6 +119,20 @@ def aggregate(ms_local: float, units_local: float, world: int):
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(t.item()), float(u.item())
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_replicas(n, argv):
+    """`--gpus N` given to a plain `python bench.py`: start N ranks of this file under torch.distributed.run
+    (one per GPU; rank 0 prints the line), as a multi-process launcher would, and return its exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(_free_port()), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
 
 
 class ClockSampler:
@@ -139,94 +174,289 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    return vis.split(",")[local_rank] if vis else local_rank
+
+
 # --------------------------------------------------------------------------------------
-# the CUDA path
+# the CUDA path: one attention stack, its inputs and the ways of decoding a grid cell
 # --------------------------------------------------------------------------------------
-def make_inputs(w, n_steps, dev, seed):
-    """Seeded N(0, sigma^2) bf16 q/k/v [n_steps, L, batch, heads, d] and the text-condition rows, in HBM."""
-    g = torch.Generator(device=dev).manual_seed(seed)
-    shape = (w.n_layers, w.batch, w.n_heads, w.head_dim)
-    per_step = 3 * int(np.prod(shape)) * 2
-    ring = min(n_steps, max(8, INPUT_RING_BYTES // per_step))
-    qkv = [torch.empty((ring,) + shape, dtype=torch.bfloat16, device=dev) for _ in range(3)]
-    for t in qkv:
-        for i in range(ring):
-            t[i] = (torch.randn(shape, generator=g, device=dev) * w.sigma).to(torch.bfloat16)
-    pshape = (w.n_layers, w.batch, w.n_heads, w.n_text, w.head_dim)
-    pk = (torch.randn(pshape, generator=g, device=dev) * w.sigma).to(torch.bfloat16)
-    pv = (torch.randn(pshape, generator=g, device=dev) * w.sigma).to(torch.bfloat16)
-    return qkv, (pk, pv), ring
+class Stack:
+    """An engine shaped like workload `w` with seeded q/k/v for `n_cells` grid cells resident in HBM."""
 
-
-def run_ours(args, rank, world, local_rank):
-    from paper_2506_18226_b200 import AdsaEngine
-
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    w = _workload(args)
-    C, HW, T0, L = w.capacity(), w.n_cells, w.n_text, w.n_layers
-    K = HW if args.steps is None else max(1, args.steps)
-    W = max(3, args.warmup)
-    # Large pages keep a stream's rows contiguous, so that one TMA box covers a whole tile; the default is
-    # the largest divisor of the capacity up to 1024 rows (cfg4: one 572-row page per stream), which also
-    # makes a full stream occupy whole pages: pool bytes = the budget's share of dense, exactly.
-    pr = args.page_rows if args.page_rows else pick_page_rows(C, hi=1024)
-    pages_per_stream = -(-C // pr)
-    eng = AdsaEngine(n_layers=L, batch=w.batch, n_heads=w.n_heads, head_dim=w.head_dim, n_text=T0, grid_h=w.grid_h,
-                     grid_w=w.grid_w, max_rows_per_stream=max(C, T0 + 2 * w.grid_w), page_rows=pr,
-                     n_pages=L * w.streams_per_layer * max(pages_per_stream, -(-(T0 + 2 * w.grid_w) // pr)),
-                     device=str(dev))
-    if args.chunk_rows:
-        eng.set_attn_chunk_rows(args.chunk_rows)
-    eng.set_staged(args.kernel_mode)
-    if args.sweep_mode != 2:
+    def __init__(self, w, args, dev, rank, n_cells):
+        from paper_2506_18226_b200 import AdsaEngine
+        self.w, self.dev = w, dev
+        self.C, self.T0, self.L, self.HW = w.capacity(), w.n_text, w.n_layers, w.n_cells
+        # Large pages keep a stream's rows contiguous, so that one TMA box covers a whole tile; the default is
+        # the largest divisor of the capacity up to 1024 rows (cfg4: one 572-row page per stream), which also
+        # makes a full stream occupy whole pages: pool bytes = the budget's share of dense, exactly.
+        self.page_rows = args.page_rows if args.page_rows else pick_page_rows(self.C, hi=1024)
+        max_rows = max(self.C, self.T0 + 2 * w.grid_w)
+        self.eng = eng = AdsaEngine(n_layers=self.L, batch=w.batch, n_heads=w.n_heads, head_dim=w.head_dim, n_text=self.T0,
+                                    grid_h=w.grid_h, grid_w=w.grid_w, max_rows_per_stream=max_rows, page_rows=self.page_rows,
+                                    n_pages=self.L * w.streams_per_layer * -(-max_rows // self.page_rows), device=str(dev))
+        if args.chunk_rows:
+            eng.set_attn_chunk_rows(args.chunk_rows)
+        eng.set_staged(args.kernel_mode)
         eng.set_single_sweep(args.sweep_mode)
-    eng.set_token_launch(args.token_launch)
-    if args.next_tiles >= 0:
-        eng.set_next_layer_hint(args.next_tiles)
-    if args.ring_stages:
-        eng.set_ring_stages(args.ring_stages)
-    if args.l2_ahead >= 0:
-        eng.set_l2_lookahead(args.l2_ahead)
-    if args.stream_warps:
-        eng.set_stream_warps(args.stream_warps)
-    (q, k, v), (pk, pv), ring = make_inputs(w, HW, dev, args.seed + 1000 * rank)
-    out = torch.zeros((2, L, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        eng.set_token_launch(args.token_launch)
+        if args.next_tiles >= 0:
+            eng.set_next_layer_hint(args.next_tiles)
+        if args.ring_stages:
+            eng.set_ring_stages(args.ring_stages)
+        if args.l2_ahead >= 0:
+            eng.set_l2_lookahead(args.l2_ahead)
+        if args.stream_warps:
+            eng.set_stream_warps(args.stream_warps)
+        self.seed = args.seed + 1000 * rank
+        g = torch.Generator(device=dev).manual_seed(self.seed)
+        self.shape = (self.L, w.batch, w.n_heads, w.head_dim)
+        per_cell = 3 * int(np.prod(self.shape)) * 2
+        self.ring = max(1, min(n_cells, max(8, INPUT_RING_BYTES // per_cell)))
+        self.qkv = [torch.empty((self.ring,) + self.shape, dtype=torch.bfloat16, device=dev) for _ in range(3)]
+        for t in self.qkv:
+            for i in range(self.ring):
+                t[i] = (torch.randn(self.shape, generator=g, device=dev) * w.sigma).to(torch.bfloat16)
+        self.out = torch.zeros((2,) + self.shape, dtype=torch.bfloat16, device=dev)
 
-    def start_generation():
-        eng.reset()
-        if T0:
-            for l in range(L):
-                eng.prefill_rows(l, pk[l], pv[l], 0)
+    # -- cache states ----------------------------------------------------------------
+    def _rows(self, g, n):
+        w = self.w
+        return (torch.randn((w.batch, w.n_heads, n, w.head_dim), generator=g, device=self.dev) * w.sigma).to(torch.bfloat16)
 
-    def decode(g):
-        eng.token_step(T0 + g, C, q[g % ring], k[g % ring], v[g % ring], out[g & 1])
+    def start_generation(self):
+        """Empty caches, then the text condition of every layer."""
+        self.eng.reset()
+        g = torch.Generator(device=self.dev).manual_seed(self.seed + 1)
+        if self.T0:
+            for l in range(self.L):
+                self.eng.prefill_rows(l, self._rows(g, self.T0), self._rows(g, self.T0), 0)
 
-    # ---- warm-up generation; its last cells also time the attention kernel on its own ----------
-    M = min(8, HW // 2)
-    start_generation()
-    for g in range(HW - 2 * M):
-        decode(g)
+    def load_late(self, cell):
+        """The caches as they look when `cell` is about to be decoded, without decoding the cells before it:
+        the text rows, the two most recent grid rows and, per stream, a random subset of the older cells
+        (min(capacity, context) rows in all), in shuffled physical order, with seeded N(0, sigma^2) payloads."""
+        w, T0 = self.w, self.T0
+        if cell <= 0:
+            return self.start_generation()
+        cur = T0 + cell
+        n = min(self.C, cur)
+        lo = max(T0, cur - 2 * w.grid_w)
+        text = torch.arange(0, T0, device=self.dev)
+        recent = torch.arange(lo, cur, device=self.dev)
+        older = torch.arange(T0, lo, device=self.dev)
+        n_old = n - T0 - recent.numel()
+        assert 0 <= n_old <= older.numel(), "capacity below text condition + two grid rows"
+        S = w.streams_per_layer
+        self.eng.reset()
+        g = torch.Generator(device=self.dev).manual_seed(self.seed + 2 + cell)
+        for l in range(self.L):
+            parts = [text.expand(S, -1)]
+            if n_old:
+                pick = torch.rand((S, older.numel()), generator=g, device=self.dev).argsort(dim=1)[:, :n_old]
+                parts.append(older[pick])
+            parts.append(recent.expand(S, -1))
+            rows = torch.cat(parts, dim=1)
+            perm = torch.rand((S, n), generator=g, device=self.dev).argsort(dim=1)
+            pos = rows.gather(1, perm).to(torch.int32).view(w.batch, w.n_heads, n).contiguous()
+            self.eng.prefill_rows(l, self._rows(g, n), self._rows(g, n), 0, pos)
+
+    # -- decoding one grid cell --------------------------------------------------------
+    def decode(self, g):
+        """One token through the whole stack (adsa_token_step)."""
+        i = g % self.ring
+        self.eng.token_step(self.T0 + g, self.C, self.qkv[0][i], self.qkv[1][i], self.qkv[2][i], self.out[g & 1])
+
+    def decode_by_layer(self, g):
+        """The same through adsa_layer_step, one launch per layer."""
+        i = g % self.ring
+        for l in range(self.L):
+            self.eng.layer_step(l, self.T0 + g, self.C, self.qkv[0][i, l], self.qkv[1][i, l], self.qkv[2][i, l], self.out[g & 1, l])
+
+    def full_cell(self):
+        """First grid cell at which the cache is full before the step (one eviction per step from there on)."""
+        return max(0, self.C - self.T0)
+
+    def bytes_per_layer_step(self, rows_before):
+        """Algorithmic bytes of one fused layer-step and of attention alone, for `rows_before` live rows per
+        stream at a full cache: retained rows x (K + V) + 16 B of metadata per live row (position, carried score,
+        inverse norm read; next score written) + q, k_new, v_new, out and the new row's K and V."""
+        w = self.w
+        d2 = w.head_dim * 2
+        retained = rows_before - 1 if rows_before >= self.C else rows_before
+        step = w.streams_per_layer * (retained * 2 * d2 + rows_before * 16 + 6 * d2)
+        attn = w.streams_per_layer * (retained * 2 * d2 + 4 * d2)
+        return step, attn
+
+
+def timed_region(st, first, K, W, world, profiler=False):
+    """Decode cells first .. first+K-1 between two CUDA events, after W untimed cells from a loaded state
+    (or, for a whole generation, after an untimed generation).  Returns (ms, launches, per-cell events)."""
+    HW = st.HW
+    if first == 0 and K >= HW:
+        st.start_generation()
+        for g in range(HW):                       # the warm-up generation
+            st.decode(g)
+        st.start_generation()
+    else:
+        st.load_late(max(0, first - W))
+        for g in range(max(0, first - W), first):
+            st.decode(g)
+    torch.cuda.synchronize(st.dev)
+    if world > 1:
+        torch.distributed.barrier()
+    n0 = st.eng.launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cells = []
+    if profiler:
+        torch.cuda.profiler.start()
+    t0.record()
+    g = first
+    for _ in range(K):
+        if g == HW:                               # K > H*W: another generation inside the timed region
+            st.start_generation()
+            g = 0
+        st.decode(g)
+        g += 1
+        if first == 0 and K == HW:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record()
+            cells.append((g - 1, e))
+    t1.record()
+    torch.cuda.synchronize(st.dev)
+    if profiler:
+        torch.cuda.profiler.stop()
+    if world > 1:
+        torch.distributed.barrier()
+    return t0.elapsed_time(t1), st.eng.launch_count() - n0, (t0, cells)
+
+
+def _roofline(kind, label, bytes_per_unit, us_per_unit, units_per_launch, launches, traffic):
+    peak, peak_kind = peaks()
+    gbs = bytes_per_unit / (us_per_unit * 1e-6) / 1e9
+    return {"bound": "hbm", "kernel": label, "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+            "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": gbs / 8000.0,
+            "us_per_layer_step": us_per_unit, "layer_steps_per_launch": units_per_launch,
+            "us_per_launch": us_per_unit * units_per_launch, "launches_timed": launches,
+            "algorithmic_bytes_per_layer_step": bytes_per_unit,
+            "algorithmic_bytes_per_launch": bytes_per_unit * units_per_launch,
+            "traffic": None if traffic is None else traffic * units_per_launch, "kind": kind}
+
+
+def pool_record(st, peak_pool_bytes):
+    """Bytes of the paged pool at its high-water mark against a dense cache, with the per-row and per-stream
+    state the library keeps beside the pool (positions, inverse norms, carried scores: 12 B per row slot;
+    carried sum, masks, counts, notes, page table per stream) counted as metadata."""
+    w, cfg = st.w, st.eng.cfg
+    n_streams = st.L * w.streams_per_layer
+    mask_words = (cfg.max_rows_per_stream + 31) // 32
+    max_pages = -(-cfg.max_rows_per_stream // cfg.page_rows)
+    meta = n_streams * (cfg.max_rows_per_stream * 12 + 256 * 4 + 2 * mask_words * 4 + 16 + 16 + max_pages * 4 + 4)
+    dense = w.dense_kv_bytes() * st.L // w.n_layers
+    return {"peak_bytes": peak_pool_bytes, "dense_bytes": dense, "ratio": peak_pool_bytes / dense,
+            "payload_bytes": peak_pool_bytes * w.head_dim // cfg.row_stride,
+            "payload_ratio": peak_pool_bytes * w.head_dim / cfg.row_stride / dense,
+            "metadata_bytes": meta, "ratio_with_metadata": (peak_pool_bytes + meta) / dense,
+            "row_stride": cfg.row_stride, "page_rows": cfg.page_rows, "budget_fraction": w.beta}
+
+
+def measure(w, args, dev, rank, world, local_rank, K, W, detail=True):
+    """The timed region of one workload (median of repeats), its rooflines and, on request, the separate
+    timings at a full cache: per-layer launches, attention alone, the four calls one by one."""
+    HW = w.n_cells
+    K = HW if K is None else max(1, K)
+    first = (HW - K) % HW if K % HW else 0
+    whole = first == 0 and K >= HW
+    M = max(1, min(8, HW // 4))
+    st = Stack(w, args, dev, rank, HW if whole else min(HW, K + W + M + 4))
+    eng, L, C, T0 = st.eng, st.L, st.C, st.T0
+    prompts = w.batch // 2 if w.batch >= 2 else w.batch
+
+    sampler = ClockSampler(gpu_index(local_rank))
+    sampler.start()
+    ms0, launches, (t0, cells) = timed_region(st, first, K, W, world, profiler=args.profiler_range)
+    regions = [ms0]
+    if not whole and not args.profiler_range:
+        worst, _ = aggregate(ms0, 0.0, world)              # every rank repeats the same number of times
+        repeats = int(min(40, max(3, np.ceil(TIMED_SECONDS * 1e3 / max(worst, 1e-3)))))
+        for _ in range(repeats - 1):
+            regions.append(timed_region(st, first, K, W, world)[0])
+    clocks = sampler.stop()
+    status, _ = eng.get_status()
+    assert status == 0, f"device status {status} after the timed region"
+    ms_local = float(np.median(regions))
+    ms, tokens = aggregate(ms_local, float(prompts * K), world)
+    rows_now = int(eng._t["n_live"].max().item())
+    assert int(eng._t["n_live"].min().item()) == rows_now == min(C, T0 + HW)
+    peak_pool_bytes = eng.pool_bytes_peak()
+
+    res = {"workload": w, "stack": st, "K": K, "W": W, "first": first, "ms": ms, "tokens": tokens, "launches": launches,
+           "clocks": clocks, "regions": len(regions), "region_ms_min_max": [float(min(regions)), float(max(regions))],
+           "kv_pool": pool_record(st, peak_pool_bytes), "prompts": prompts, "detail": {}}
+
+    # ---- roofline of the headline path at a full cache -------------------------------------------
+    step_bytes, attn_bytes = st.bytes_per_layer_step(rows_now)
+    launch_kind = "token-launch" if launches == K else "layer-launch"
+    if whole:
+        prev, per_cell = t0, {}
+        for gcell, e in cells:
+            per_cell[gcell] = prev.elapsed_time(e) * 1e3 / L
+            prev = e
+        span = lambda a, n=16: float(np.median([per_cell[i] for i in range(a, min(HW, a + n))]))
+        res["detail"]["fused_layer_step_us_by_cell"] = {
+            "start_cells_0_15": span(0), "middle": span(max(0, HW // 2 - 8)), "end_last_16": span(max(0, HW - 16)),
+            "rows_at": {"start": T0 + 1, "middle": min(C, T0 + HW // 2), "end": min(C, T0 + HW)}}
+        us_unit, n_timed = span(max(0, HW - 16)), 16 * launches // K
+    elif first >= st.full_cell():
+        us_unit, n_timed = ms_local * 1e3 / (K * L), launches
+    else:
+        us_unit, n_timed = None, 0
+    if us_unit:
+        per_launch = L if launch_kind == "token-launch" else 1
+        res["roofline"] = _roofline("fused", f"fused layer-step (adsa_token_step, {launch_kind}: {per_launch} layer-step(s) per launch)",
+                                    step_bytes, us_unit, per_launch, n_timed,
+                                    dram_traffic("fused", args.workload if w.name.startswith(args.workload) else w.name[:4],
+                                                 st.page_rows, launch_kind))
+    if detail and rank == 0 and T0 + HW > C:
+        res["detail"].update(full_cache_detail(st, args, M, step_bytes, attn_bytes))
+    return res
+
+
+def full_cache_detail(st, args, M, step_bytes, attn_bytes):
+    """Separate timings over the last M cells (cache full): the fused step launched layer by layer, the
+    attention call alone (every layer's launch back to back, after every layer's score and select), and each
+    of the four calls.  The keep masks are per layer, so the grouped calls are a valid trajectory."""
+    eng, L, C, T0, HW, dev = st.eng, st.L, st.C, st.T0, st.HW, st.dev
+    out = {}
+    wname = st.w.name[:4]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # the fused layer-step kernel on its own, cache full: L launches per cell, each a different layer's KV
-    step_ms, step_launches = 0.0, 0
-    for g in range(HW - 2 * M, HW - M):
-        torch.cuda.synchronize(dev)
-        n0 = eng.launch_count()
-        e0.record()
-        decode(g)
-        e1.record()
-        torch.cuda.synchronize(dev)
-        step_ms += e0.elapsed_time(e1)
-        step_launches += eng.launch_count() - n0
-    rows_step = int(eng._t["n_live"].max().item())
-    # (the keep mask and counts are stored per layer, so grouping the calls like this is a valid trajectory: every
-    # layer attends and evicts by its own selection; the timed generation below starts from a reset all the same)
-    attn_ms, attn_launches = 0.0, 0
-    call_ms = {"adsa_score": [], "adsa_select": [], "adsa_sparse_decode_attn": [], "adsa_kv_update": []}
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    # (1) one launch per layer, as a decoder whose layers feed each other has to do
+    eng.set_token_launch(0)
+    st.load_late(HW - M - 2)
+    for g in range(HW - M - 2, HW - M):
+        st.decode_by_layer(g)
+    torch.cuda.synchronize(dev)
+    n0 = eng.launch_count()
+    e0.record()
     for g in range(HW - M, HW):
-        cur, r = T0 + g, g % ring
+        st.decode_by_layer(g)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    launches = eng.launch_count() - n0
+    out["roofline_layer_launch"] = _roofline("fused", "fused layer-step, one launch per layer (adsa_layer_step)", step_bytes,
+                                             e0.elapsed_time(e1) * 1e3 / launches, 1, launches,
+                                             dram_traffic("fused", wname, st.page_rows, "layer-launch"))
+    eng.set_token_launch(args.token_launch)
+    # (2) the four calls
+    st.load_late(HW - M)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    call_us = {"adsa_score": [], "adsa_select": [], "adsa_sparse_decode_attn": [], "adsa_kv_update": []}
+    attn_ms = 0.0
+    for g in range(HW - M, HW):
+        cur, i = T0 + g, g % st.ring
+        q, k, v = (t[i] for t in st.qkv)
         ev[0].record()
         for l in range(L):
             eng.score(l, cur)
@@ -235,155 +465,158 @@ def run_ours(args, rank, world, local_rank):
             eng.select(l, cur, C)
         ev[2].record()
         for l in range(L):                          # L launches back to back, each reads a different layer's KV
-            eng.sparse_decode_attn(l, cur, q[r, l], k[r, l], v[r, l], out[g & 1, l])
+            eng.sparse_decode_attn(l, cur, q[l], k[l], v[l], st.out[g & 1, l])
         ev[3].record()
         for l in range(L):
-            eng.kv_update(l, cur, k[r, l], v[r, l])
+            eng.kv_update(l, cur, k[l], v[l])
         ev[4].record()
         torch.cuda.synchronize(dev)
         attn_ms += ev[2].elapsed_time(ev[3])
-        attn_launches += L
-        if g > HW - M:      # in the first of these cells the scores were left behind by the fused step: no score kernel runs
-            for i, name in enumerate(call_ms):
-                call_ms[name].append(ev[i].elapsed_time(ev[i + 1]) * 1e3 / L)
-    status, _ = eng.get_status()
-    assert status == 0, f"device status {status} after the warm-up generation"
-    n_live = eng._t["n_live"]
-    rows_full = int(n_live.max().item())
-    assert int(n_live.min().item()) == rows_full == min(C, T0 + HW)
-    peak_pool_bytes = eng.pool_bytes_peak()
+        for j, name in enumerate(call_us):
+            call_us[name].append(ev[j].elapsed_time(ev[j + 1]) * 1e3 / L)
+    assert eng.get_status()[0] == 0
+    out["roofline_attn"] = _roofline("attn", "attention alone (adsa_sparse_decode_attn)", attn_bytes, attn_ms * 1e3 / (M * L), 1,
+                                     M * L, dram_traffic("attn", wname, st.page_rows, "layer-launch"))
+    per_call = {n: float(np.median(v)) for n, v in call_us.items()}
+    per_call["four_call_sequence"] = float(sum(per_call.values()))
+    out["per_call_us_cache_full"] = per_call
+    return out
 
-    # ---- timed: the last K cells of a generation ----------------------------------------------
-    start_generation()
-    first = (HW - K) % HW if K % HW else 0
-    for g in range(first):
-        decode(g)
-    torch.cuda.synchronize(dev)
-    if world > 1:
-        torch.distributed.barrier()
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
-    sampler.start()
-    launches0 = eng.launch_count()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if args.profiler_range:
-        torch.cuda.profiler.start()
-    t0.record()
-    g = first
-    cell_ev = []                                    # one event per cell: where in the generation the time goes
-    for _ in range(K):
-        if g == HW:                                 # K > H*W: start another generation inside the timed region
-            start_generation()
-            g = 0
-        decode(g)
-        g += 1
-        if K <= 4096:
-            e = torch.cuda.Event(enable_timing=True)
-            e.record()
-            cell_ev.append((g - 1, e))
-    t1.record()
-    torch.cuda.synchronize(dev)
-    if args.profiler_range:
-        torch.cuda.profiler.stop()
-    if world > 1:
-        torch.distributed.barrier()
-    ms_local = t0.elapsed_time(t1)
-    clocks = sampler.stop()
-    launches = eng.launch_count() - launches0
-    status, _ = eng.get_status()
-    assert status == 0, f"device status {status} after the timed region"
 
-    prompts = w.batch // 2 if w.batch >= 2 else w.batch
-    ms, tokens = aggregate(ms_local, float(prompts * K), world)
-
-    # ---- end to end: same cells through the host-buffer entry point -----------------------------
-    e2e = None
-    if not args.no_e2e:
-        Ke = min(K, 256, HW)
-        start_generation()
-        for g in range(HW - Ke):
-            decode(g)
-        shape = (L, w.batch, w.n_heads, w.head_dim)
-        hq, hk, hv = (torch.empty((Ke,) + shape, dtype=torch.bfloat16).pin_memory() for _ in range(3))
-        for i, g in enumerate(range(HW - Ke, HW)):
-            hq[i].copy_(q[g % ring]); hk[i].copy_(k[g % ring]); hv[i].copy_(v[g % ring])
-        ho = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
-        torch.cuda.synchronize(dev)
+def end_to_end(st, args, K, W, world, prompts):
+    """The same cells through adsa_token_step_host: pinned host q/k/v in, host output out, every step's copies
+    inside the timed region, which is bracketed by wall-clock reads after a device synchronisation."""
+    HW, T0, C = st.HW, st.T0, st.C
+    Ke = min(K, 64, HW)
+    hq, hk, hv = (torch.empty((Ke,) + st.shape, dtype=torch.bfloat16).pin_memory() for _ in range(3))
+    ho = torch.empty(st.shape, dtype=torch.bfloat16).pin_memory()
+    for i, g in enumerate(range(HW - Ke, HW)):
+        j = g % st.ring
+        hq[i].copy_(st.qkv[0][j]); hk[i].copy_(st.qkv[1][j]); hv[i].copy_(st.qkv[2][j])
+    regions = []
+    for _ in range(5):
+        st.load_late(max(0, HW - Ke - W))
+        for g in range(max(0, HW - Ke - W), HW - Ke):
+            st.decode(g)
+        torch.cuda.synchronize(st.dev)
         if world > 1:
             torch.distributed.barrier()
         tw = time.perf_counter()
         for i, g in enumerate(range(HW - Ke, HW)):
-            eng.token_step_host(T0 + g, C, hq[i], hk[i], hv[i], ho)      # synchronises: the result is on the host
-        e2e_ms_local = (time.perf_counter() - tw) * 1e3
-        e2e_ms, e2e_tokens = aggregate(e2e_ms_local, float(prompts * Ke), world)
-        per = int(np.prod(shape)) * 2
-        e2e = {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 3 * per,
-               "d2h_bytes_per_step": per, "steps": Ke, "ms_per_step": e2e_ms / Ke,
-               "api": "adsa_token_step_host (pinned host q/k/v in, host output out, copies in chunks of layers under the "
-                      "compute, one sync per token)"}
+            st.eng.token_step_host(T0 + g, C, hq[i], hk[i], hv[i], ho)      # synchronises: the result is on the host
+        regions.append((time.perf_counter() - tw) * 1e3)
+    ms, tokens = aggregate(float(np.median(regions)), float(prompts * Ke), world)
+    per = int(np.prod(st.shape)) * 2
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 3 * per, "d2h_bytes_per_step": per,
+            "steps": Ke, "ms_per_step": ms / Ke, "regions": len(regions),
+            "api": "adsa_token_step_host (pinned host q/k/v in, host output out, copies in chunks of layers under the "
+                   "compute, one sync per token)"}
 
+
+def compact(res):
+    """One configuration's figures for detail.all_configs."""
+    w, L = res["workload"], res["workload"].n_layers
+    d = res["detail"]
+    out = {"workload": w.name, "budget_fraction": w.beta, "capacity_rows": w.capacity(),
+           "image_tokens_per_s": res["tokens"] / (res["ms"] * 1e-3), "ms_per_token": res["ms"] / res["K"],
+           "us_per_layer_step": res["ms"] * 1e3 / (res["K"] * L), "cells_timed": [res["first"], res["first"] + res["K"]],
+           "regions": res["regions"], "gpu_launches": res["launches"],
+           "pool_ratio": res["kv_pool"]["ratio"], "pool_payload_ratio": res["kv_pool"]["payload_ratio"],
+           "pool_ratio_with_metadata": res["kv_pool"]["ratio_with_metadata"], "page_rows": res["kv_pool"]["page_rows"],
+           "clocks": res["clocks"]}
+    for key, r in (("fused", res.get("roofline")), ("fused_layer_launch", d.get("roofline_layer_launch")),
+                   ("attn_alone", d.get("roofline_attn"))):
+        if r:
+            out[key] = {"us_per_layer_step": r["us_per_layer_step"], "achieved_gbs": r["achieved"], "frac": r["frac"],
+                        "frac_of_nominal_8000": r["frac_of_nominal_8000"]}
+    return out
+
+
+def memory_vs_batch(args, dev):
+    """Fig. 8-style table on the XL shape: bytes of the KV pool (+ the library's metadata) against a dense
+    cache for batch 2 .. 64, with the XL decoder's bf16 weights beside them as context."""
+    from dataclasses import replace
+    rows = []
+    base = get_workload(4)
+    for batch in (2, 4, 8, 16, 32, 64):
+        w = replace(base, batch=batch, name=f"cfg4-batch{batch}")
+        st = Stack(w, args, dev, 0, 4)
+        st.load_late(st.HW - 3)
+        for g in range(st.HW - 3, st.HW):
+            st.decode(g)
+        assert st.eng.get_status()[0] == 0
+        rec = pool_record(st, st.eng.pool_bytes_peak())
+        rows.append({"batch": batch, "adsa_pool_bytes": rec["peak_bytes"], "metadata_bytes": rec["metadata_bytes"],
+                     "dense_kv_bytes": rec["dense_bytes"], "kv_ratio": rec["ratio"], "kv_ratio_with_metadata": rec["ratio_with_metadata"],
+                     "weights_bytes": LLAMAGEN_XL_PARAM_BYTES,
+                     "total_ratio_with_weights": (rec["peak_bytes"] + rec["metadata_bytes"] + LLAMAGEN_XL_PARAM_BYTES) /
+                                                 (rec["dense_bytes"] + LLAMAGEN_XL_PARAM_BYTES)})
+        del st
+        torch.cuda.empty_cache()
+    return rows
+
+
+def run_ours(args, rank, world, local_rank):
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = _workload(args)
+    W = max(3, args.warmup)
+    res = measure(w, args, dev, rank, world, local_rank, args.steps, W, detail=not args.no_detail)
+    st, K, L, C = res["stack"], res["K"], w.n_layers, w.capacity()
+    e2e = None if args.no_e2e else end_to_end(st, args, K, W, world, res["prompts"])
+    peak_pool_gb = res["kv_pool"]["peak_bytes"] / 1e9
+    ring = st.ring
+    res["stack"] = None
+    del st
+    torch.cuda.empty_cache()
     if rank != 0:
         return
-    # per call (cache full, median over cells, per layer) and per cell of the timed generation
-    detail = {"per_call_us_cache_full": {n: float(np.median(v)) for n, v in call_ms.items() if v}}
-    if detail["per_call_us_cache_full"]:
-        detail["per_call_us_cache_full"]["four_call_sequence"] = float(sum(detail["per_call_us_cache_full"].values()))
-    if len(cell_ev) >= 48 and K == HW and first == 0:
-        prev, per_cell = t0, {}
-        for gcell, e in cell_ev:
-            per_cell[gcell] = prev.elapsed_time(e) * 1e3 / L
-            prev = e
-        span = lambda a: float(np.median([per_cell[i] for i in range(a, a + 16)]))
-        detail["fused_layer_step_us_by_cell"] = {"start_cells_0_15": span(0), "middle": span(HW // 2 - 8),
-                                                  "end_last_16": span(HW - 16),
-                                                  "rows_at": {"start": T0 + 1, "middle": min(C, T0 + HW // 2), "end": min(C, T0 + HW)}}
-    # ---- rooflines, steady state (cache full, one eviction per step) ----------------------------
-    # The dominant kernel is the fused layer-step (one launch per layer-step: select, attend, the next
-    # step's scores, update).  Algorithmic bytes per stream: retained rows x (K + V) + 16 B of metadata per
-    # live row (position, carried score, inverse norm read; next score written) + q, k_new, v_new, out and
-    # the new row's K and V.  The attention kernel alone (adsa_sparse_decode_attn) is reported beside it.
-    peak, peak_kind = peaks()
-    d2 = w.head_dim * 2
-    retained = rows_full - 1 if rows_full == C else rows_full          # one eviction per step once full
-    step_bytes = w.streams_per_layer * (retained * 2 * d2 + rows_step * 16 + 6 * d2)
-    step_us = step_ms * 1e3 / max(1, step_launches)
-    step_gbs = step_bytes / (step_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": "fused layer-step (adsa_layer_step / adsa_token_step)", "achieved": step_gbs,
-                "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8000": step_gbs / 8000.0, "us_per_launch": step_us, "launches_timed": step_launches,
-                "algorithmic_bytes_per_launch": step_bytes, "traffic": STEP_DRAM_TRAFFIC_BYTES.get(args.workload)}
-    attn_bytes = w.streams_per_layer * (retained * 2 * d2 + 4 * d2)
-    attn_us = attn_ms * 1e3 / attn_launches
-    achieved = attn_bytes / (attn_us * 1e-6) / 1e9
-    roofline_attn = {"bound": "hbm", "kernel": "attention alone (adsa_sparse_decode_attn)", "achieved": achieved,
-                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "frac_of_nominal_8000": achieved / 8000.0, "us_per_launch": attn_us,
-                     "launches_timed": attn_launches, "algorithmic_bytes_per_launch": attn_bytes,
-                     "traffic": ATTN_DRAM_TRAFFIC_BYTES.get(args.workload)}
+    detail = res["detail"]
+    if not args.no_all_configs and world == 1:      # short runs of every configuration (one GPU only: ranks are not held for it)
+        import copy
+        rows = []
+        for name, beta in [("cfg1", None), ("cfg2", None), ("cfg3", None), ("cfg4", None), ("cfg5", 0.25), ("cfg5", 0.5), ("cfg5", 0.75)]:
+            w2 = _workload(args, name, beta)
+            if w2.name == w.name and w2.beta == w.beta and args.layers is None:
+                rows.append(compact(res))
+                continue
+            a2 = copy.copy(args)
+            a2.page_rows, a2.layers, a2.workload, a2.profiler_range = 0, None, name, False
+            r2 = measure(w2, a2, dev, 0, 1, local_rank, min(20, w2.n_cells), 5, detail=True)
+            r2["stack"] = None
+            rows.append(compact(r2))
+            del r2
+            torch.cuda.empty_cache()
+        detail["all_configs"] = rows
+    if not args.no_memory_sweep and world == 1:
+        detail["memory_vs_batch"] = memory_vs_batch(args, dev)
 
+    ms, tokens = res["ms"], res["tokens"]
     line = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "impl": "ours",
         "config": {"workload": w.name, "layers": L, "batch": w.batch, "heads": w.n_heads, "head_dim": w.head_dim,
-                   "n_text": T0, "grid": [w.grid_h, w.grid_w], "budget_fraction": w.beta, "capacity_rows": C,
-                   "page_rows": pr, "storage": "bf16 KV pool, fp32 arithmetic", "parallelism": "replicas only",
-                   "cells_timed": [first, first + K] if K <= HW else "whole generations",
-                   "l2": "inputs larger than L2: every step sweeps the whole KV pool "
-                         f"({peak_pool_bytes / 1e9:.2f} GB) against 126 MB of L2",
+                   "n_text": w.n_text, "grid": [w.grid_h, w.grid_w], "budget_fraction": w.beta, "capacity_rows": C,
+                   "page_rows": res["kv_pool"]["page_rows"], "storage": "bf16 KV pool, fp32 arithmetic",
+                   "parallelism": "replicas only",
+                   "cells_timed": [res["first"], res["first"] + K] if K <= w.n_cells else "whole generations",
+                   "timed_regions": f"median of {res['regions']} regions of {K} steps each (min {res['region_ms_min_max'][0]:.3f} ms, "
+                                    f"max {res['region_ms_min_max'][1]:.3f} ms), each after a reload of the cache state and {W} untimed steps",
+                   "launch": "one launch per token (all layers)" if res["launches"] == K else "one launch per layer",
+                   "l2": f"inputs larger than L2: every step sweeps the whole KV pool ({peak_pool_gb:.2f} GB) against 126 MB of L2",
                    "inputs": f"q/k/v ring of {ring} steps resident in HBM"},
         "us_per_layer_step": ms * 1e3 / (K * L),
-        "batch_rows_per_s": tokens / (ms * 1e-3) * (w.batch / prompts),
-        "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_attn": roofline_attn,
-        "detail": detail,
-        # peak_bytes counts whole pool rows (row_stride elements: d rounded up to a 16-byte multiple);
-        # payload_bytes the d elements of each row, which is what dense_bytes counts
-        "kv_pool": {"peak_bytes": peak_pool_bytes, "dense_bytes": w.dense_kv_bytes(),
-                    "ratio": peak_pool_bytes / w.dense_kv_bytes(),
-                    "payload_bytes": peak_pool_bytes * w.head_dim // eng.cfg.row_stride,
-                    "payload_ratio": peak_pool_bytes * w.head_dim / eng.cfg.row_stride / w.dense_kv_bytes(),
-                    "row_stride": eng.cfg.row_stride, "budget_fraction": w.beta},
+        "batch_rows_per_s": tokens / (ms * 1e-3) * (w.batch / res["prompts"]),
+        "gpu_launches": res["launches"], "clocks": res["clocks"],
     }
+    if "roofline" in res:
+        line["roofline"] = res["roofline"]
+    for key in ("roofline_layer_launch", "roofline_attn"):
+        if key in detail:
+            line[key] = detail.pop(key)
+    line["detail"] = detail
+    line["kv_pool"] = res["kv_pool"]
     if e2e:
         line["e2e"] = e2e
     if world == 1 and not args.no_cpu_baseline:
@@ -480,14 +713,35 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    args = parse_args()
+def run_selftest(args, rank, world):
+    """--impl selftest: no GPU work.  Every rank reports a made-up time and unit count through the same
+    aggregation and printing as the real arms, so that the multi-process plumbing can be checked on CPUs."""
+    ms, units = aggregate(10.0 + 5.0 * rank, 16.0 * (rank + 1), world)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": units / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "impl": "selftest",
+                          "ms": ms, "units": units}), flush=True)
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
+    args = parse_args(argv)
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl != "reference":
+        raise SystemExit(spawn_replicas(args.gpus, argv))      # N independent replicas, one process per GPU
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         if rank == 0:
             run_reference(args)
+        return
+    if args.impl == "selftest":
+        if world > 1:
+            torch.distributed.init_process_group(args.backend)
+        try:
+            run_selftest(args, rank, world)
+        finally:
+            if world > 1:
+                torch.distributed.destroy_process_group()
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")

@@ -554,13 +554,10 @@ int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows,
     return cuda_fail(ctx, e);
 }
 
-int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
-                    const void *v_new, void *out_bf16, adsa_stream_t stream)
+// One step of layers l0 .. l0 + NL - 1 (q, k_new, v_new, out_bf16 point at layer l0's tensors).
+static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                       const void *v_new, void *out_bf16, adsa_stream_t stream)
 {
-    if (!ctx || !q || !k_new || !v_new || !out_bf16) return ADSA_EINVAL;
-    if (ctx->cuda_error) return ADSA_ECUDA;
-    if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
-    const int NL = ctx->cfg.n_layers;
     size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k_new,
                         *vb = (const __nv_bfloat16 *)v_new;
@@ -573,9 +570,9 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
     // every layer is between steps and in the same carried state; otherwise layer by layer.
     bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok;
     if (one_launch) {
-        const LayerState &L0 = ctx->layers[0];
+        const LayerState &L0 = ctx->layers[l0];
         for (int l = 0; l < NL && one_launch; ++l) {
-            const LayerState &L = ctx->layers[l];
+            const LayerState &L = ctx->layers[l0 + l];
             one_launch = L.phase == kIdle && (L.scores_pos == cur_pos) == (L0.scores_pos == cur_pos) &&
                          (L.svec_pos == cur_pos) == (L0.svec_pos == cur_pos);
         }
@@ -588,7 +585,7 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
     }
     if (!one_launch) {
         for (int l = 0; l < NL; ++l) {
-            int rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
+            int rc = adsa_layer_step(ctx, l0 + l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
                                      vb + l * per_layer, ob + l * per_layer, stream);
             if (rc) return rc;
         }
@@ -600,17 +597,21 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
     std::vector<int> after(NL);
     {
         long long need = 0;
-        for (int l = 0; l < NL; ++l) {
+        for (int l = 0; l < ctx->cfg.n_layers; ++l) {
             const int hi = ctx->layers[l].rows_hi;
-            after[l] = hi + 1 < cap ? hi + 1 : cap;
-            if (after[l] > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
-            need += (long long)ctx->dev.S * pages_for(ctx, after[l] > hi ? after[l] : hi);
+            int rows = hi;
+            if (l >= l0 && l < l0 + NL) {
+                after[l - l0] = hi + 1 < cap ? hi + 1 : cap;
+                if (after[l - l0] > ctx->cfg.max_rows_per_stream) return ADSA_ENOMEM;
+                rows = after[l - l0] > hi ? after[l - l0] : hi;
+            }
+            need += (long long)ctx->dev.S * pages_for(ctx, rows);
         }
         if (need > ctx->cfg.n_pages) return ADSA_ENOMEM;
     }
     cudaStream_t st = (cudaStream_t)stream;
-    if (ctx->layers[0].scores_pos != cur_pos) {   // nothing carried in (first step, or the caches were rewritten)
-        for (int l = 0; l < NL; ++l) {
+    if (ctx->layers[l0].scores_pos != cur_pos) {   // nothing carried in (first step, or the caches were rewritten)
+        for (int l = l0; l < l0 + NL; ++l) {
             ++ctx->launches;
             ctx->layers[l].svec_pos = -1;
             note_launch(ctx, l, false, true, stream);
@@ -618,12 +619,12 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
             if (rc) return rc;
         }
     }
-    const bool have_svec = ctx->layers[0].svec_pos == cur_pos;
+    const bool have_svec = ctx->layers[l0].svec_pos == cur_pos;
     ++ctx->launches;
-    int rc = cuda_fail(ctx, launch_wstep(ctx->dev, wp, ctx->maps, true, 0, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
+    int rc = cuda_fail(ctx, launch_wstep(ctx->dev, wp, ctx->maps, true, l0, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
                                          st, have_svec && ctx->sweep_mode >= 1, false, ctx->sweep_mode >= 2, -1, ctx->next_tiles, NL));
     for (int l = 0; l < NL; ++l) {
-        LayerState &L = ctx->layers[l];
+        LayerState &L = ctx->layers[l0 + l];
         L.rows_hi = after[l];
         L.cur_pos = cur_pos;
         L.scores_pos = cur_pos + 1;
@@ -635,12 +636,22 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
     return rc;
 }
 
+int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                    const void *v_new, void *out_bf16, adsa_stream_t stream)
+{
+    if (!ctx || !q || !k_new || !v_new || !out_bf16) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
+    return step_layers(ctx, 0, ctx->cfg.n_layers, cur_pos, budget_rows, q, k_new, v_new, out_bf16, stream);
+}
+
 int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host, const void *k_new_host,
                          const void *v_new_host, void *out_host, adsa_stream_t stream)
 {
     if (!ctx) return ADSA_EINVAL;
     if (ctx->cuda_error) return ADSA_ECUDA;
     if (!q_host || !k_new_host || !v_new_host || !out_host) return ADSA_EINVAL;
+    if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     const int L = ctx->cfg.n_layers;
     // chunk boundaries: a first chunk of one layer, so that computing starts after a short copy, then up to five
@@ -691,9 +702,9 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
         const int l0 = bound[c], l1 = bound[c + 1];
         const size_t off = (size_t)l0 * per_layer, bytes = (size_t)(l1 - l0) * per_layer * sizeof(__nv_bfloat16);
         e = cudaStreamWaitEvent(st, ctx->ev_in[c], 0);
-        for (int l = l0; l < l1 && e == cudaSuccess && rc == ADSA_OK; ++l)
-            rc = adsa_layer_step(ctx, l, cur_pos, budget_rows, ctx->stage_q + l * per_layer, ctx->stage_k + l * per_layer,
-                                 ctx->stage_v + l * per_layer, ctx->stage_o + l * per_layer, stream);
+        if (e == cudaSuccess)   // the chunk's layers: one launch when the tensor-core kernel can take them together
+            rc = step_layers(ctx, l0, l1 - l0, cur_pos, budget_rows, ctx->stage_q + l0 * per_layer, ctx->stage_k + l0 * per_layer,
+                             ctx->stage_v + l0 * per_layer, ctx->stage_o + l0 * per_layer, stream);
         if (e != cudaSuccess || rc != ADSA_OK) break;
         e = cudaEventRecord(ctx->ev_done[c], st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[c], 0);

@@ -47,3 +47,17 @@ def test_single_rank_is_the_identity():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.aggregate(3.5, 7.0, 1) == (3.5, 7.0)
+
+
+def test_gpus_flag_spawns_replicas_that_aggregate():
+    """`python bench.py --gpus 2` without a launcher around it starts two ranks of itself; with the
+    made-up timings of --impl selftest over gloo, rank 0 prints the max time and the summed units."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "selftest", "--backend", "gloo"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms"] == 15.0 and lines[0]["units"] == 48.0
