@@ -31,7 +31,7 @@ struct LayerState {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, status, staging, total;
+    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, wscratch, status, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -49,6 +49,7 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.svec = off;        off = align_up(off + S * (size_t)cfg.n_layers * 256 * sizeof(float), 256);
     w.carry = off;       off = align_up(off + S * (size_t)cfg.n_layers * 4 * sizeof(int32_t), 256);
     w.cand_mask = off;   off = align_up(off + S * (size_t)cfg.n_layers * mask_words_of(cfg) * sizeof(uint32_t), 256);
+    w.wscratch = off;    off = align_up(off + (size_t)kScratchCtas * kScratchGroups * (2 * R + 4) * sizeof(unsigned long long), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
     w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
@@ -299,6 +300,7 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.svec = (float *)(w + ws.svec);
     d.carry = (int32_t *)(w + ws.carry);
     d.cand_mask = (uint32_t *)(w + ws.cand_mask);
+    d.wscratch = (unsigned long long *)(w + ws.wscratch);
     d.status = (uint32_t *)(w + ws.status);
     d.d = cfg->head_dim;
     d.row_stride = cfg->row_stride;

@@ -16,6 +16,8 @@ constexpr int kRegionLocal = 2;
 constexpr int kRegionInvalid = 3;
 
 constexpr int kMaxSplits = 32;         // attention chunks per stream
+constexpr int kScratchCtas = 160;      // CTAs of the tensor-core kernel that own a slice of rare-step scratch (its grid is capped here)
+constexpr int kScratchGroups = 8;      // ... and streams such a CTA serves at a time
 constexpr float kNormEps = 1e-8f;      // clamp of |v| (an all-zero row has similarity 0 with everything)
 constexpr int kRingSpinLimit = 1 << 16;
 
@@ -38,6 +40,7 @@ struct DevCtx {
                             //                      highest-scoring row of its previous region; -1 = not known), number of rows
                             //                      in that region, bit 0 = some cached V row has a clamped norm, spare
     uint32_t *cand_mask;    // [n_layers * S][mask_words]  bit s = slot s lies in the previous region of the next step
+    unsigned long long *wscratch;   // [kScratchCtas][kScratchGroups][2 * max_rows + 4]  rare-step scratch of the tensor-core kernel
     uint32_t *status;       // [1]
     int d, row_stride, page_rows, n_pages, max_rows, max_pages, mask_words, S;
     int partial_stride;     // floats per split partial: row_stride + 2 (m, l)

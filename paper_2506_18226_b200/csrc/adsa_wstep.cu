@@ -120,13 +120,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
+// part `role` (0 hi, 1 mid, 2 lo) of the three-way bf16 split of the pair (w0, w1): hi = bf16(w), mid = bf16(w - hi),
+// lo = bf16(w - hi - mid), 24 bits in all
+__device__ __forceinline__ uint32_t split_part(float w0, float w1, int role)
+{
+    const uint32_t h = pack_bf16(w0, w1);
+    const float r0 = w0 - bf16_lo(h), r1 = w1 - bf16_hi(h);
+    const uint32_t m = pack_bf16(r0, r1);
+    const uint32_t l = pack_bf16(r0 - bf16_lo(m), r1 - bf16_hi(m));
+    return role == 0 ? h : role == 1 ? m : l;
+}
 // byte offset of 16-byte chunk c of row r inside a tile written with the 128-byte swizzle
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * kWRowBytes + ((c ^ (r & 7)) << 4)); }
 
 // Shared memory of one group (the G warps that share a stream): a fixed part, then one ring per warp.
 struct WLayout {
-    uint32_t bars, hdr, pt, inv, keys, prevm, candm, kmask, cmask, wsplit, hist, part, rings;
-    uint32_t inv_words, w_rows, mwords;
+    uint32_t bars, hdr, pt, inv, prevm, candm, kmask, cmask, hist, part, rings;
+    uint32_t inv_words, mwords;
     uint32_t ring_bytes;    // one warp's ring
     uint32_t per_group;
 };
@@ -142,20 +152,12 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     L.pt = off;     off += w_align(max_pages * 4, 16);
     L.inv_words = w_align(max_rows + 8, 4);
     L.inv = off;    off += fused ? L.inv_words * 4 : 0;                   // inverse norms by slot
-    L.w_rows = w_align(max_rows + kWTile, 32);
-    // one region, three lives: selection keys; then the row weights (bf16 hi | mid | lo) during pass 1;
-    // then the compaction lists (holes, survivors)
-    {
-        uint32_t kb = w_align((max_rows + 2) * 8, 16), wb = 3 * L.w_rows * 2;
-        L.keys = off; L.wsplit = off;
-        off += fused ? (kb > wb ? kb : wb) : 0;
-    }
     L.mwords = mask_words + 1;
     L.prevm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows of the previous region
     L.candm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows in the previous region of the next step
     L.kmask = off;  off += w_align(L.mwords * 4, 16);                     // retained rows
     L.cmask = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // retained rows the next step scores
-    L.part = off;   off += kWMaxGroupWarps * kWPart * 4;                  // per warp: acc[64] | s[64] | m, l | flags
+    L.part = off;   off += (G * kWPart * 4 > 1024 ? G * kWPart * 4 : 1024);   // per warp: acc[64] | s[64] | m, l | flags (at least the histogram's 1 KB)
     L.hist = L.part;                                                      // radix histogram: used before any partial state exists
     off = w_align(off, 1024);                                             // the swizzle pattern repeats every 1024 bytes
     L.rings = off;
@@ -179,6 +181,7 @@ struct WStepArgs {
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out_bf16;
     float *out_f32;
+    unsigned long long *scratch; // [grid][n_groups][2 * max_rows + 4] words of 8 bytes: keys, compaction lists
 };
 
 struct WSelPartial {      // what one warp of a group found in its share of the rows (32 bytes)
@@ -204,12 +207,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     WSelPartial *sel_part = reinterpret_cast<WSelPartial *>(smem + L.hdr);
     unsigned long long *sel_thr = reinterpret_cast<unsigned long long *>(smem + L.hdr + kWMaxGroupWarps * 32);
     int32_t *pt_s = reinterpret_cast<int32_t *>(smem + L.pt);
-    unsigned long long *sm_keys = reinterpret_cast<unsigned long long *>(smem + L.keys);
+    // Selection keys (any K) and the compaction lists (several evictions at once) are needed on rare steps only:
+    // they live in global memory, a slice per group of every CTA (same-SM traffic, served by L1/L2), so that shared
+    // memory holds more streams.
+    unsigned long long *sm_keys = a.scratch + ((size_t)blockIdx.x * a.n_groups + gi) * (size_t)(2 * c.max_rows + 4);
     uint32_t *prevm = reinterpret_cast<uint32_t *>(smem + L.prevm);
     uint32_t *candm = reinterpret_cast<uint32_t *>(smem + L.candm);
     uint32_t *kmask = reinterpret_cast<uint32_t *>(smem + L.kmask);
     uint32_t *cmask = reinterpret_cast<uint32_t *>(smem + L.cmask);
-    __nv_bfloat16 *wsplit = reinterpret_cast<__nv_bfloat16 *>(smem + L.wsplit);
     int *hist = reinterpret_cast<int *>(smem + L.hist);
     float *part = reinterpret_cast<float *>(smem + L.part);
 
@@ -233,7 +238,6 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
     //   V^T (transposing loads), rows 16*a + 8*(mi>>1) + lr, chunk 2*b + (mi&1):   a*2048 + (vt_off ^ (b << 5))
     const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
-    const uint32_t *w_role = reinterpret_cast<const uint32_t *>(wsplit + (size_t)(g >= 2 && g <= 4 ? g - 2 : 0) * L.w_rows);
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     // the local window does not move between this step and the next, and the new row stays inside it: the next
     // step's previous region is this one's minus whatever is evicted
@@ -860,27 +864,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (!single) total = 2 * mt;
             rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;   // p' <= 1: every score is 0
             __syncwarp();
-            // w = 1/|v| for the retained rows the next step scores, as three bf16 parts (24 bits); they
-            // take the place of the keys, which nobody reads any more
+            // does one of the rows this warp will score have a clamped norm?  (their weights 1/|v| are split into
+            // bf16 parts tile by tile during the sweep)
             if (general) group_sync();
             {
-                uint32_t *ws = reinterpret_cast<uint32_t *>(wsplit);
                 float w_big = 0.f;   // the largest 1/|v| among the rows this warp will score
-                for (int i = 0; rk + i * G < n_tiles; i += 2) {   // two of the warp's blocks per trip, a pair of rows per lane
-                    const int b = rk + (i + (lane >> 4)) * G;
-                    if (b < n_tiles) {
-                        const int slot = b * 32 + 2 * (lane & 15);
-                        const uint32_t cm = cmask[b] >> (2 * (lane & 15));
-                        float w0 = 0.f, w1 = 0.f;
-                        if (cm & 1u) w0 = inv_s[slot];
-                        if (cm & 2u) w1 = inv_s[slot + 1];
-                        w_big = fmaxf(w_big, fmaxf(w0, w1));
-                        const uint32_t h = pack_bf16(w0, w1);
-                        const float r0 = w0 - bf16_lo(h), r1 = w1 - bf16_hi(h);
-                        const uint32_t md = pack_bf16(r0, r1);
-                        const uint32_t lo = pack_bf16(r0 - bf16_lo(md), r1 - bf16_hi(md));
-                        ws[slot >> 1] = h; ws[(L.w_rows + slot) >> 1] = md; ws[(2 * L.w_rows + slot) >> 1] = lo;
-                    }
+                for (int i = 0; rk + i * G < n_tiles; ++i) {
+                    const int b = rk + i * G;
+                    if ((cmask[b] >> lane) & 1u) w_big = fmaxf(w_big, inv_s[b * 32 + lane]);
                 }
                 warp_clamped = __any_sync(0xffffffffu, w_big >= 1.0f / kNormEps);
                 warp_rare = warp_clamped || n2 < n;
@@ -989,8 +980,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 uint32_t l2 = pack_bf16(p10 - bf16_lo(h2), p11 - bf16_hi(h2));
                 uint32_t w0 = 0u, w2 = 0u;
                 if (FUSED && !fast) {   // the short way carries s' on instead of summing it again: no row weights
-                    w0 = w_role[(r0 + 16 * ks + 2 * t) >> 1];
-                    w2 = w_role[(r0 + 16 * ks + 8 + 2 * t) >> 1];
+                    // w = 1/|v| of rows 2t, 2t + 1 (+ 8) of this k-step if the next step scores them, else 0; this
+                    // lane's part of the split (g = 2, 3, 4: hi, mid, lo)
+                    const int s0 = r0 + 16 * ks + 2 * t;
+                    const uint32_t cm = cmask[tl] >> (16 * ks + 2 * t);
+                    w0 = split_part((cm & 1u) ? inv_s[s0] : 0.f, (cm & 2u) ? inv_s[s0 + 1] : 0.f, g - 2);
+                    w2 = split_part((cm & 0x100u) ? inv_s[s0 + 8] : 0.f, (cm & 0x200u) ? inv_s[s0 + 9] : 0.f, g - 2);
                 }
                 pb0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
                 pb2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
@@ -1256,6 +1251,8 @@ cudaError_t configure_wstep_kernel(const DevCtx &c)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
     return e;
@@ -1270,7 +1267,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
     if (!wstep_supported(c)) return p;
     const int n_streams = c.S * (n_run < 1 ? 1 : n_run);   // streams one launch serves
     int groups = (n_streams + sm_count - 1) / sm_count;
-    groups = groups < 1 ? 1 : groups > 8 ? 8 : groups;
+    groups = groups < 1 ? 1 : groups > kScratchGroups ? kScratchGroups : groups;
     const int cap = max_depth > 0 && max_depth < kWMaxDepth ? max_depth : kWMaxDepth;
     if (n_run > 1 && group_warps <= 0) {
         // A launch over several layers has more streams than any grouping can hold at once, so what counts is how
@@ -1297,6 +1294,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
                 p.l2_ahead = fused ? 1 : 0;   // measured: with the ring this makes a three-deep pipeline; deeper is slower
                 p.smem_bytes = (size_t)L.per_group * groups;
                 p.grid = n_streams < sm_count ? n_streams : sm_count;   // spread the streams over every SM
+                if (p.grid > kScratchCtas) p.grid = kScratchCtas;
                 return p;
             }
             if (group_warps > 0) break;
@@ -1321,10 +1319,12 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     a.g_magic = (uint32_t)((1ull << 32) / (uint32_t)plan.group_warps) + 1u;   // exact for x < 2^16 at least (group_warps <= 4)
     a.q = (const __nv_bfloat16 *)q; a.k_new = (const __nv_bfloat16 *)k_new; a.v_new = (const __nv_bfloat16 *)v_new;
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
+    a.scratch = c.wscratch;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
     void (*kern)(DevCtx, WStepArgs, WStepMaps);
     if (warps <= 8) kern = fused ? wstep_kernel<true, 8> : wstep_kernel<false, 8>;
     else if (warps <= 10) kern = fused ? wstep_kernel<true, 10> : wstep_kernel<false, 10>;   // 5 streams x 2 warps, the LlamaGen-XL shape: room for 204 registers per thread
+    else if (warps <= 12) kern = fused ? wstep_kernel<true, 12> : wstep_kernel<false, 12>;   // 6 streams x 2 warps: 168 registers per thread
     else kern = fused ? wstep_kernel<true, 16> : wstep_kernel<false, 16>;
     // launched so that its set-up overlaps the tail of the kernel before it in the stream (the kernel
     // itself waits for that kernel's completion before it reads or writes global memory)
