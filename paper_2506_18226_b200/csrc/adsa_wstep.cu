@@ -69,13 +69,20 @@
 
 namespace adsa {
 
-constexpr int kWTile = 32;                        // rows per tile
-constexpr int kWRowBytes = 128;                   // 64 bf16
-constexpr int kWTileBytes = kWTile * kWRowBytes;  // one K (or V) tile
-constexpr int kWStageBytes = 2 * kWTileBytes;
+// The kernel is compiled for two row layouts (template parameters RS = elements per pool row, TR = rows per
+// ring stage):
+//   RS = 64,  TR = 32   128-byte rows written with the 128-byte swizzle; a stage is a whole 32-row block;
+//   RS = 104, TR = 16   208-byte rows (head_dim 97 .. 104) written as they lie: a pitch of 208 bytes puts the eight
+//                       rows of an ldmatrix on eight different bank groups without any swizzle; a stage is half a
+//                       block (6.5 KB instead of 13 KB), so that shared memory still holds rings for ten warps.
+// Rows are always dealt to the warps of a group in 32-row blocks (one word of every row mask).
+constexpr int kWTile = 32;                        // rows per block
 constexpr int kWMaxDepth = 8;                     // stages per warp
 constexpr int kWMaxGroupWarps = 4;                // warps that may share a stream
-constexpr int kWPart = 136;                       // floats of one warp's partial state: acc[64] | s[64] | m, l | flags
+constexpr int kWWideMaxWarps = 10;                // warps per CTA of the 104-element instantiation (registers)
+__host__ __device__ constexpr int w_stage_bytes(int rs, int tr) { return 2 * tr * rs * 2; }          // a K tile and a V tile
+__host__ __device__ constexpr int w_sets(int rs) { return (rs + 63) / 64; }                           // 64-element sets of a row (two elements per lane)
+__host__ __device__ constexpr int w_part_floats(int rs) { return 128 * w_sets(rs) + 8; }             // one warp's partial state: acc | s | m, l, flags
 
 // ---- PTX wrappers ---------------------------------------------------------
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
@@ -131,7 +138,7 @@ __device__ __forceinline__ uint32_t split_part(float w0, float w1, int role)
     return role == 0 ? h : role == 1 ? m : l;
 }
 // byte offset of 16-byte chunk c of row r inside a tile written with the 128-byte swizzle
-__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * kWRowBytes + ((c ^ (r & 7)) << 4)); }
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 // Shared memory of one group (the G warps that share a stream): a fixed part, then one ring per warp.
 struct WLayout {
@@ -143,12 +150,12 @@ struct WLayout {
 
 __host__ __device__ inline uint32_t w_align(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-__host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mask_words, int depth, int G, bool fused)
+__host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mask_words, int depth, int G, bool fused, int rs, int tr)
 {
     WLayout L;
     uint32_t off = 0;
     L.bars = off;   off += (kWMaxGroupWarps * kWMaxDepth + 2) * 8;       // tile barriers per warp, then the metadata barrier
-    L.hdr = off;    off += kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16 + kWMaxGroupWarps * 8;   // per-warp selection partials, the threshold, per-warp highest carried scores, per-warp look at the next launch's stream
+    L.hdr = off;    off += kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16 + kWMaxGroupWarps * 8 + 16;   // per-warp selection partials, the threshold, per-warp highest carried scores, per-warp look at the next launch's stream, 16 zero bytes
     L.pt = off;     off += w_align(max_pages * 4, 16);
     L.inv_words = w_align(max_rows + 8, 4);
     L.inv = off;    off += fused ? L.inv_words * 4 : 0;                   // inverse norms by slot
@@ -157,11 +164,11 @@ __host__ __device__ inline WLayout w_layout(int max_rows, int max_pages, int mas
     L.candm = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // rows in the previous region of the next step
     L.kmask = off;  off += w_align(L.mwords * 4, 16);                     // retained rows
     L.cmask = off;  off += fused ? w_align(L.mwords * 4, 16) : 0;         // retained rows the next step scores
-    L.part = off;   off += (G * kWPart * 4 > 1024 ? G * kWPart * 4 : 1024);   // per warp: acc[64] | s[64] | m, l | flags (at least the histogram's 1 KB)
+    L.part = off;   off += (G * w_part_floats(rs) * 4 > 1024 ? G * w_part_floats(rs) * 4 : 1024);   // per warp: acc | s | m, l, flags (at least the histogram's 1 KB)
     L.hist = L.part;                                                      // radix histogram: used before any partial state exists
     off = w_align(off, 1024);                                             // the swizzle pattern repeats every 1024 bytes
     L.rings = off;
-    L.ring_bytes = depth * kWStageBytes;
+    L.ring_bytes = depth * w_stage_bytes(rs, tr);
     L.per_group = off + G * L.ring_bytes;
     return L;
 }
@@ -189,16 +196,25 @@ struct WSelPartial {      // what one warp of a group found in its share of the 
     int max_slot, n_pre, n_loc, p, n_cand, n_cand_not_prev;
 };
 
-template <bool FUSED, int MAXW>
+template <bool FUSED, int MAXW, int RS, int TR>
 __global__ void __launch_bounds__(MAXW * 32, 1)
 wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 {
+    constexpr int kWRowBytes = RS * 2;                 // bytes of a pool row
+    constexpr int kWTileBytes = TR * kWRowBytes;       // one K (or V) tile of a stage
+    constexpr int kWStageBytes = 2 * kWTileBytes;
+    constexpr int KS = (RS + 15) / 16;                 // 16-element steps over a row: k-steps of S = K.q and of the score product, M blocks of O^T
+    constexpr int NJ = w_sets(RS);                     // a lane holds elements 64*j + 2*lane, + 1 of a row, j < NJ
+    constexpr int NH = kWTile / TR, MB = TR / 16;      // stages per 32-row block, 16-row MMA blocks per stage
+    constexpr bool SWZ = RS == 64;                     // tiles written with the 128-byte swizzle
+    constexpr bool RAGGED = RS % 16 != 0;              // the last 16-element step has only its first 8 elements
+    constexpr int kWPart = w_part_floats(RS);
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = a.group_warps, D = a.depth;
     auto div_g = [&](int x) { return G == 1 ? x : (int)__umulhi((uint32_t)x, a.g_magic); };   // x / G without a division
     const int gi = div_g(warp), rk = warp - gi * G;      // group in the CTA, rank in the group
-    const WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, D, G, FUSED);
+    const WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, D, G, FUSED, RS, TR);
     unsigned char *smem = smem_all + (size_t)gi * L.per_group;
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + L.bars) + rk * kWMaxDepth;
     const uint32_t bar_meta = smem_u32(reinterpret_cast<unsigned long long *>(smem + L.bars) + kWMaxGroupWarps * kWMaxDepth);
@@ -218,9 +234,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     int *hist = reinterpret_cast<int *>(smem + L.hist);
     float *part = reinterpret_cast<float *>(smem + L.part);
 
+    const uint32_t zero_u32 = smem_u32(smem + L.hdr + kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16 + kWMaxGroupWarps * 8);
     if (lane == 0) {
         for (int s = 0; s < D; ++s) mbar_init(smem_u32(bars + s), 1);
-        if (rk == 0) mbar_init(bar_meta, 1);
+        if (rk == 0) {
+            mbar_init(bar_meta, 1);
+            *reinterpret_cast<uint4 *>(smem + L.hdr + kWMaxGroupWarps * 32 + 32 + kWMaxGroupWarps * 16 + kWMaxGroupWarps * 8) = make_uint4(0u, 0u, 0u, 0u);
+        }
         mbar_init_fence();
     }
     // launch-wide constants (integer divisions among them) come before the dependency wait as well
@@ -232,12 +252,32 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     const int g = lane >> 2, t = lane & 3;          // MMA fragment coordinates
     const int mi = lane >> 3, lr = lane & 7;        // ldmatrix: matrix index, row within the matrix
     const bool new_cand = FUSED && region_of(c, a.cur_pos, a.cur_pos + 1) == kRegionPrevious;
-    // ldmatrix row addresses inside a tile.  Tile rows used by a lane are (multiple of 8) + lr, so the
-    // swizzle term is (chunk ^ lr) << 4 and every address is a per-lane base xor a small constant:
-    //   rows of K or V as the A operand, rows 16*a + 8*(mi&1) + lr, chunk 2*b + (mi>>1):   a*2048 + (v_off ^ (b << 5))
-    const uint32_t v_off = (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4));
-    //   V^T (transposing loads), rows 16*a + 8*(mi>>1) + lr, chunk 2*b + (mi&1):   a*2048 + (vt_off ^ (b << 5))
-    const uint32_t vt_off = (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4));
+    // ldmatrix addresses inside a K or V tile, for 16-row block `blk` of the tile and 16-element step `b` of the row:
+    //   rows as the A operand: matrix mi holds rows 16*blk + 8*(mi&1) + lr, 16-byte chunk 2*b + (mi>>1)
+    //   V^T (transposing loads): matrix mi holds rows 16*blk + 8*(mi>>1) + lr, chunk 2*b + (mi&1)
+    // Swizzled tiles: the rows a lane uses are (multiple of 8) + lr, so the swizzle term is (chunk ^ lr) << 4 and the
+    // address is a per-lane base xor (b << 5).  Plain tiles: base + 32*b.  When the row ends in the middle of the last
+    // step, the lanes whose chunk lies beyond it read 16 zero bytes instead.
+    const uint32_t v_off = SWZ ? (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4))
+                               : (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + ((mi >> 1) << 4));
+    const uint32_t vt_off = SWZ ? (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4))
+                                : (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + ((mi & 1) << 4));
+    auto a_addr = [&](uint32_t tile, int blk, int b) -> uint32_t {
+        if (RAGGED && b == KS - 1 && (mi >> 1)) return zero_u32;
+        return tile + blk * 16 * kWRowBytes + (SWZ ? (v_off ^ (uint32_t)(b << 5)) : v_off + (uint32_t)(b << 5));
+    };
+    auto t_addr = [&](uint32_t tile, int blk, int b) -> uint32_t {
+        if (RAGGED && b == KS - 1 && (mi & 1)) return zero_u32;
+        return tile + blk * 16 * kWRowBytes + (SWZ ? (vt_off ^ (uint32_t)(b << 5)) : vt_off + (uint32_t)(b << 5));
+    };
+    // byte offset of 16-byte chunk ch of row r inside a tile
+    auto chunk_off = [&](int r, int ch) -> uint32_t { return SWZ ? swz(r, ch) : (uint32_t)(r * kWRowBytes + (ch << 4)); };
+    // one L2 hint per 128-byte line of a pool row
+    auto hint_row = [&](const __nv_bfloat16 *row) {
+#pragma unroll
+        for (int o = 0; o < kWRowBytes; o += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + o));
+        if (kWRowBytes % 128 != 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + kWRowBytes - 16));
+    };
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     // the local window does not move between this step and the next, and the new row stays inside it: the next
     // step's previous region is this one's minus whatever is evicted
@@ -278,15 +318,15 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 // value costs a useless prefetch).
                 const int n0 = __ldcg(c.n_live + sid0);
                 const int32_t *pt0 = c.page_table + (size_t)sid0 * c.max_pages;
-                for (int u = 0; u < D + (FUSED ? a.l2_ahead : 0); ++u) {
+                for (int u = 0; u < (D + NH - 1) / NH + (FUSED ? a.l2_ahead : 0); ++u) {   // the blocks the ring will hold, and those asked ahead
                     const int row = (rk + u * G) * kWTile + lane;
                     if (row < n0 && row < c.max_rows) {
                         const uint32_t pg = __umulhi((uint32_t)row, c.pr_magic);
                         const int page = __ldcg(pt0 + pg);
                         if (page >= 0 && page < c.n_pages) {
                             const size_t off = ((size_t)page * c.page_rows + ((uint32_t)row - pg * (uint32_t)c.page_rows)) * (size_t)c.row_stride;
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
+                            hint_row(c.k_pool + off);
+                            hint_row(c.v_pool + off);
                         }
                     }
                 }
@@ -355,23 +395,32 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             nxt[0] = __ldcg(c.n_live + sid2);
             nxt[1] = __ldcg(c.page_table + (size_t)sid2 * c.max_pages);
         }
-        // the caller's inputs: q as the A operand (rows 0-7 = q, rows 8-15 = 0), four k-steps of 16 elements; for the
-        // first warp elements 2*lane, 2*lane + 1 of q and of the new row's K and V; attention alone: this lane's
+        // the caller's inputs: q as the B operand of S = K.q (the same in every column), KS k-steps of 16 elements; for
+        // the first warp elements 64*j + 2*lane, + 1 of q and of the new row's K and V; attention alone: this lane's
         // first keep-mask word.  Requested with the other prologue loads when the dependency wait is behind us.
-        uint32_t qa0[4] = {0u, 0u, 0u, 0u}, qa2[4] = {0u, 0u, 0u, 0u};
-        uint32_t qn = 0u, kn = 0u, vn = 0u, km0 = 0u;
+        uint32_t qa0[KS], qa2[KS];
+        uint32_t qn[NJ], kn[NJ], vn[NJ], km0 = 0u;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) { qa0[ks] = 0u; qa2[ks] = 0u; }
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) { qn[j] = 0u; kn[j] = 0u; vn[j] = 0u; }
         auto load_inputs = [&]() {
             const uint32_t *q2 = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d);   // c.d is even
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
+            for (int ks = 0; ks < KS; ++ks) {
                 int e0 = 16 * ks + 2 * t, e1 = e0 + 8;
                 qa0[ks] = e0 < c.d ? q2[e0 >> 1] : 0u;
                 qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
             }
-            if (rk == 0 && 2 * lane < c.d) {
-                qn = q2[lane];
-                kn = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[lane];
-                vn = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[lane];
+            if (rk == 0) {
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) {
+                    if (64 * j + 2 * lane < c.d) {
+                        qn[j] = q2[32 * j + lane];
+                        kn[j] = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[32 * j + lane];
+                        vn[j] = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[32 * j + lane];
+                    }
+                }
             }
             if constexpr (!FUSED) {
                 if (rk + lane * G < c.mask_words) km0 = c.keep_mask[(size_t)sid * c.mask_words + rk + lane * G];
@@ -396,14 +445,19 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 sc0[u] = in ? sc_g[slot] : 0.f;
             }
         }
-        float st0 = 0.f, st1 = 0.f;   // carried s[2*lane], s[2*lane + 1] of this step's previous region
+        float st0[NJ], st1[NJ];   // carried s[64*j + 2*lane], s[64*j + 2*lane + 1] of this step's previous region
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) { st0[j] = 0.f; st1[j] = 0.f; }
         // (the two halves of a stream's 256 floats take turns: a step reads one and writes the other)
         float *const svec_in = c.svec + (size_t)sid * 256 + (a.cur_pos & 1) * 128, *const svec_out = c.svec + (size_t)sid * 256 + ((a.cur_pos + 1) & 1) * 128;
-        if (FUSED && a.have_svec) { st0 = svec_in[2 * lane]; st1 = svec_in[2 * lane + 1]; }
+        if (FUSED && a.have_svec) {
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) { st0[j] = svec_in[64 * j + 2 * lane]; st1[j] = svec_in[64 * j + 2 * lane + 1]; }
+        }
         if (n < 0 || n > c.max_rows) { if (lane == 0 && rk == 0) set_status(c, ADSA_DEV_ROW_OVERFLOW); n = 0; }
         const int n_tiles = (n + kWTile - 1) / kWTile;
         const int mt = rk < n_tiles ? div_g(n_tiles - rk + G - 1) : 0;   // this warp's tiles: rk, rk + G, ...
-        int total = mt;   // pass 1 tiles; the fused kernel adds pass 2 tiles (V only) unless it can score during pass 1
+        int total = 0;    // stages to fetch: pass 1, and for the fused kernel pass 2 (V only) unless it can score during pass 1
         const float *inv_s = nullptr;
         if constexpr (FUSED) {
             // inverse norms into shared memory: aligned interior by bulk copy, ragged ends by plain loads
@@ -426,29 +480,45 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         __syncwarp();
 
         // ---- the warp's own copy pipeline ----------------------------------------------------------
-        // Tiles of this warp, in issue order: u = 0 .. mt-1 are pass 1 (K and V), u = mt .. 2mt-1 pass 2 (V).
-        int cur_pg = 0, cur_in = 0;   // page and row-in-page of the next tile to issue (lane 0's copy is the one used)
-        auto seek = [&](int tl) {
-            cur_pg = (int)__umulhi((uint32_t)(tl * kWTile), c.pr_magic);
-            cur_in = tl * kWTile - cur_pg * c.page_rows;
+        // Stages of this warp, in issue order: u = 0 .. ms-1 are pass 1 (K and V), u = ms .. 2ms-1 pass 2 (V only);
+        // stage v of a pass is part v % NH (TR rows) of the warp's block v / NH, i.e. of block rk + (v / NH) * G.
+        const int ms = mt * NH;
+        total = ms;
+        auto stage_row0 = [&](int u) {
+            const int v = u >= ms ? u - ms : u;
+            return (rk + (NH == 1 ? v : v >> 1) * G) * kWTile + (NH == 1 ? 0 : (v & 1) * TR);
         };
-        seek(rk);
-        auto issue = [&](int u) {   // all lanes (the copies themselves by lanes 0 and 1): this warp's u-th tile of the stream into the next free stage
+        auto issue = [&](int u) {   // all lanes (the copies themselves by lanes 0 and 1): this warp's u-th stage into the next free ring slot
             const int stage = i_stage;
-            const int pass = u >= mt ? 1 : 0, tl = rk + (pass ? u - mt : u) * G;
-            if (u == mt) seek(rk);
-            const int r0 = tl * kWTile, r1 = min(n, r0 + kWTile);
+            const int pass = u >= ms ? 1 : 0;
+            const int r0 = stage_row0(u), r1 = max(r0, min(n, r0 + TR));
             const uint32_t kdst = stages_u32 + stage * kWStageBytes, vdst = kdst + kWTileBytes;
             const uint32_t bar = smem_u32(bars + stage);
             if (lane == 0) mbar_expect_tx(bar, (uint32_t)(r1 - r0) * kWRowBytes * (pass == 0 ? 2u : 1u));
             __syncwarp();
-            if (r1 - r0 == kWTile && cur_in + kWTile <= c.page_rows) {
+            const int pg0 = (int)__umulhi((uint32_t)r0, c.pr_magic), in0 = r0 - pg0 * c.page_rows;
+            if constexpr (!SWZ) {
+                // Plain tiles are the pool's rows as they lie: every page piece is one untiled bulk copy per pool
+                // (a tensor copy wants its destination on a 128-byte boundary, which rows of 208 bytes do not keep).
+                if (lane == 1 || (lane == 0 && pass == 0)) {
+                    const __nv_bfloat16 *pool = lane ? c.v_pool : c.k_pool;
+                    const uint32_t dst = lane ? vdst : kdst;
+                    int r = r0, pg = pg0, in = in0;
+                    while (r < r1) {
+                        const int cnt = min(r1 - r, c.page_rows - in);
+                        bulk_g2s(dst + (uint32_t)(r - r0) * kWRowBytes, pool + ((size_t)pt_s[pg] * c.page_rows + in) * (size_t)RS,
+                                 (uint32_t)cnt * kWRowBytes, bar);
+                        r += cnt; in = 0; ++pg;
+                    }
+                }
+            } else if (r1 - r0 == TR && in0 + TR <= c.page_rows) {
                 // the common case: a whole tile inside one page is one box per pool; lane 0 copies K, lane 1 copies V
-                const int y = pt_s[cur_pg] * c.page_rows + cur_in;
+                constexpr int kBox = TR == 32 ? 5 : 4;
+                const int y = pt_s[pg0] * c.page_rows + in0;
                 if (lane == 1 || (lane == 0 && pass == 0))
-                    tma_2d(lane ? vdst : kdst, lane ? &maps.v[5] : &maps.k[5], 0, y, bar);
+                    tma_2d(lane ? vdst : kdst, lane ? &maps.v[kBox] : &maps.k[kBox], 0, y, bar);
             } else if (lane == 0) {
-                int r = r0, pg = cur_pg, in = cur_in;
+                int r = r0, pg = pg0, in = in0;
                 while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
                     int cnt = min(r1 - r, c.page_rows - in);
                     int y = pt_s[pg] * c.page_rows + in;
@@ -463,36 +533,36 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     }
                 }
             }
-            cur_in += G * kWTile;   // the warp's next tile is G tiles further on
-            while (cur_in >= c.page_rows) { cur_in -= c.page_rows; ++cur_pg; }
         };
         // Rows of a partial tile that the copy does not write must hold finite numbers (their weights
         // are zero, and 0 * NaN would not be): all lanes clear them before the tile is requested.
         auto clear_tail = [&](int u) {
-            const int tl = rk + (u >= mt ? u - mt : u) * G;
-            const int rows = min(n, (tl + 1) * kWTile) - tl * kWTile;
-            if (rows < kWTile) {
+            constexpr int kChunks = kWRowBytes / 16;
+            const int r0 = stage_row0(u);
+            const int rows = max(0, min(n - r0, TR));
+            if (rows < TR) {
                 uint4 *z = reinterpret_cast<uint4 *>(ring + i_stage * kWStageBytes);
-                for (int i = rows * 8 + lane; i < kWTile * 8; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
+                for (int i = rows * kChunks + lane; i < TR * kChunks; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
             }
         };
-        // HBM is otherwise idle until the attention sweep starts (the ring holds `depth` tiles and the
-        // selection comes first), so the rows of the tiles after those are asked into L2 now, and one
-        // tile further with every tile consumed: the sweep then finds them in L2.
-        auto l2_ask = [&](int u) {   // this warp's u-th tile of pass 1, a row per lane
+        // HBM is otherwise idle until the attention sweep starts (the ring holds `depth` stages and the
+        // selection comes first), so the rows of the blocks after those are asked into L2 now, and one
+        // block further with every block consumed: the sweep then finds them in L2.
+        auto l2_ask = [&](int u) {   // this warp's u-th block, a row per lane
             const int row = (rk + u * G) * kWTile + lane;
             if (u < mt && row < n) {
                 const size_t off = c.max_pages == 1 ? ((size_t)pt_s[0] * c.page_rows + row) * (size_t)c.row_stride
                                                     : row_offset(c, pt_s, row);
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(c.k_pool + off));
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(c.v_pool + off));
+                hint_row(c.k_pool + off);
+                hint_row(c.v_pool + off);
             }
         };
-        const int partial_tl = (n & (kWTile - 1)) ? n_tiles - 1 : -1;   // the tile with fewer than 32 rows, if any
-        const int partial_u = mt > 0 && rk + (mt - 1) * G == partial_tl ? mt - 1 : -1;   // it can only be the warp's last tile
+        // stages with fewer than TR rows: only in the stream's last block, from the part that holds row n on
+        const int partial_v = (n & (kWTile - 1)) && mt > 0 && rk + (mt - 1) * G == n_tiles - 1
+                                  ? (mt - 1) * NH + (n & (kWTile - 1)) / TR : 0x7fffffff;
         int next_issue = 0;
         for (; next_issue < total && next_issue < D; ++next_issue) {
-            if (next_issue == partial_u) {   // generic-proxy stores into a stage are fenced before the copy that follows them
+            if (next_issue >= partial_v) {   // generic-proxy stores into a stage are fenced before the copy that follows them
                 clear_tail(next_issue);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
@@ -502,16 +572,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         }
 
         if constexpr (FUSED) {
-            for (int u = D; u < D + a.l2_ahead; ++u) l2_ask(u);
+            for (int u = (D + NH - 1) / NH; u < (D + NH - 1) / NH + a.l2_ahead; ++u) l2_ask(u);
         }
         // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
         // (the reads are complete once their results have been used, which in-order issue guarantees
         // for this thread and __syncwarp for the others; a fence is needed only after the generic-proxy
         // stores of clear_tail)
         auto release_and_refill = [&]() {
-            if (FUSED && a.l2_ahead > 0) l2_ask(next_issue + a.l2_ahead);
+            if (FUSED && a.l2_ahead > 0 && (NH == 1 || (next_issue & 1) == 0)) l2_ask((NH == 1 ? next_issue : next_issue >> 1) + a.l2_ahead);
             if (next_issue < total) {
-                if (partial_u >= 0 && (next_issue == partial_u || next_issue == partial_u + mt)) {
+                if ((next_issue >= ms ? next_issue - ms : next_issue) >= partial_v) {
                     clear_tail(next_issue);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
@@ -531,25 +601,30 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             ready = more && mbar_try_wait(smem_u32(bars + ns), ns == 0 ? c_par ^ 1u : c_par);
         };
 
-        // s (lane-distributed: s[2*lane], s[2*lane + 1]) as the B operand of the score product: columns
+        // s (lane-distributed: s[64*j + 2*lane], + 1) as the B operand of the score product: columns
         // 0, 1, 2 = its bf16 hi, mid, lo parts
-        uint32_t sb0[4] = {0u, 0u, 0u, 0u}, sb1[4] = {0u, 0u, 0u, 0u};
-        auto make_sb = [&](float s0, float s1) {
-            // each lane splits its own two elements (hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid)),
-            // packed in pairs; the fragments are then gathered with shuffles
-            const uint32_t ph = pack_bf16(s0, s1);
-            const float r0 = s0 - bf16_lo(ph), r1 = s1 - bf16_hi(ph);
-            const uint32_t pm = pack_bf16(r0, r1);
-            const uint32_t pl = pack_bf16(r0 - bf16_lo(pm), r1 - bf16_hi(pm));
+        uint32_t sb0[KS], sb1[KS];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const int src = 8 * ks + t;   // elements 16*ks + 2t, + 1 live in lane 8*ks + t; + 8, + 9 four lanes on
-                const uint32_t ah = __shfl_sync(0xffffffffu, ph, src), am = __shfl_sync(0xffffffffu, pm, src),
-                               al = __shfl_sync(0xffffffffu, pl, src);
-                const uint32_t bh = __shfl_sync(0xffffffffu, ph, src + 4), bm = __shfl_sync(0xffffffffu, pm, src + 4),
-                               bl = __shfl_sync(0xffffffffu, pl, src + 4);
-                sb0[ks] = g == 0 ? ah : g == 1 ? am : g == 2 ? al : 0u;
-                sb1[ks] = g == 0 ? bh : g == 1 ? bm : g == 2 ? bl : 0u;
+        for (int ks = 0; ks < KS; ++ks) { sb0[ks] = 0u; sb1[ks] = 0u; }
+        auto make_sb = [&](const float (&s0)[NJ], const float (&s1)[NJ]) {
+            // each lane splits its own elements (hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid)),
+            // packed in pairs; the fragments are then gathered with shuffles
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const uint32_t ph = pack_bf16(s0[j], s1[j]);
+                const float r0 = s0[j] - bf16_lo(ph), r1 = s1[j] - bf16_hi(ph);
+                const uint32_t pm = pack_bf16(r0, r1);
+                const uint32_t pl = pack_bf16(r0 - bf16_lo(pm), r1 - bf16_hi(pm));
+#pragma unroll
+                for (int ks = 4 * j; ks < 4 * j + 4 && ks < KS; ++ks) {
+                    const int src = 8 * (ks & 3) + t;   // elements 16*ks + 2t, + 1 live in lane 8*(ks % 4) + t of set ks / 4; + 8, + 9 four lanes on
+                    const uint32_t ah = __shfl_sync(0xffffffffu, ph, src), am = __shfl_sync(0xffffffffu, pm, src),
+                                   al = __shfl_sync(0xffffffffu, pl, src);
+                    const uint32_t bh = __shfl_sync(0xffffffffu, ph, src + 4), bm = __shfl_sync(0xffffffffu, pm, src + 4),
+                                   bl = __shfl_sync(0xffffffffu, pl, src + 4);
+                    sb0[ks] = g == 0 ? ah : g == 1 ? am : g == 2 ? al : 0u;
+                    sb1[ks] = g == 0 ? bh : g == 1 ? bm : g == 2 ? bl : 0u;
+                }
             }
         };
         // Eq. 1-2 for the next step on one tile of V rows: dot_i = v_i . s by MMA,
@@ -558,28 +633,28 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         bool warp_rare = false, warp_clamped = false;   // warp_clamped: one of the rows this warp scores has a clamped norm
         float rden = 0.f;
         // (two halves, so that the products can be issued early and their results used later)
-        auto score_mma = [&](uint32_t vb, float (&dt)[2][4]) {
+        auto score_mma = [&](uint32_t vb, float (&dt)[MB][4]) {
 #pragma unroll
-            for (int mbk = 0; mbk < 2; ++mbk) {
+            for (int mbk = 0; mbk < MB; ++mbk) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
+                for (int ks = 0; ks < KS; ++ks) {
                     uint32_t af[4];
-                    ldsm_x4(vb + mbk * 2048 + (v_off ^ (uint32_t)(ks << 5)), af);
+                    ldsm_x4(a_addr(vb, mbk, ks), af);
                     if (ks == 0) mma_bf16_z(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                     else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                 }
             }
         };
-        auto score_write = [&](const float (&dt)[2][4], const unsigned char *vtile, int tl, uint32_t cw) {
+        // r0: the stream row of the tile's first row; cw: bit i = row r0 + i is to be scored
+        auto score_write = [&](const float (&dt)[MB][4], const unsigned char *vtile, int r0, uint32_t cw) {
             float *scores = c.scores + (size_t)sid * c.max_rows;
             int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
-            const int r0 = tl * kWTile;
             // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
-            float sval[4], invv[4], dotv[4];
-            bool want[4];
+            float sval[2 * MB], invv[2 * MB], dotv[2 * MB];
+            bool want[2 * MB];
             const uint32_t cwg = t == 0 ? cw >> g : 0u;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 2 * MB; ++i) {
                 const int mbk = i >> 1, hh = i & 1;
                 const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
                 const int row = r0 + 16 * mbk + 8 * hh + g;
@@ -592,19 +667,19 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // norm, or rows move down in the update; otherwise every row is written where it stands
             if (!warp_rare) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                for (int i = 0; i < 2 * MB; ++i)
                     if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
             } else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < 2 * MB; ++i) {
                     if (!want[i]) continue;
                     const int mbk = i >> 1, hh = i & 1, row = r0 + 16 * mbk + 8 * hh + g;
                     float s_out = sval[i];
                     if (invv[i] >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
                         float ss = 0.f;
-                        for (int ch = 0; ch < 8; ++ch) {
+                        for (int ch = 0; ch < RS / 8; ++ch) {
                             float f[8];
-                            unpack8(*reinterpret_cast<const uint4 *>(vtile + swz(row - r0, ch)), f);
+                            unpack8(*reinterpret_cast<const uint4 *>(vtile + chunk_off(row - r0, ch)), f);
                             for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
                         }
                         s_out = (invv[i] * dotv[i] - invv[i] * invv[i] * ss) * rden + 0.0f;
@@ -683,7 +758,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;
             warp_clamped = (note.z & 1) != 0;   // known for the stream as a whole
             warp_rare = warp_clamped;
-            const uint32_t ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
+            uint32_t ve[NJ];
+            {
+                const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot));
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
+            }
             const uint32_t *cm_g = c.cand_mask + (size_t)sid * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {   // one block per lane
                 const int valid = n - b * 32;
@@ -693,9 +773,14 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             wait(bar_meta, streams_done & 1);   // the inverse norms are in shared memory
             const float inv_e = inv_s[evict_slot];
-            const float sp0 = fmaf(-inv_e, bf16_lo(ve), st0), sp1 = fmaf(-inv_e, bf16_hi(ve), st1);
+            float sp0[NJ], sp1[NJ];
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) { sp0[j] = fmaf(-inv_e, bf16_lo(ve[j]), st0[j]); sp1[j] = fmaf(-inv_e, bf16_hi(ve[j]), st1[j]); }
             make_sb(sp0, sp1);
-            if (rk == 0) { svec_out[2 * lane] = sp0; svec_out[2 * lane + 1] = sp1; }   // s' is what the next step starts from
+            if (rk == 0) {   // s' is what the next step starts from
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) { svec_out[64 * j + 2 * lane] = sp0[j]; svec_out[64 * j + 2 * lane + 1] = sp1[j]; }
+            }
         } else if constexpr (FUSED) {
             const int32_t *pos_g = c.pos + (size_t)sid * c.max_rows;
             const float *sc_g = c.scores + (size_t)sid * c.max_rows;
@@ -775,12 +860,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             wait(bar_meta, streams_done & 1);   // the inverse norms are in shared memory
             const bool general = K > 0 && K < p - 1;
             single = a.have_svec && !general && n_evict <= 1 && n_cand_np == 0 && !new_cand;
-            uint32_t ve = 0u;      // single sweep: the evicted row's elements 2*lane, 2*lane + 1, requested as early as possible
+            uint32_t ve[NJ];       // single sweep: the evicted row's elements 64*j + 2*lane, + 1, requested as early as possible
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) ve[j] = 0u;
             float inv_e = 0.f;
             if (!general) {
                 if (K == p - 1 && p > 0) evict_slot = max_slot;
                 if (single && evict_slot >= 0) {
-                    ve = *reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot) + 2 * lane);
+                    const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot));
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
                     inv_e = inv_s[evict_slot];
                 }
                 const bool drop_prev = K == 0 && p > 0;
@@ -861,7 +950,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 }
             }
             p_next += new_cand ? 1 : 0;
-            if (!single) total = 2 * mt;
+            if (!single) total = 2 * ms;
             rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;   // p' <= 1: every score is 0
             __syncwarp();
             // does one of the rows this warp will score have a clamped norm?  (their weights 1/|v| are split into
@@ -877,7 +966,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 warp_rare = warp_clamped || n2 < n;
             }
             if (single)   // s' = s - u_e: the evicted row (if any) leaves the previous region
-                make_sb(fmaf(-inv_e, bf16_lo(ve), st0), fmaf(-inv_e, bf16_hi(ve), st1));
+            {
+                float sp0[NJ], sp1[NJ];
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) { sp0[j] = fmaf(-inv_e, bf16_lo(ve[j]), st0[j]); sp1[j] = fmaf(-inv_e, bf16_hi(ve[j]), st1[j]); }
+                make_sb(sp0, sp1);
+            }
         } else {
             if (!waited) { dep_wait(); load_inputs(); }
             const uint32_t *gm = c.keep_mask + (size_t)sid * c.mask_words;
@@ -893,13 +987,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // ---- the running state; the first warp starts from the new row: weight 1 for role 0, its 1/|v| for role 2 ----
         // o_run[md][0..3]: dimension 16*md + g (0, 1) and 16*md + g + 8 (2, 3), roles 2t (0, 2) and 2t + 1 (1, 3), where
         // role 0/1 = softmax.V through P_hi / P_lo and roles 2/3/4 = s through w_hi / w_mid / w_lo.
-        float m_run = -FLT_MAX, l_run = 0.f, o_run[4][4];
+        float m_run = -FLT_MAX, l_run = 0.f, o_run[KS][4];
 #pragma unroll
-        for (int md = 0; md < 4; ++md) { o_run[md][0] = o_run[md][1] = o_run[md][2] = o_run[md][3] = 0.f; }
+        for (int md = 0; md < KS; ++md) { o_run[md][0] = o_run[md][1] = o_run[md][2] = o_run[md][3] = 0.f; }
         float ss_new = 0.f, inv_row_new = 0.f;   // first warp: |v_new|^2 and 1 / max(|v_new|, eps)
         if (rk == 0) {
-            float s = fmaf(bf16_hi(qn), bf16_hi(kn), fmaf(bf16_lo(qn), bf16_lo(kn), 0.f));
-            float ss = fmaf(bf16_hi(vn), bf16_hi(vn), fmaf(bf16_lo(vn), bf16_lo(vn), 0.f));
+            float s = 0.f, ss = 0.f;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                s = fmaf(bf16_hi(qn[j]), bf16_hi(kn[j]), fmaf(bf16_lo(qn[j]), bf16_lo(kn[j]), s));
+                ss = fmaf(bf16_hi(vn[j]), bf16_hi(vn[j]), fmaf(bf16_lo(vn[j]), bf16_lo(vn[j]), ss));
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -912,42 +1010,45 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             l_run = g == 0 ? 1.f : 0.f;   // summed over the eight g lanes at the end
             const float wrole = t == 0 ? 1.f : t == 1 ? inv_new : 0.f;   // role 0 in lanes t = 0, role 2 in lanes t = 1
 #pragma unroll
-            for (int md = 0; md < 4; ++md) {
-                // elements 16*md + g and 16*md + g + 8 sit in lanes 8*md + g/2 and 8*md + g/2 + 4, half g & 1
-                const uint32_t w0 = __shfl_sync(0xffffffffu, vn, 8 * md + (g >> 1)), w1 = __shfl_sync(0xffffffffu, vn, 8 * md + (g >> 1) + 4);
+            for (int md = 0; md < KS; ++md) {
+                // elements 16*md + g and 16*md + g + 8 sit in set md / 4, lanes 8*(md % 4) + g/2 and + 4, half g & 1
+                const uint32_t w0 = __shfl_sync(0xffffffffu, vn[md >> 2], 8 * (md & 3) + (g >> 1)),
+                               w1 = __shfl_sync(0xffffffffu, vn[md >> 2], 8 * (md & 3) + (g >> 1) + 4);
                 o_run[md][0] = wrole * ((g & 1) ? bf16_hi(w0) : bf16_lo(w0));
                 o_run[md][2] = wrole * ((g & 1) ? bf16_hi(w1) : bf16_lo(w1));
             }
         }
 
-        // ---- pass 1 --------------------------------------------------------------------------------
+        // ---- pass 1: block by block, a block in NH stages of TR rows --------------------------------
         for (int tl = rk; tl < n_tiles; tl += G) {
+#pragma unroll
+          for (int part_i = 0; part_i < NH; ++part_i) {
             const int stage = c_stage;
             if (!ready) wait(smem_u32(bars + stage), c_par);
             const uint32_t kb = stages_u32 + stage * kWStageBytes, vb = kb + kWTileBytes;
-            const int r0 = tl * kWTile;
-            const uint32_t kw = kmask[tl] >> g;   // bits 0, 8, 16, 24: rows g, g + 8, g + 16, g + 24 are retained
+            const int r0 = tl * kWTile + part_i * TR;
+            const uint32_t kw = (kmask[tl] >> (part_i * TR)) >> g;   // bits 0, 8 (, 16, 24): rows g, g + 8 (, g + 16, g + 24) of the stage are retained
             // S = K.q: A = 16 rows of K, B = q in every column, so every lane of a group of four holds the
             // logits of rows 16*mb + g (c0 = c1) and 16*mb + g + 8 (c2 = c3)
-            float sc[2][4];
+            float sc[MB][4];
 #pragma unroll
-            for (int mb = 0; mb < 2; ++mb) {
+            for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
+                for (int ks = 0; ks < KS; ++ks) {
                     uint32_t kf[4];
-                    ldsm_x4(kb + mb * 2048 + (v_off ^ (uint32_t)(ks << 5)), kf);
+                    ldsm_x4(a_addr(kb, mb, ks), kf);
                     if (ks == 0) mma_bf16_z(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                     else mma_bf16(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                 }
             }
-            peek_next(tl + G < n_tiles || (FUSED && !single));
-            float dts[2][4];   // the score products of this tile, started before the softmax arithmetic
+            peek_next(part_i + 1 < NH || tl + G < n_tiles || (FUSED && !single));
+            float dts[MB][4];   // the score products of this tile, started before the softmax arithmetic
             if constexpr (FUSED) {
                 if (single) score_mma(vb, dts);
             }
-            float x[2][2], mx = -INFINITY;   // x[mb][h]: row 16*mb + 8*h + g
+            float x[MB][2], mx = -INFINITY;   // x[mb][h]: row 16*mb + 8*h + g
 #pragma unroll
-            for (int mb = 0; mb < 2; ++mb) {
+            for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     bool kept = (kw >> (16 * mb + 8 * h)) & 1u;
@@ -963,16 +1064,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             m_run = m_new;
             float psum = 0.f;
 #pragma unroll
-            for (int mb = 0; mb < 2; ++mb) {
+            for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) { x[mb][h] = ex2(x[mb][h] - m_new); psum += x[mb][h]; }
             }
             l_run = fmaf(l_run, corr, psum);
-            // B' fragments for the two 16-row k-steps of O^T = V^T.B': column g of B' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0.
+            // B' fragments for the 16-row k-steps of O^T = V^T.B': column g of B' is P_hi, P_lo, w_hi, w_mid, w_lo, 0, 0, 0.
             // The weights of rows 2t, 2t + 1 (+ 8) of a k-step sit in the lanes of groups g' = 2t and 2t + 1.
-            uint32_t pb0[2], pb2[2];
+            uint32_t pb0[MB], pb2[MB];
 #pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
+            for (int ks = 0; ks < MB; ++ks) {
                 const float p00 = __shfl_sync(0xffffffffu, x[ks][0], 8 * t), p01 = __shfl_sync(0xffffffffu, x[ks][0], 8 * t + 4);
                 const float p10 = __shfl_sync(0xffffffffu, x[ks][1], 8 * t), p11 = __shfl_sync(0xffffffffu, x[ks][1], 8 * t + 4);
                 uint32_t h0 = pack_bf16(p00, p01), h2 = pack_bf16(p10, p11);
@@ -983,7 +1084,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     // w = 1/|v| of rows 2t, 2t + 1 (+ 8) of this k-step if the next step scores them, else 0; this
                     // lane's part of the split (g = 2, 3, 4: hi, mid, lo)
                     const int s0 = r0 + 16 * ks + 2 * t;
-                    const uint32_t cm = cmask[tl] >> (16 * ks + 2 * t);
+                    const uint32_t cm = cmask[tl] >> (part_i * TR + 16 * ks + 2 * t);
                     w0 = split_part((cm & 1u) ? inv_s[s0] : 0.f, (cm & 2u) ? inv_s[s0 + 1] : 0.f, g - 2);
                     w2 = split_part((cm & 0x100u) ? inv_s[s0 + 8] : 0.f, (cm & 0x200u) ? inv_s[s0 + 9] : 0.f, g - 2);
                 }
@@ -991,29 +1092,32 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 pb2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
             }
             // O^T_tile = V^T.B' from zero (A = V^T through transposing ldmatrix), then folded into the running sums
-            float ot[4][4];
+            float ot[KS][4];
 #pragma unroll
-            for (int md = 0; md < 4; ++md) {
+            for (int md = 0; md < KS; ++md) {
                 uint32_t vf[4];
-                ldsm_x4_t(vb + (vt_off ^ (uint32_t)(md << 5)), vf);
+                ldsm_x4_t(t_addr(vb, 0, md), vf);
                 mma_bf16_z(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[0], pb2[0]);
             }
+            if constexpr (MB == 2) {
 #pragma unroll
-            for (int md = 0; md < 4; ++md) {
-                uint32_t vf[4];
-                ldsm_x4_t(vb + 2048 + (vt_off ^ (uint32_t)(md << 5)), vf);
-                mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[1], pb2[1]);
+                for (int md = 0; md < KS; ++md) {
+                    uint32_t vf[4];
+                    ldsm_x4_t(t_addr(vb, 1, md), vf);
+                    mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[MB - 1], pb2[MB - 1]);
+                }
             }
             if constexpr (FUSED) {
-                if (single) score_write(dts, ring + stage * kWStageBytes + kWTileBytes, tl, n2 <= c.max_rows ? cmask[tl] : 0u);
+                if (single) score_write(dts, ring + stage * kWStageBytes + kWTileBytes, r0, n2 <= c.max_rows ? cmask[tl] >> (part_i * TR) : 0u);
             }
             release_and_refill();
             const float corr_role = t == 0 ? corr : 1.0f;     // roles 0, 1 carry softmax weights; the weight sums are not rescaled
 #pragma unroll
-            for (int md = 0; md < 4; ++md) {
+            for (int md = 0; md < KS; ++md) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) o_run[md][i] = fmaf(o_run[md][i], corr_role, ot[md][i]);
             }
+          }
         }
 
         // ---- HBM has nothing more to do for this stream: the first tiles the next launch will ask for go into L2 now,
@@ -1047,50 +1151,58 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 4);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 8);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
+        constexpr int kAcc = 0, kSum = 64 * NJ, kML = 128 * NJ;   // offsets inside a warp's partial state
         {
             float *w = part + rk * kWPart;
 #pragma unroll
-            for (int md = 0; md < 4; ++md) {
+            for (int md = 0; md < KS; ++md) {
                 const float lo0 = __shfl_down_sync(0xffffffffu, o_run[md][0], 1), lo2 = __shfl_down_sync(0xffffffffu, o_run[md][2], 1);
                 const int x0 = 16 * md + g, x1 = x0 + 8;
-                if (t == 0) { w[x0] = o_run[md][0] + o_run[md][1]; w[x1] = o_run[md][2] + o_run[md][3]; }
-                if (t == 1) { w[64 + x0] = (o_run[md][0] + o_run[md][1]) + lo0; w[64 + x1] = (o_run[md][2] + o_run[md][3]) + lo2; }
+                if (t == 0) { w[kAcc + x0] = o_run[md][0] + o_run[md][1]; w[kAcc + x1] = o_run[md][2] + o_run[md][3]; }
+                if (t == 1) { w[kSum + x0] = (o_run[md][0] + o_run[md][1]) + lo0; w[kSum + x1] = (o_run[md][2] + o_run[md][3]) + lo2; }
             }
-            if (lane == 0) { w[128] = m_run; w[129] = l_run; reinterpret_cast<int *>(w)[130] = warp_clamped ? 1 : 0; }
+            if (lane == 0) { w[kML] = m_run; w[kML + 1] = l_run; reinterpret_cast<int *>(w)[kML + 2] = warp_clamped ? 1 : 0; }
         }
         group_sync();
-        float sv0, sv1;   // s[2*lane], s[2*lane + 1]
+        float sv0[NJ], sv1[NJ];   // s[64*j + 2*lane], s[64*j + 2*lane + 1]
         {
             float M = -FLT_MAX;
-            for (int w = 0; w < G; ++w) M = fmaxf(M, part[w * kWPart + 128]);
-            float Lb = 0.f, A0 = 0.f, A1 = 0.f;
-            sv0 = 0.f; sv1 = 0.f;
+            for (int w = 0; w < G; ++w) M = fmaxf(M, part[w * kWPart + kML]);
+            float Lb = 0.f, A0[NJ], A1[NJ];
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) { A0[j] = 0.f; A1[j] = 0.f; sv0[j] = 0.f; sv1[j] = 0.f; }
             for (int w = 0; w < G; ++w) {
                 const float *ws = part + w * kWPart;
-                float wgt = ex2(ws[128] - M);
-                Lb = fmaf(ws[129], wgt, Lb);
-                A0 = fmaf(ws[2 * lane], wgt, A0);
-                A1 = fmaf(ws[2 * lane + 1], wgt, A1);
-                sv0 += ws[64 + 2 * lane];
-                sv1 += ws[64 + 2 * lane + 1];
-            }
-            const int xx = 2 * lane;
-            if (rk == 0 && xx < c.d) {
-                const float rl = 1.0f / Lb;
-                float o0 = A0 * rl, o1 = A1 * rl;
-                if (a.out_f32) {
-                    a.out_f32[(size_t)local * c.d + xx] = o0;
-                    if (xx + 1 < c.d) a.out_f32[(size_t)local * c.d + xx + 1] = o1;
+                float wgt = ex2(ws[kML] - M);
+                Lb = fmaf(ws[kML + 1], wgt, Lb);
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) {
+                    A0[j] = fmaf(ws[kAcc + 64 * j + 2 * lane], wgt, A0[j]);
+                    A1[j] = fmaf(ws[kAcc + 64 * j + 2 * lane + 1], wgt, A1[j]);
+                    sv0[j] += ws[kSum + 64 * j + 2 * lane];
+                    sv1[j] += ws[kSum + 64 * j + 2 * lane + 1];
                 }
-                if (a.out_bf16)
-                    *reinterpret_cast<uint32_t *>(a.out_bf16 + (size_t)local * c.d + xx) = pack_bf16(o0, o1);
+            }
+            const float rl = 1.0f / Lb;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const int xx = 64 * j + 2 * lane;
+                if (rk == 0 && xx < c.d) {
+                    float o0 = A0[j] * rl, o1 = A1[j] * rl;
+                    if (a.out_f32) {
+                        a.out_f32[(size_t)local * c.d + xx] = o0;
+                        if (xx + 1 < c.d) a.out_f32[(size_t)local * c.d + xx + 1] = o1;
+                    }
+                    if (a.out_bf16)
+                        *reinterpret_cast<uint32_t *>(a.out_bf16 + (size_t)local * c.d + xx) = pack_bf16(o0, o1);
+                }
             }
         }
 
         if constexpr (FUSED) {
             if (rk == 0 && !fast) {   // carried to the next step together with the scores (the short way has written s' already)
-                svec_out[2 * lane] = sv0;
-                svec_out[2 * lane + 1] = sv1;
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) { svec_out[64 * j + 2 * lane] = sv0[j]; svec_out[64 * j + 2 * lane + 1] = sv1[j]; }
             }
             // ---- Section 4.2 bookkeeping: holes below the new length, survivors above it ----------
             int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;   // keys are dead now
@@ -1132,13 +1244,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 // ---- pass 2: the next step's scores from a second sweep over V, against the sum just completed ----
                 make_sb(sv0, sv1);
                 for (int tl = rk; tl < n_tiles; tl += G) {
-                    const int stage = c_stage;
-                    if (!ready) wait(smem_u32(bars + stage), c_par);
-                    peek_next(tl + G < n_tiles);
-                    float dt2[2][4];
-                    score_mma(stages_u32 + stage * kWStageBytes + kWTileBytes, dt2);
-                    score_write(dt2, ring + stage * kWStageBytes + kWTileBytes, tl, okay ? cmask[tl] : 0u);
-                    release_and_refill();
+#pragma unroll
+                    for (int part_i = 0; part_i < NH; ++part_i) {
+                        const int stage = c_stage;
+                        if (!ready) wait(smem_u32(bars + stage), c_par);
+                        peek_next(part_i + 1 < NH || tl + G < n_tiles);
+                        float dt2[MB][4];
+                        score_mma(stages_u32 + stage * kWStageBytes + kWTileBytes, dt2);
+                        score_write(dt2, ring + stage * kWStageBytes + kWTileBytes, tl * kWTile + part_i * TR,
+                                    okay ? cmask[tl] >> (part_i * TR) : 0u);
+                        release_and_refill();
+                    }
                 }
             }
             // every warp's copies of this stream have landed before rows move or pages are freed (after a single
@@ -1163,19 +1279,21 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             }
             if (rk == 0 && lane == 0) {
                 int clamped = 0;
-                for (int w = 0; w < G; ++w) clamped |= reinterpret_cast<const int *>(part + w * kWPart)[130];
+                for (int w = 0; w < G; ++w) clamped |= reinterpret_cast<const int *>(part + w * kWPart)[kML + 2];
                 // rows that moved were scored at their new slots, but the mask above is by old slot: no note then
                 *reinterpret_cast<int4 *>(c.carry + (size_t)sid * 4) = make_int4(okay && ns == 0 ? 1 : 0, p_next, clamped, 0);
             }
 
             // ---- the update itself, by the first warp ---------------------------------------------------
             if (okay && rk == 0) {
-                for (int i = 0; i < ns; ++i) {   // survivors move down: 8 + 8 pieces of 16 bytes
+                for (int i = 0; i < ns; ++i) {   // survivors move down: K and V rows in pieces of 16 bytes
+                    constexpr int kChunks = kWRowBytes / 16;
                     const int row = surv[i], dst = holes[i];
                     size_t so = row_offset(c, pt, row), go = row_offset(c, pt, dst);
-                    if (lane < 16) {
-                        __nv_bfloat16 *pool = lane < 8 ? c.k_pool : c.v_pool;
-                        reinterpret_cast<uint4 *>(pool + go)[lane & 7] = reinterpret_cast<const uint4 *>(pool + so)[lane & 7];
+                    if (lane < 2 * kChunks) {
+                        __nv_bfloat16 *pool = lane < kChunks ? c.k_pool : c.v_pool;
+                        const int ch = lane < kChunks ? lane : lane - kChunks;
+                        reinterpret_cast<uint4 *>(pool + go)[ch] = reinterpret_cast<const uint4 *>(pool + so)[ch];
                     }
                     if (lane == 0) {
                         c.pos[(size_t)sid * c.max_rows + dst] = c.pos[(size_t)sid * c.max_rows + row];
@@ -1183,7 +1301,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     }
                 }
                 if (new_cand) {   // the new row's own score for the next step
-                    float dot = fmaf(bf16_hi(vn), sv1, fmaf(bf16_lo(vn), sv0, 0.f));
+                    float dot = 0.f;
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) dot = fmaf(bf16_hi(vn[j]), sv1[j], fmaf(bf16_lo(vn[j]), sv0[j], dot));
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
                     if (lane == 0) scores[last_hole] = (inv_row_new * dot - inv_row_new * inv_row_new * ss_new) * rden + 0.0f;
@@ -1194,8 +1314,13 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         __syncwarp();
                     }
                     const size_t off = row_offset(c, pt_s, last_hole);
-                    *reinterpret_cast<uint32_t *>(c.k_pool + off + 2 * lane) = kn;
-                    *reinterpret_cast<uint32_t *>(c.v_pool + off + 2 * lane) = vn;
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) {
+                        if (64 * j + 2 * lane < RS) {
+                            *reinterpret_cast<uint32_t *>(c.k_pool + off + 64 * j + 2 * lane) = kn[j];
+                            *reinterpret_cast<uint32_t *>(c.v_pool + off + 64 * j + 2 * lane) = vn[j];
+                        }
+                    }
                 }
                 if (lane == 0) {
                     c.pos[(size_t)sid * c.max_rows + last_hole] = a.cur_pos;
@@ -1210,10 +1335,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 }
 
 // ---- host side ------------------------------------------------------------
-bool wstep_supported(const DevCtx &c) { return c.row_stride == 64 && c.d % 2 == 0; }
+// Row layouts the kernel is compiled for: 64-element rows (32-row stages) and 104-element rows (16-row stages).
+bool wstep_supported(const DevCtx &c) { return (c.row_stride == 64 || c.row_stride == 104) && c.d % 2 == 0; }
+static int wstep_stage_rows(const DevCtx &c) { return c.row_stride == 64 ? 32 : 16; }
 
-// Tensor maps of both pools for boxes of 1, 2, 4, .. 32 rows (128-byte swizzle).  The encoder is
-// cuTensorMapEncodeTiled, looked up at run time so that the library links cudart only.
+// Tensor maps of both pools for boxes of 1, 2, 4, .. 32 rows (128-byte swizzle for 128-byte rows, none
+// otherwise).  The encoder is cuTensorMapEncodeTiled, looked up at run time so that the library links cudart only.
 int build_wstep_maps(const DevCtx &c, WStepMaps *out)
 {
     void *fn = nullptr;
@@ -1227,16 +1354,17 @@ int build_wstep_maps(const DevCtx &c, WStepMaps *out)
                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
     encode_t encode = (encode_t)fn;
-    const cuuint64_t dims[2] = {64, (cuuint64_t)c.n_pages * (cuuint64_t)c.page_rows};
+    const cuuint64_t dims[2] = {(cuuint64_t)c.row_stride, (cuuint64_t)c.n_pages * (cuuint64_t)c.page_rows};
     if (dims[1] > (1ull << 31)) return -1;
-    const cuuint64_t strides[1] = {kWRowBytes};
+    const cuuint64_t strides[1] = {(cuuint64_t)c.row_stride * 2};
     const cuuint32_t estr[2] = {1, 1};
     for (int pool = 0; pool < 2; ++pool) {
         for (int hb = 0; hb < 6; ++hb) {
-            const cuuint32_t box[2] = {64, 1u << hb};
+            const cuuint32_t box[2] = {(cuuint32_t)c.row_stride, 1u << hb};
             CUtensorMap *m = pool == 0 ? &out->k[hb] : &out->v[hb];
             CUresult r = encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pool == 0 ? (void *)c.k_pool : (void *)c.v_pool,
-                                dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                c.row_stride == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return -1;
         }
@@ -1244,52 +1372,69 @@ int build_wstep_maps(const DevCtx &c, WStepMaps *out)
     return 0;
 }
 
+typedef void (*wstep_fn)(DevCtx, WStepArgs, WStepMaps);
+
+// the instantiation for a row layout, a CTA size and a flavour (nullptr: not compiled)
+static wstep_fn wstep_variant(int row_stride, int warps, bool fused)
+{
+    if (row_stride == 64) {
+        if (warps <= 8) return fused ? wstep_kernel<true, 8, 64, 32> : wstep_kernel<false, 8, 64, 32>;
+        if (warps <= 10) return fused ? wstep_kernel<true, 10, 64, 32> : wstep_kernel<false, 10, 64, 32>;   // 5 streams x 2 warps, the LlamaGen-XL shape
+        if (warps <= 12) return fused ? wstep_kernel<true, 12, 64, 32> : wstep_kernel<false, 12, 64, 32>;   // 6 streams x 2 warps: 168 registers per thread
+        return fused ? wstep_kernel<true, 16, 64, 32> : wstep_kernel<false, 16, 64, 32>;
+    }
+    if (row_stride == 104) {
+        if (warps <= 8) return fused ? wstep_kernel<true, 8, 104, 16> : wstep_kernel<false, 8, 104, 16>;
+        if (warps <= kWWideMaxWarps) return fused ? wstep_kernel<true, kWWideMaxWarps, 104, 16> : wstep_kernel<false, kWWideMaxWarps, 104, 16>;
+    }
+    return nullptr;
+}
+
 cudaError_t configure_wstep_kernel(const DevCtx &c)
 {
-    (void)c;
-    cudaError_t e = cudaFuncSetAttribute(wstep_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wstep_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+    cudaError_t e = cudaSuccess;
+    for (int warps : {8, 10, 12, 16})
+        for (int fused = 0; fused < 2 && e == cudaSuccess; ++fused) {
+            wstep_fn f = wstep_variant(c.row_stride, warps, fused != 0);
+            if (f) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
+        }
     return e;
 }
 
 // Groups per CTA, warps per group and ring depth per warp.  As many groups as the SM has streams to
 // serve (at most 8), then as many warps per group as shared memory and the 16 warps of a CTA allow
-// with a ring of at least two tiles each.  group_warps > 0 fixes the group size.
+// with a ring of at least two stages each.  group_warps > 0 fixes the group size.
 WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, int group_warps, int n_run)
 {
     WStepPlan p = {};
     if (!wstep_supported(c)) return p;
+    const int rs = c.row_stride, tr = wstep_stage_rows(c), stage_bytes = w_stage_bytes(rs, tr);
+    const int max_warps = rs == 64 ? 16 : kWWideMaxWarps;   // the wide-row kernel needs more registers per thread
     const int n_streams = c.S * (n_run < 1 ? 1 : n_run);   // streams one launch serves
     int groups = (n_streams + sm_count - 1) / sm_count;
     groups = groups < 1 ? 1 : groups > kScratchGroups ? kScratchGroups : groups;
     const int cap = max_depth > 0 && max_depth < kWMaxDepth ? max_depth : kWMaxDepth;
-    if (n_run > 1 && group_warps <= 0) {
-        // A launch over several layers has more streams than any grouping can hold at once, so what counts is how
-        // many streams an SM keeps in flight and how fast each moves.  Measured on the XL shape (us per layer-step):
-        // 5 streams x 2 warps 19.2, 8 x 1 20.8, 3 x 4 22.9.  So: two warps per stream, as many streams as shared
-        // memory allows with rings of two tiles; one warp per stream if even one pair does not fit.
+    if (n_streams > 5 * sm_count + sm_count / 2 && group_warps <= 0) {
+        // A launch with more streams than any grouping can hold at once (several layers, or a large batch): what
+        // counts is how many streams an SM keeps in flight and how fast each moves.  Measured on the XL shape (us
+        // per layer-step): 5 streams x 2 warps 19.2, 8 x 1 20.8, 3 x 4 22.9.  So: two warps per stream, as many
+        // streams as shared memory allows with rings of two stages; one warp per stream if even one pair does not fit.
         for (int G = 2; G >= 1 && group_warps <= 0; --G)
             for (int gr = groups; gr >= 1; --gr) {
-                if (gr * G > 16) continue;
-                const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused).per_group;
-                if ((long long)kWSmemLimit / gr - fixed >= 2ll * G * kWStageBytes) { groups = gr; group_warps = G; break; }
+                if (gr * G > max_warps) continue;
+                const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused, rs, tr).per_group;
+                if ((long long)kWSmemLimit / gr - fixed >= 2ll * G * stage_bytes) { groups = gr; group_warps = G; break; }
             }
     }
     for (; groups >= 1; --groups) {
         for (int G = group_warps > 0 ? group_warps : kWMaxGroupWarps; G >= 1; --G) {
-            if (G > kWMaxGroupWarps || groups * G > 16) { if (group_warps > 0) break; continue; }
-            const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused).per_group;
+            if (G > kWMaxGroupWarps || groups * G > max_warps) { if (group_warps > 0) break; continue; }
+            const uint32_t fixed = w_layout(c.max_rows, c.max_pages, c.mask_words, 0, G, fused, rs, tr).per_group;
             const long long room = (long long)kWSmemLimit / groups - fixed;
-            int depth = room > 0 ? (int)(room / ((long long)G * kWStageBytes)) : 0;
+            int depth = room > 0 ? (int)(room / ((long long)G * stage_bytes)) : 0;
             depth = depth > cap ? cap : depth;
             if (depth >= 2 || (depth >= 1 && G == 1 && groups == 1)) {
-                WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, G, fused);
+                WLayout L = w_layout(c.max_rows, c.max_pages, c.mask_words, depth, G, fused, rs, tr);
                 p.n_groups = groups; p.group_warps = G; p.depth = depth;
                 p.l2_ahead = fused ? 1 : 0;   // measured: with the ring this makes a three-deep pipeline; deeper is slower
                 p.smem_bytes = (size_t)L.per_group * groups;
@@ -1321,11 +1466,8 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
     a.scratch = c.wscratch;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
-    void (*kern)(DevCtx, WStepArgs, WStepMaps);
-    if (warps <= 8) kern = fused ? wstep_kernel<true, 8> : wstep_kernel<false, 8>;
-    else if (warps <= 10) kern = fused ? wstep_kernel<true, 10> : wstep_kernel<false, 10>;   // 5 streams x 2 warps, the LlamaGen-XL shape: room for 204 registers per thread
-    else if (warps <= 12) kern = fused ? wstep_kernel<true, 12> : wstep_kernel<false, 12>;   // 6 streams x 2 warps: 168 registers per thread
-    else kern = fused ? wstep_kernel<true, 16> : wstep_kernel<false, 16>;
+    wstep_fn kern = wstep_variant(c.row_stride, warps, fused);
+    if (!kern) return cudaErrorInvalidConfiguration;
     // launched so that its set-up overlaps the tail of the kernel before it in the stream (the kernel
     // itself waits for that kernel's completion before it reads or writes global memory)
     cudaLaunchAttribute attr[1];
