@@ -97,7 +97,9 @@ typedef struct {
     int32_t n_text, grid_h, grid_w;   /* position -> grid cell mapping */
     int32_t n_prefix;                 /* rows with pos < n_prefix are always kept (Section 4.1 "prefix") */
     int32_t local_rows_back;          /* R: the local window holds the current grid row and R rows above it */
-    int32_t score_mode;               /* 0 = mean V-cosine similarity, keep the lowest (Eq. 1-3) */
+    int32_t score_mode;               /* 0 = mean V-cosine similarity, keep the lowest (Eq. 1-3): the paper's rule.
+                                         1 = attention mass, keep the highest: the attention-score pruning that
+                                         Section 3.4 argues against, as a comparison (see below) */
     float softmax_scale;              /* 0 => 1/sqrt(head_dim) */
 } adsa_config;
 
@@ -154,7 +156,15 @@ ADSA_API int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const 
  * different layers may be interleaved in any way: score and select for every
  * layer, then every layer's attention, then every update, is a valid sequence. */
 
-/* Eq. 1-2.  For every row i of the previous region of every stream of `layer`:
+/* score_mode 1 (comparison method, Section 3.4): every cached row carries the attention mass it has received,
+ * the sum of its softmax weights over the steps in which it was attended (its insertion step included; rows
+ * loaded by adsa_prefill_rows / adsa_set_stream_rows start at 0).  adsa_score then computes nothing and only
+ * reports the masses; adsa_select keeps the K previous rows with the HIGHEST mass (equal masses: lower position
+ * first); adsa_kv_update adds this step's weights to the retained rows' masses, so it must follow
+ * adsa_sparse_decode_attn (ADSA_ESTATE otherwise).  The mode runs on the four stand-alone kernels
+ * (adsa_layer_step and adsa_token_step launch them one after the other).
+ *
+ * Eq. 1-2.  For every row i of the previous region of every stream of `layer`:
  * S_i = (1/(p-1)) sum_{j != i} cos(v_i, v_j), j over the same region (p rows);
  * p <= 1 gives 0.  Computed through the identity sum_j cos = u_i.(sum_j u_j) - u_i.u_i
  * with u = v * inv_norm.  Scores stay in the workspace for adsa_select.

@@ -22,6 +22,9 @@
  * budget covers the context, brute-force grid-neighbour enumeration,
  * closed forms and hand cases for Eq. 1-2, exhaustive subset search for Eq. 3,
  * set invariants of the update, and the cache sizes printed in Tables 1-2.
+ * The attention-mass variant (the comparison method of Section 3.4) is pinned
+ * by its own tests: masses add up to the number of steps, subset search for
+ * the K highest, a dominant key survives, K = p - 1 evicts the least attended.
  * Image-quality figures (FID, IS, CLIP) are parity unpinned: they need
  * datasets and trained weights.
  */
@@ -257,6 +260,125 @@ int adsa_oracle_layer_step(const adsa_oracle_params *prm, int d, int cap_rows,
 done:
     free(region); free(keep); free(cv); free(gk); free(gv);
     return rc;
+}
+
+/* -------------------------------------------------------------------------
+ * The comparison method of Section 3.4: pruning by attention score, which the
+ * paper argues against for image generation (high scores cluster near the
+ * current token, so global context is lost).  It is NOT the paper's method;
+ * it exists so that the two selection rules can be run side by side on the
+ * same cache machinery.  Reading taken here (the paper only names the idea):
+ * every cached row carries the attention mass it has received so far, i.e. the
+ * sum of its softmax weights over the steps in which it was attended (its own
+ * insertion step included); among the "previous" rows the K with the HIGHEST
+ * mass are kept, equal masses ordered by position, lower position first.
+ * Partition, K, attention and update are those of the step above.
+ * ------------------------------------------------------------------------- */
+static int cand_more(const void *a, const void *b)
+{
+    const cand_t *x = (const cand_t *)a, *y = (const cand_t *)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return (x->pos > y->pos) - (x->pos < y->pos);
+}
+
+void adsa_oracle_select_highest(const float *score, const int *pos, int p, int K, int *keep)
+{
+    cand_t *c = (cand_t *)malloc((size_t)(p > 0 ? p : 1) * sizeof(cand_t));
+    for (int i = 0; i < p; ++i) { c[i].score = score[i]; c[i].pos = pos[i]; c[i].idx = i; keep[i] = 0; }
+    qsort(c, (size_t)p, sizeof(cand_t), cand_more);
+    for (int r = 0; r < p && r < K; ++r) keep[c[r].idx] = 1;
+    free(c);
+}
+
+/* One layer-step of one stream under attention-mass pruning.  mass[i] belongs
+ * to cached row i and is updated in place: after the step a retained row's
+ * mass has grown by its softmax weight of this step, the new row's mass is its
+ * own weight.  Masses are kept as float32 (rounded once per step from a double
+ * sum).  cand_score reports the masses the selection saw. */
+int adsa_oracle_layer_step_mass(const adsa_oracle_params *prm, int d, int cap_rows,
+                                int *n_live, int *pos, float *k, float *v, float *mass,
+                                const float *q, const float *k_new, const float *v_new, int cur_pos, int budget,
+                                double *out, int *n_kept, int *kept_pos, int *n_evict, int *evict_pos,
+                                int *n_cand, int *cand_pos, float *cand_score)
+{
+    int n = *n_live;
+    int *region = (int *)malloc((size_t)(n + 1) * sizeof(int));
+    int *keep = (int *)malloc((size_t)(n + 1) * sizeof(int));
+    float *gk = (float *)malloc((size_t)(n + 1) * d * sizeof(float));
+    float *gv = (float *)malloc((size_t)(n + 1) * d * sizeof(float));
+    float *gm = (float *)malloc((size_t)(n + 1) * sizeof(float));
+    double *w = (double *)malloc((size_t)(n + 1) * sizeof(double));
+    int rc = 0, n_pre = 0, n_loc = 0, p = 0;
+    for (int i = 0; i < n; ++i) {
+        region[i] = adsa_oracle_region(pos[i], cur_pos, prm->n_text, prm->grid_w, prm->n_prefix, prm->rows_back);
+        if (region[i] == ADSA_REGION_INVALID) { rc = -1; goto done; }
+        if (region[i] == ADSA_REGION_PREFIX) ++n_pre;
+        else if (region[i] == ADSA_REGION_LOCAL) ++n_loc;
+        else { cand_pos[p] = pos[i]; cand_score[p] = mass[i]; ++p; }
+    }
+    *n_cand = p;
+    {
+        int K = budget - n_pre - n_loc - 1;
+        if (K < 0) K = 0;
+        if (K > p) K = p;
+        adsa_oracle_select_highest(cand_score, cand_pos, p, K, keep);
+    }
+    {
+        int m = 0, e = 0, c = 0;
+        for (int i = 0; i < n; ++i) {
+            int kept = 1;
+            if (region[i] == ADSA_REGION_PREVIOUS) kept = keep[c++];
+            if (kept) {
+                kept_pos[m] = pos[i];
+                gm[m] = mass[i];
+                memcpy(gk + (size_t)m * d, k + (size_t)i * d, (size_t)d * sizeof(float));
+                memcpy(gv + (size_t)m * d, v + (size_t)i * d, (size_t)d * sizeof(float));
+                ++m;
+            } else {
+                evict_pos[e++] = pos[i];
+            }
+        }
+        *n_kept = m; *n_evict = e;
+        if (m + 1 > cap_rows) { rc = -1; goto done; }
+        memcpy(gk + (size_t)m * d, k_new, (size_t)d * sizeof(float));
+        memcpy(gv + (size_t)m * d, v_new, (size_t)d * sizeof(float));
+        double scale = prm->softmax_scale != 0.0 ? prm->softmax_scale : 1.0 / sqrt((double)d);
+        adsa_oracle_attend(q, gk, gv, m + 1, d, scale, out, w);
+        memcpy(k, gk, (size_t)(m + 1) * d * sizeof(float));
+        memcpy(v, gv, (size_t)(m + 1) * d * sizeof(float));
+        memcpy(pos, kept_pos, (size_t)m * sizeof(int));
+        pos[m] = cur_pos;
+        for (int j = 0; j < m; ++j) mass[j] = (float)((double)gm[j] + w[j]);
+        mass[m] = (float)w[m];
+        *n_live = m + 1;
+    }
+done:
+    free(region); free(keep); free(gk); free(gv); free(gm); free(w);
+    return rc;
+}
+
+int adsa_oracle_layer_step_mass_batch(const adsa_oracle_params *prm, int n_streams, int d, int cap_rows,
+                                      int *n_live, int *pos, float *k, float *v, float *mass,
+                                      const float *q, const float *k_new, const float *v_new, int cur_pos, int budget,
+                                      double *out, int *n_kept, int *kept_pos, int *n_evict, int *evict_pos,
+                                      int *n_cand, int *cand_pos, float *cand_score, int n_threads)
+{
+    int failed = 0;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : failed)
+#endif
+    for (int s = 0; s < n_streams; ++s) {
+        size_t r = (size_t)s * cap_rows;
+        int rc = adsa_oracle_layer_step_mass(prm, d, cap_rows, n_live + s, pos + r, k + r * d, v + r * d, mass + r,
+                                             q + (size_t)s * d, k_new + (size_t)s * d, v_new + (size_t)s * d,
+                                             cur_pos, budget, out + (size_t)s * d,
+                                             n_kept + s, kept_pos + r, n_evict + s, evict_pos + r,
+                                             n_cand + s, cand_pos + r, cand_score + r);
+        if (rc != 0) ++failed;
+    }
+    return failed;
 }
 
 /* The same step for many independent streams.  Arrays carry a leading stream

@@ -45,6 +45,7 @@ def lib():
         _lib.adsa_oracle_region.restype = C.c_int
         _lib.adsa_oracle_layer_step.restype = C.c_int
         _lib.adsa_oracle_layer_step_batch.restype = C.c_int
+        _lib.adsa_oracle_layer_step_mass_batch.restype = C.c_int
         _lib.adsa_oracle_max_threads.restype = C.c_int
     return _lib
 
@@ -89,6 +90,15 @@ def select_lowest(score, pos, K) -> np.ndarray:
     return keep
 
 
+def select_highest(score, pos, K) -> np.ndarray:
+    """The K highest scores, equal scores by lower position first (attention-mass pruning, Section 3.4's foil)."""
+    score = _f32(score)
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    keep = np.zeros(score.shape[0], dtype=np.int32)
+    lib().adsa_oracle_select_highest(_p(score, C.c_float), _p(pos, C.c_int), score.shape[0], int(K), _p(keep, C.c_int))
+    return keep
+
+
 def attend(q, k, v, scale=None):
     """softmax(q.k^T * scale) . v over the given rows.  Returns (out[d], weights[n]) in float64."""
     q, k, v = _f32(q), _f32(k), _f32(v)
@@ -114,8 +124,12 @@ class OracleStreams:
     """Cache state of `n_streams` independent streams plus the step function over them."""
 
     def __init__(self, n_streams, head_dim, cap_rows, n_text, grid_w, n_prefix, rows_back=1,
-                 softmax_scale=0.0, score_variant=0):
+                 softmax_scale=0.0, score_variant=0, score_mode=0):
+        """score_mode 0: the paper's rule (Eq. 1-3 on V); 1: attention-mass pruning (Section 3.4's foil), with
+        a per-row mass carried beside the rows (zero for rows loaded from outside)."""
         self.n_streams, self.d, self.cap = n_streams, head_dim, cap_rows
+        self.score_mode = score_mode
+        self.mass = np.zeros((n_streams, cap_rows), dtype=np.float32)
         self.prm = _Params(n_text, grid_w, n_prefix, rows_back, score_variant, softmax_scale)
         self.n_live = np.zeros(n_streams, dtype=np.int32)
         self.pos = np.zeros((n_streams, cap_rows), dtype=np.int32)
@@ -130,6 +144,7 @@ class OracleStreams:
         self.pos[stream, :n] = pos
         self.k[stream, :n] = k
         self.v[stream, :n] = v
+        self.mass[stream, :n] = 0.0
 
     def append_rows(self, k, v, first_pos):
         """Append rows [streams, n, d] at consecutive positions to every stream (the text condition)."""
@@ -140,6 +155,7 @@ class OracleStreams:
             self.pos[s, a:a + n] = np.arange(first_pos, first_pos + n)
             self.k[s, a:a + n] = k[s]
             self.v[s, a:a + n] = v[s]
+            self.mass[s, a:a + n] = 0.0
             self.n_live[s] = a + n
 
     def rows(self, stream):
@@ -158,12 +174,20 @@ class OracleStreams:
         evict_pos = np.zeros((S, cap), dtype=np.int32)
         cand_pos = np.zeros((S, cap), dtype=np.int32)
         cand_score = np.zeros((S, cap), dtype=np.float32)
-        failed = lib().adsa_oracle_layer_step_batch(
-            C.byref(self.prm), S, d, cap, _p(self.n_live, C.c_int), _p(self.pos, C.c_int),
-            _p(self.k, C.c_float), _p(self.v, C.c_float), _p(q, C.c_float), _p(k_new, C.c_float),
-            _p(v_new, C.c_float), int(cur_pos), int(budget), _p(out, C.c_double),
-            _p(n_kept, C.c_int), _p(kept_pos, C.c_int), _p(n_evict, C.c_int), _p(evict_pos, C.c_int),
-            _p(n_cand, C.c_int), _p(cand_pos, C.c_int), _p(cand_score, C.c_float), int(n_threads))
+        if self.score_mode == 1:
+            failed = lib().adsa_oracle_layer_step_mass_batch(
+                C.byref(self.prm), S, d, cap, _p(self.n_live, C.c_int), _p(self.pos, C.c_int),
+                _p(self.k, C.c_float), _p(self.v, C.c_float), _p(self.mass, C.c_float), _p(q, C.c_float),
+                _p(k_new, C.c_float), _p(v_new, C.c_float), int(cur_pos), int(budget), _p(out, C.c_double),
+                _p(n_kept, C.c_int), _p(kept_pos, C.c_int), _p(n_evict, C.c_int), _p(evict_pos, C.c_int),
+                _p(n_cand, C.c_int), _p(cand_pos, C.c_int), _p(cand_score, C.c_float), int(n_threads))
+        else:
+            failed = lib().adsa_oracle_layer_step_batch(
+                C.byref(self.prm), S, d, cap, _p(self.n_live, C.c_int), _p(self.pos, C.c_int),
+                _p(self.k, C.c_float), _p(self.v, C.c_float), _p(q, C.c_float), _p(k_new, C.c_float),
+                _p(v_new, C.c_float), int(cur_pos), int(budget), _p(out, C.c_double),
+                _p(n_kept, C.c_int), _p(kept_pos, C.c_int), _p(n_evict, C.c_int), _p(evict_pos, C.c_int),
+                _p(n_cand, C.c_int), _p(cand_pos, C.c_int), _p(cand_score, C.c_float), int(n_threads))
         if failed:
             raise RuntimeError(f"oracle: {failed} stream(s) rejected the step (bad position or overflow)")
         return StepResult(

@@ -31,7 +31,7 @@ struct LayerState {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, wscratch, status, staging, total;
+    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, wscratch, logit, ml, status, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -50,6 +50,8 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.carry = off;       off = align_up(off + S * (size_t)cfg.n_layers * 4 * sizeof(int32_t), 256);
     w.cand_mask = off;   off = align_up(off + S * (size_t)cfg.n_layers * mask_words_of(cfg) * sizeof(uint32_t), 256);
     w.wscratch = off;    off = align_up(off + (size_t)kScratchCtas * kScratchGroups * (2 * R + 4) * sizeof(unsigned long long), 256);
+    w.logit = off;       off = align_up(off + (cfg.score_mode == 1 ? S * (size_t)cfg.n_layers * R * sizeof(float) : 0), 256);
+    w.ml = off;          off = align_up(off + (cfg.score_mode == 1 ? S * (size_t)cfg.n_layers * 4 * sizeof(float) : 0), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
     w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
@@ -67,7 +69,7 @@ int check_config(const adsa_config *c)
     if (c->max_rows_per_stream < 1 || c->max_rows_per_stream > 16384) return ADSA_EINVAL;
     if (c->n_text < 0 || c->grid_h < 1 || c->grid_w < 1) return ADSA_EINVAL;
     if (c->n_prefix < 0 || c->local_rows_back < 0) return ADSA_EINVAL;
-    if (c->score_mode != 0) return ADSA_EINVAL;
+    if (c->score_mode != 0 && c->score_mode != 1) return ADSA_EINVAL;
     if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return ADSA_EINVAL;
     if ((long long)c->n_layers * c->batch * c->n_heads > (1ll << 24)) return ADSA_EINVAL;
     if ((long long)c->n_pages * c->page_rows * c->row_stride > (1ll << 40)) return ADSA_EINVAL;
@@ -191,6 +193,7 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     StagedChoice ch = {};
     const int m = ctx->kernel_mode;
     if (m == 0) return ch;
+    if (ctx->cfg.score_mode != 0) return ch;   // attention-mass pruning (the comparison method) runs on the four stand-alone kernels
     if ((m == 1 || m == 4) && ctx->mma_ok) {
         ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages, ctx->stream_warps);
         if (ctx->l2_ahead >= 0) ch.wp.l2_ahead = ctx->l2_ahead;
@@ -301,6 +304,9 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.carry = (int32_t *)(w + ws.carry);
     d.cand_mask = (uint32_t *)(w + ws.cand_mask);
     d.wscratch = (unsigned long long *)(w + ws.wscratch);
+    d.logit = (float *)(w + ws.logit);
+    d.ml = (float *)(w + ws.ml);
+    d.score_mode = cfg->score_mode;
     d.status = (uint32_t *)(w + ws.status);
     d.d = cfg->head_dim;
     d.row_stride = cfg->row_stride;
@@ -416,6 +422,12 @@ int adsa_score(adsa_ctx *ctx, int layer, int cur_pos, float *scores_out, adsa_st
     if (L.phase != kIdle) return ADSA_ESTATE;
     L.phase = kScored;
     L.cur_pos = cur_pos;
+    if (ctx->cfg.score_mode == 1) {   // the masses are carried with the rows: nothing to compute
+        if (!scores_out) return ADSA_OK;
+        note_launch(ctx, layer, false, false, stream);
+        ++ctx->launches;
+        return cuda_fail(ctx, launch_scores_copy(ctx->dev, layer, cur_pos, scores_out, (cudaStream_t)stream));
+    }
     if (L.scores_pos == cur_pos) {   // carried in from the previous fused step: nothing to compute
         if (!scores_out) return ADSA_OK;
         note_launch(ctx, layer, false, false, stream);
@@ -480,6 +492,7 @@ int adsa_kv_update(adsa_ctx *ctx, int layer, int cur_pos, const void *k_new, con
     if (!k_new || !v_new) return ADSA_EINVAL;
     LayerState &L = ctx->layers[layer];
     if ((L.phase != kSelected && L.phase != kAttended) || L.cur_pos != cur_pos) return ADSA_ESTATE;
+    if (ctx->cfg.score_mode == 1 && L.phase != kAttended) return ADSA_ESTATE;   // the masses grow by this step's attention weights
     int mand = mandatory_rows_bound(ctx, cur_pos) + 1;
     int cap = L.budget > mand ? L.budget : mand;
     L.rows_hi = L.rows_hi + 1 < cap ? L.rows_hi + 1 : cap;
@@ -570,7 +583,8 @@ static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_ro
     // The warps of a multiprocessor then sit in different phases of different streams (locating rows,
     // sweeping, updating) instead of all starting and all draining together once per layer.  Taken when
     // every layer is between steps and in the same carried state; otherwise layer by layer.
-    bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok;
+    bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok &&
+                      ctx->cfg.score_mode == 0;
     if (one_launch) {
         const LayerState &L0 = ctx->layers[l0];
         for (int l = 0; l < NL && one_launch; ++l) {

@@ -79,6 +79,7 @@ attn_kernel(DevCtx c, int layer, int chunk_rows, int n_splits, const __nv_bfloat
             m = s; l = 1.f;
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = vf[e];
+            if (c.score_mode == 1 && sub == 0) c.ml[(size_t)sid * 4 + 2] = s;
         }
     }
 
@@ -109,6 +110,8 @@ attn_kernel(DevCtx c, int layer, int chunk_rows, int n_splits, const __nv_bfloat
             for (int o = 1; o < LPR; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
             s[u] = ok[u] ? t : -INFINITY;
             m_new = fmaxf(m_new, s[u]);
+            // attention-mass mode: the row's logit is kept for the update, which turns it into this step's weight
+            if (c.score_mode == 1 && ok[u] && sub == 0) c.logit[(size_t)sid * c.max_rows + it0 + u * STEP + grp] = t;
         }
         float corr = exp2f(m - m_new);
         l *= corr;
@@ -156,6 +159,7 @@ attn_kernel(DevCtx c, int layer, int chunk_rows, int n_splits, const __nv_bfloat
         }
     }
     if (n_splits == 1) {
+        if (c.score_mode == 1 && x == 0) { c.ml[(size_t)sid * 4] = M; c.ml[(size_t)sid * 4 + 1] = L; }
         if (x < c.d) {
             float o = A / L;
             if (out_f32) out_f32[(size_t)local * c.d + x] = o;
@@ -188,6 +192,7 @@ attn_kernel(DevCtx c, int layer, int chunk_rows, int n_splits, const __nv_bfloat
             Lx = fmaf(__ldcg(ps + c.row_stride + 1), wgt, Lx);
             Ax = fmaf(__ldcg(ps + x), wgt, Ax);
         }
+        if (c.score_mode == 1 && x == 0) { c.ml[(size_t)sid * 4] = Mx; c.ml[(size_t)sid * 4 + 1] = Lx; }
         float o = Ax / Lx;
         if (out_f32) out_f32[(size_t)local * c.d + x] = o;
         if (out_bf16) out_bf16[(size_t)local * c.d + x] = __float2bfloat16_rn(o);

@@ -40,12 +40,15 @@ struct DevCtx {
                             //                      highest-scoring row of its previous region; -1 = not known), number of rows
                             //                      in that region, bit 0 = some cached V row has a clamped norm, spare
     uint32_t *cand_mask;    // [n_layers * S][mask_words]  bit s = slot s lies in the previous region of the next step
+    float *logit;           // [n_layers * S][max_rows]  score_mode 1: this step's logits (log2 units) by slot, from attention to the update
+    float *ml;              // [n_layers * S][4]         score_mode 1: softmax maximum, denominator, the new row's logit
     unsigned long long *wscratch;   // [kScratchCtas][kScratchGroups][2 * max_rows + 4]  rare-step scratch of the tensor-core kernel
     uint32_t *status;       // [1]
     int d, row_stride, page_rows, n_pages, max_rows, max_pages, mask_words, S;
     int partial_stride;     // floats per split partial: row_stride + 2 (m, l)
     uint32_t pr_magic;      // slot / page_rows == __umulhi(slot, pr_magic)
     int n_text, grid_w, n_prefix, rows_back;
+    int score_mode;         // 0: Eq. 1-3 (mean V-cosine similarity, keep the lowest); 1: attention mass, keep the highest
     float scale_log2e;      // softmax scale * log2(e)
 };
 
@@ -171,6 +174,7 @@ __device__ inline void write_row(const DevCtx &c, const int32_t *pt, int sid, in
     if (lane == 0) {
         c.pos[(size_t)sid * c.max_rows + slot] = pos;
         c.inv_norm[(size_t)sid * c.max_rows + slot] = 1.0f / fmaxf(sqrtf(ss), kNormEps);
+        if (c.score_mode == 1) c.scores[(size_t)sid * c.max_rows + slot] = 0.f;   // a row from outside has received no attention yet
     }
 }
 

@@ -123,6 +123,18 @@ kv_update_kernel(DevCtx c, int layer, int cur_pos, const __nv_bfloat16 *k_new, c
         if (threadIdx.x == 0) set_status(c, ADSA_DEV_BAD_EVICT);
         return;
     }
+    // attention-mass mode: every retained row's mass grows by the softmax weight it had in this step's attention
+    // (logits, maximum and denominator were left by the attention kernel), before rows move
+    float *mass = c.scores + (size_t)sid * c.max_rows;
+    float w_new = 0.f;
+    if (c.score_mode == 1) {
+        const float *lg = c.logit + (size_t)sid * c.max_rows;
+        const float M = c.ml[(size_t)sid * 4], Ld = c.ml[(size_t)sid * 4 + 1];
+        w_new = exp2f(c.ml[(size_t)sid * 4 + 2] - M) / Ld;
+        for (int s = threadIdx.x; s < n; s += kUpdateThreads)
+            if ((mask[s >> 5] >> (s & 31)) & 1u) mass[s] += exp2f(lg[s] - M) / Ld;
+        __syncthreads();
+    }
     // survivors move down: a row is row_stride bf16 = row_stride/8 16-byte pieces, for K and for V
     int pieces = c.row_stride >> 3;
     for (int i = warp; i < ns; i += kUpdateThreads / 32) {
@@ -136,9 +148,13 @@ kv_update_kernel(DevCtx c, int layer, int cur_pos, const __nv_bfloat16 *k_new, c
             size_t m = (size_t)sid * c.max_rows;
             c.pos[m + holes[i]] = c.pos[m + surv[i]];
             c.inv_norm[m + holes[i]] = c.inv_norm[m + surv[i]];
+            if (c.score_mode == 1) mass[holes[i]] = mass[surv[i]];
         }
     }
-    if (warp == 0) write_row(c, pt, sid, holes[ns], k_new + (size_t)local * c.d, v_new + (size_t)local * c.d, cur_pos);
+    if (warp == 0) {
+        write_row(c, pt, sid, holes[ns], k_new + (size_t)local * c.d, v_new + (size_t)local * c.d, cur_pos);
+        if (c.score_mode == 1 && lane == 0) mass[holes[ns]] = w_new;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         if (need < have) resize_pages(c, pt, have, need);

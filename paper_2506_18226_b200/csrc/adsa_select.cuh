@@ -72,7 +72,10 @@ __device__ inline SelResult block_select(const DevCtx &c, const int32_t *__restr
             region[slot] = rb;
             unsigned long long key = ~0ull;
             if (reg == kRegionPrevious) {
-                key = ((unsigned long long)orderable(scores[slot]) << 32) | (uint32_t)ps;
+                // the K lowest keys are kept: the score itself (Eq. 3), or its complement when the highest are wanted
+                // (attention mass); the position breaks ties either way, lower first
+                const uint32_t hi = c.score_mode == 1 ? ~orderable(scores[slot]) : orderable(scores[slot]);
+                key = ((unsigned long long)hi << 32) | (uint32_t)ps;
                 my_max = key > my_max ? key : my_max;
             }
             sm_keys[slot] = key;

@@ -23,6 +23,9 @@ TIE_BAND = 1e-6          # selection may differ only on scores this close to the
 OUT_MAX_ABS = 2e-2       # bf16 output vs oracle
 OUT_MEAN_ABS = 2e-3
 OUT_F32_MAX_ABS = 1e-4   # fp32 output: only summation order and exp2 vs exp differ (scaled by max|out|, >= 1)
+# attention-mass mode (score_mode 1): the score is a running fp32 sum of softmax weights, one rounding of the sum and
+# one of the weight (exp2, division: a few 1e-7) per step attended, so the bands are per accumulated quantity
+MASS_ATOL = 2e-5
 
 
 def dev_bf16(bits: np.ndarray, device="cuda:0") -> torch.Tensor:
@@ -55,8 +58,11 @@ class LayerHarness:
         self.S, self.d = eng.S, cfg.head_dim
         # sample: the streams (indices within the layer) the oracle follows; None = all
         self.sample = list(range(self.S)) if sample is None else list(sample)
+        self.mass_mode = cfg.score_mode == 1
+        self.score_atol = MASS_ATOL if self.mass_mode else SCORE_ATOL
+        self.tie_band = MASS_ATOL if self.mass_mode else TIE_BAND
         self.orc = orc.OracleStreams(len(self.sample), self.d, oracle_cap, cfg.n_text, cfg.grid_w, cfg.n_prefix,
-                                     cfg.local_rows_back, float(cfg.softmax_scale), score_variant)
+                                     cfg.local_rows_back, float(cfg.softmax_scale), score_variant, score_mode=cfg.score_mode)
         dev = eng.device
         R = cfg.max_rows_per_stream
         self.scores = torch.zeros((self.S, R), dtype=torch.float32, device=dev)
@@ -87,6 +93,7 @@ class LayerHarness:
 
     def _resync(self, i, s):
         pos, k, v = self.orc.rows(i)
+        self.orc.load(i, pos, k, v)          # (attention-mass mode: a reloaded stream starts from zero mass on both sides)
         from adsa_workloads import f32_to_bf16_bits
         b, h = divmod(s, self.eng.cfg.n_heads)
         dev = self.eng.device
@@ -151,7 +158,7 @@ class LayerHarness:
                 g = np.array([scores[s, slot_of[int(pp)]] for pp in res.cand_pos[i]], dtype=np.float64)
                 err = float(np.max(np.abs(g - res.cand_score[i].astype(np.float64))))
                 st.max_score_err = max(st.max_score_err, err)
-                assert err <= SCORE_ATOL, f"score mismatch {err} at pos {cur_pos} stream {s}"
+                assert err <= self.score_atol, f"score mismatch {err} at pos {cur_pos} stream {s}"
             # Eq. 3 + always-kept regions: retained / evicted position sets
             o_keep, o_ev = set(res.kept_pos[i].tolist()), set(res.evict_pos[i].tolist())
             assert len(g_keep) == n_keep and len(g_ev) == n_ev
@@ -159,9 +166,10 @@ class LayerHarness:
             if g_keep != o_keep:
                 assert len(g_keep) == len(o_keep), f"retained set sizes differ at pos {cur_pos} stream {s}"
                 sc = dict(zip(res.cand_pos[i].tolist(), res.cand_score[i].tolist()))
-                theta = max([sc[pp] for pp in o_keep if pp in sc] or [float('-inf')])
+                kept_sc = [sc[pp] for pp in o_keep if pp in sc]
+                theta = (min(kept_sc) if self.mass_mode else max(kept_sc)) if kept_sc else float('-inf')
                 for pp in g_keep ^ o_keep:
-                    assert abs(sc[pp] - theta) <= TIE_BAND, \
+                    assert abs(sc[pp] - theta) <= self.tie_band, \
                         f"selection differs outside the tie band at pos {cur_pos} stream {s}: {sc[pp]} vs {theta}"
                 st.tolerated_divergences += 1
                 st.log.append((cur_pos, s, sorted(g_keep ^ o_keep)))

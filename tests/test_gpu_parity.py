@@ -43,11 +43,11 @@ def _apply_mode(eng, mode):
 
 
 def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=None, steps=None, n_prefix=None,
-                    rows_back=1, sample=None, chunk_rows=0, score_variant=0, mode="calls"):
+                    rows_back=1, sample=None, chunk_rows=0, score_variant=0, mode="calls", score_mode=0):
     H = _harness()
     cap = max(budget_fn(w.n_text + g) for g in range(w.n_cells))
     eng = H.engine_for(w, n_layers=n_layers_engine, page_rows=page_rows, capacity=cap, n_prefix=n_prefix,
-                       local_rows_back=rows_back)
+                       local_rows_back=rows_back, score_mode=score_mode)
     if chunk_rows:
         eng.set_attn_chunk_rows(chunk_rows)
     lh = H.LayerHarness(eng, 0, oracle_cap=w.l_max + 1, sample=sample, score_variant=score_variant,
@@ -305,6 +305,51 @@ def test_tensor_core_kernel_group_sizes_and_ring_depths(warps, depth, ahead):
             q, kn, vn = layer_step_qkv(w, 4, 0, g)
             lh.step(q, kn, vn, w.n_text + g, C)
         assert eng.get_status()[0] == 0 and lh.stats.steps == w.n_cells
+
+
+# ---------------------------------------------------------------------------
+# the comparison method of Section 3.4: attention-mass pruning (score_mode 1)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("mode", ["calls", "fused"])
+@pytest.mark.parametrize("seed", [0, 1])
+def test_attention_mass_mode_config1_full_trajectory(seed, mode):
+    """Config 1 (its eight keys scaled x4 are made for this rule) under attention-mass pruning: masses, kept
+    and evicted sets, outputs and cache contents against the oracle at every step."""
+    w = get_workload(1)
+    C = w.capacity()
+    lh, eng = _run_trajectory(w, 0, seed, lambda cur: C, mode=mode, score_mode=1)
+    assert lh.stats.steps == 256
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+
+
+@pytest.mark.parametrize("d,page_rows,T0,gh,gw,beta,n_prefix", [
+    (64, 7, 5, 6, 5, 0.5, None),
+    (100, 5, 9, 5, 7, 0.5, None),
+    (32, 3, 4, 6, 6, 0.4, 0),        # no prefix: the text rows compete too, with zero mass at first
+])
+def test_attention_mass_mode_small_shapes(d, page_rows, T0, gh, gw, beta, n_prefix):
+    w = Workload(f"mass-d{d}", 80 + d % 7, 1, 2, 3, d, T0, gh, gw, beta, 1.0)
+    C = max(2, w.capacity())
+    lh, eng = _run_trajectory(w, 0, 3, lambda cur: C, page_rows=page_rows, n_prefix=n_prefix, score_mode=1)
+    assert lh.stats.steps == gh * gw
+    # a budget that moves: several rows go at once, survivors (and their masses) move
+    lh, eng = _run_trajectory(w, 0, 4, lambda cur: C - (3 if (cur // 4) % 2 else 0), page_rows=page_rows, n_prefix=n_prefix, score_mode=1)
+    assert lh.stats.steps == gh * gw
+
+
+def test_attention_mass_mode_update_needs_the_attention_first():
+    import paper_2506_18226_b200 as A
+    H = _harness()
+    w = get_workload(1)
+    eng = H.engine_for(w, capacity=w.capacity(), score_mode=1)
+    k, v = prefix_kv(w, 0, 0)
+    eng.prefill_rows(0, H.dev_bf16(k), H.dev_bf16(v), 0)
+    q, kn, vn = (H.dev_bf16(x) for x in layer_step_qkv(w, 0, 0, 0))
+    eng.score(0, 120)
+    eng.select(0, 120, w.capacity())
+    with pytest.raises(A.AdsaError) as e:
+        eng.kv_update(0, 120, kn, vn)
+    assert e.value.status == A.binding.ESTATE
 
 
 # ---------------------------------------------------------------------------

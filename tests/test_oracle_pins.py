@@ -358,6 +358,108 @@ def test_step_scores_equal_eq_1_2_on_the_cached_value_rows():
     assert differs >= 20
 
 
+# --------------------------------------------------------------------------
+# The comparison method of Section 3.4 (attention-mass pruning, score_mode 1)
+# --------------------------------------------------------------------------
+def test_select_highest_equals_argmax_over_all_subsets():
+    rng = np.random.default_rng(31)
+    for trial in range(30):
+        p = int(rng.integers(1, 11))
+        score = (rng.integers(0, 9, size=p) / 8.0).astype(np.float32)      # dyadic masses: exact sums, frequent ties
+        pos = rng.permutation(40)[:p].astype(np.int32)
+        for K in range(p + 1):
+            best = None
+            for sub in itertools.combinations(range(p), K):
+                key = (-sum(float(score[i]) for i in sub), tuple(sorted(int(pos[i]) for i in sub)))
+                if best is None or key < best[0]:
+                    best = (key, sub)
+            keep = orc.select_highest(score, pos, K)
+            assert set(np.flatnonzero(keep).tolist()) == (set(best[1]) if best else set())
+
+
+def _run_mass_steps(T0, H, W, d, budget_fn, n_prefix, seed, n_streams=2, k_scale=None):
+    rng = np.random.default_rng(seed)
+    L = T0 + H * W
+    st = orc.OracleStreams(n_streams, d, L, T0, W, n_prefix, score_mode=1)
+    hk, hv = np.zeros((n_streams, L, d), np.float32), np.zeros((n_streams, L, d), np.float32)
+    hq = np.zeros((n_streams, L, d), np.float32)
+    if T0:
+        hk[:, :T0], hv[:, :T0] = _randn(rng, n_streams, T0, d), _randn(rng, n_streams, T0, d)
+        st.append_rows(hk[:, :T0], hv[:, :T0], 0)
+    log = []
+    for g in range(H * W):
+        cur = T0 + g
+        q, kn, vn = _randn(rng, n_streams, d), _randn(rng, n_streams, d), _randn(rng, n_streams, d)
+        if k_scale is not None:
+            kn = kn * np.float32(k_scale(cur))
+        hq[:, cur], hk[:, cur], hv[:, cur] = q, kn, vn
+        res = st.step(q, kn, vn, cur, budget_fn(cur))
+        log.append((cur, res, st.n_live.copy()))
+    return st, hq, hk, hv, log
+
+
+def test_mass_without_eviction_is_the_column_sum_of_the_attention_matrix():
+    """With room for everything the method is dense attention, and a row's mass is the sum of its softmax
+    weights over the steps since its insertion: the column sums of the causal attention matrix, here from
+    torch's softmax in float64.  Every step hands out a total weight of 1."""
+    T0, H, W, d = 5, 5, 4, 16
+    st, hq, hk, hv, log = _run_mass_steps(T0, H, W, d, lambda cur: 10_000, T0, seed=32)
+    L = T0 + H * W
+    for s in range(2):
+        pos, k, v = st.rows(s)
+        want = np.zeros(L)
+        for cur in range(T0, L):
+            logits = torch.from_numpy(hk[s, :cur + 1].astype(np.float64)) @ torch.from_numpy(hq[s, cur].astype(np.float64)) / np.sqrt(d)
+            want[:cur + 1] += torch.softmax(logits, dim=0).numpy()
+        got = st.mass[s, :len(pos)]
+        np.testing.assert_allclose(got, want[pos], atol=2e-6)
+        assert abs(float(got.astype(np.float64).sum()) - H * W) < 1e-4
+
+
+def test_mass_is_conserved_under_eviction_and_the_least_attended_row_goes():
+    T0, H, W, d = 4, 7, 6, 8
+    C = (T0 + H * W) // 2
+    st, hq, hk, hv, log = _run_mass_steps(T0, H, W, d, lambda cur: C, T0, seed=33)
+    for s in range(2):
+        lost = 0.0
+        for cur, res, n_live in log:
+            sc = dict(zip(res.cand_pos[s].tolist(), res.cand_score[s].tolist()))
+            ev = res.evict_pos[s].tolist()
+            lost += sum(sc[p_] for p_ in ev)
+            if len(ev) == 1:      # cache full: exactly the least attended candidate goes, the higher position on a tie
+                lo = min(sc.values())
+                assert sc[ev[0]] == lo and ev[0] == max(p_ for p_, m in sc.items() if m == lo)
+            kept_c = [sc[p_] for p_ in res.kept_pos[s].tolist() if p_ in sc]
+            assert not ev or not kept_c or max(sc[p_] for p_ in ev) <= min(kept_c)
+        n = int(st.n_live[s])
+        total = float(st.mass[s, :n].astype(np.float64).sum()) + lost
+        assert abs(total - H * W) < 1e-3
+
+
+def test_a_key_that_draws_the_attention_survives_where_similarity_pruning_would_not_care():
+    """Keys of some positions scaled x4 (the benchmark's 'global' keys) draw far more attention than the rest;
+    under attention-mass pruning their rows, once candidates, carry more mass than the median candidate and
+    outlive it.  The V-cosine rule of the paper is blind to key scale."""
+    T0, H, W, d = 6, 10, 8, 32
+    big = {T0 + 3, T0 + 11, T0 + 20}
+    C = (T0 + H * W) // 2
+    st, hq, hk, hv, log = _run_mass_steps(T0, H, W, d, lambda cur: C, T0, seed=34, n_streams=4,
+                                          k_scale=lambda cur: 4.0 if cur in big else 1.0)
+    above, seen = 0, 0
+    for cur, res, n_live in log:
+        for s in range(4):
+            sc = dict(zip(res.cand_pos[s].tolist(), res.cand_score[s].tolist()))
+            if len(sc) < 8:
+                continue
+            med = float(np.median(list(sc.values())))
+            for p_ in big & set(sc):
+                seen += 1
+                above += sc[p_] > med
+    assert seen > 100 and above / seen > 0.9
+    for s in range(4):                       # and they are still cached at the end, in every stream
+        assert big <= set(st.rows(s)[0].tolist())
+
+
 def _golden_rows():
     rows = []
     with open(GOLDEN) as f:
