@@ -100,6 +100,12 @@ typedef struct {
     int32_t score_mode;               /* 0 = mean V-cosine similarity, keep the lowest (Eq. 1-3): the paper's rule.
                                          1 = attention mass, keep the highest: the attention-score pruning that
                                          Section 3.4 argues against, as a comparison (see below) */
+    int32_t score_share;              /* 0 = one score per stream (a head's V row).  1 = one score per batch row and token:
+                                         Eq. 1-2 on the token's V rows of all heads of the layer laid end to end, so
+                                         every head keeps the same tokens (the paper does not fix the granularity of
+                                         the comparison).  Needs score_mode 0; the heads of a batch row must be loaded
+                                         and stepped together (same positions slot by slot, ADSA_DEV_BAD_POSITION
+                                         otherwise); runs on the four stand-alone kernels */
     float softmax_scale;              /* 0 => 1/sqrt(head_dim) */
 } adsa_config;
 

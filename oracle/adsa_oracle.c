@@ -381,6 +381,111 @@ int adsa_oracle_layer_step_mass_batch(const adsa_oracle_params *prm, int n_strea
     return failed;
 }
 
+/* -------------------------------------------------------------------------
+ * Granularity variant.  The paper does not say at which granularity V rows are
+ * compared (Section 4.1 speaks of "the V of each token").  The default reading
+ * is per stream (one head).  This variant compares a token's V over ALL heads of
+ * a layer as one vector of n_heads * d elements, so one score per (batch row,
+ * token) and the same tokens kept for every head.  The n_heads streams of a
+ * batch row are stepped together; their caches must hold the same positions in
+ * the same order (they do if they are always stepped together).  Partition, K,
+ * attention (per head) and update are those of the per-stream step.
+ * Returns 0, -1 on malformed input, -2 if the heads' caches differ.
+ * ------------------------------------------------------------------------- */
+int adsa_oracle_layer_step_shared(const adsa_oracle_params *prm, int n_heads, int d, int cap_rows,
+                                  int *n_live, int *pos, float *k, float *v, /* [n_heads] streams, stride cap_rows */
+                                  const float *q, const float *k_new, const float *v_new, int cur_pos, int budget,
+                                  double *out, int *n_kept, int *kept_pos, int *n_evict, int *evict_pos,
+                                  int *n_cand, int *cand_pos, float *cand_score)
+{
+    const int n = n_live[0], D = n_heads * d;
+    for (int h = 1; h < n_heads; ++h) {
+        if (n_live[h] != n) return -2;
+        for (int i = 0; i < n; ++i) if (pos[(size_t)h * cap_rows + i] != pos[i]) return -2;
+    }
+    int *region = (int *)malloc((size_t)(n + 1) * sizeof(int));
+    int *keep = (int *)malloc((size_t)(n + 1) * sizeof(int));
+    int *cpos = (int *)malloc((size_t)(n + 1) * sizeof(int));
+    float *cscore = (float *)malloc((size_t)(n + 1) * sizeof(float));
+    float *cv = (float *)malloc((size_t)(n + 1) * D * sizeof(float));
+    float *gk = (float *)malloc((size_t)(n + 1) * d * sizeof(float));
+    float *gv = (float *)malloc((size_t)(n + 1) * d * sizeof(float));
+    int rc = 0, n_pre = 0, n_loc = 0, p = 0;
+    for (int i = 0; i < n; ++i) {
+        region[i] = adsa_oracle_region(pos[i], cur_pos, prm->n_text, prm->grid_w, prm->n_prefix, prm->rows_back);
+        if (region[i] == ADSA_REGION_INVALID) { rc = -1; goto done; }
+        if (region[i] == ADSA_REGION_PREFIX) ++n_pre;
+        else if (region[i] == ADSA_REGION_LOCAL) ++n_loc;
+        else {
+            cpos[p] = pos[i];
+            for (int h = 0; h < n_heads; ++h)   /* the token's V over all heads, head after head */
+                memcpy(cv + (size_t)p * D + (size_t)h * d, v + ((size_t)h * cap_rows + i) * d, (size_t)d * sizeof(float));
+            ++p;
+        }
+    }
+    adsa_oracle_score_definition(cv, p, D, cscore);
+    {
+        int K = budget - n_pre - n_loc - 1;
+        if (K < 0) K = 0;
+        if (K > p) K = p;
+        adsa_oracle_select_lowest(cscore, cpos, p, K, keep);
+    }
+    for (int h = 0; h < n_heads && rc == 0; ++h) {
+        size_t r = (size_t)h * cap_rows;
+        int m = 0, e = 0, c = 0;
+        for (int i = 0; i < n; ++i) {
+            int kept = 1;
+            if (region[i] == ADSA_REGION_PREVIOUS) kept = keep[c++];
+            if (kept) {
+                kept_pos[r + m] = pos[r + i];
+                memcpy(gk + (size_t)m * d, k + (r + i) * d, (size_t)d * sizeof(float));
+                memcpy(gv + (size_t)m * d, v + (r + i) * d, (size_t)d * sizeof(float));
+                ++m;
+            } else {
+                evict_pos[r + e++] = pos[r + i];
+            }
+        }
+        n_kept[h] = m; n_evict[h] = e; n_cand[h] = p;
+        memcpy(cand_pos + r, cpos, (size_t)p * sizeof(int));
+        memcpy(cand_score + r, cscore, (size_t)p * sizeof(float));
+        if (m + 1 > cap_rows) { rc = -1; break; }
+        memcpy(gk + (size_t)m * d, k_new + (size_t)h * d, (size_t)d * sizeof(float));
+        memcpy(gv + (size_t)m * d, v_new + (size_t)h * d, (size_t)d * sizeof(float));
+        double scale = prm->softmax_scale != 0.0 ? prm->softmax_scale : 1.0 / sqrt((double)d);
+        adsa_oracle_attend(q + (size_t)h * d, gk, gv, m + 1, d, scale, out + (size_t)h * d, NULL);
+        memcpy(k + r * d, gk, (size_t)(m + 1) * d * sizeof(float));
+        memcpy(v + r * d, gv, (size_t)(m + 1) * d * sizeof(float));
+        memcpy(pos + r, kept_pos + r, (size_t)m * sizeof(int));
+        pos[r + m] = cur_pos;
+        n_live[h] = m + 1;
+    }
+done:
+    free(region); free(keep); free(cpos); free(cscore); free(cv); free(gk); free(gv);
+    return rc;
+}
+
+int adsa_oracle_layer_step_shared_batch(const adsa_oracle_params *prm, int n_rows_batch, int n_heads, int d, int cap_rows,
+                                        int *n_live, int *pos, float *k, float *v,
+                                        const float *q, const float *k_new, const float *v_new, int cur_pos, int budget,
+                                        double *out, int *n_kept, int *kept_pos, int *n_evict, int *evict_pos,
+                                        int *n_cand, int *cand_pos, float *cand_score, int n_threads)
+{
+    int failed = 0;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : failed)
+#endif
+    for (int b = 0; b < n_rows_batch; ++b) {
+        size_t s0 = (size_t)b * n_heads, r = s0 * cap_rows;
+        int rc = adsa_oracle_layer_step_shared(prm, n_heads, d, cap_rows, n_live + s0, pos + r, k + r * d, v + r * d,
+                                               q + s0 * d, k_new + s0 * d, v_new + s0 * d, cur_pos, budget, out + s0 * d,
+                                               n_kept + s0, kept_pos + r, n_evict + s0, evict_pos + r,
+                                               n_cand + s0, cand_pos + r, cand_score + r);
+        if (rc != 0) ++failed;
+    }
+    return failed;
+}
+
 /* The same step for many independent streams.  Arrays carry a leading stream
  * dimension with stride cap_rows (state, lists) or d (q, k_new, v_new, out).
  * Threads split the streams; nothing else is parallel.  Returns the number of

@@ -46,6 +46,7 @@ def lib():
         _lib.adsa_oracle_layer_step.restype = C.c_int
         _lib.adsa_oracle_layer_step_batch.restype = C.c_int
         _lib.adsa_oracle_layer_step_mass_batch.restype = C.c_int
+        _lib.adsa_oracle_layer_step_shared_batch.restype = C.c_int
         _lib.adsa_oracle_max_threads.restype = C.c_int
     return _lib
 
@@ -124,9 +125,13 @@ class OracleStreams:
     """Cache state of `n_streams` independent streams plus the step function over them."""
 
     def __init__(self, n_streams, head_dim, cap_rows, n_text, grid_w, n_prefix, rows_back=1,
-                 softmax_scale=0.0, score_variant=0, score_mode=0):
+                 softmax_scale=0.0, score_variant=0, score_mode=0, share_heads=0):
         """score_mode 0: the paper's rule (Eq. 1-3 on V); 1: attention-mass pruning (Section 3.4's foil), with
-        a per-row mass carried beside the rows (zero for rows loaded from outside)."""
+        a per-row mass carried beside the rows (zero for rows loaded from outside).
+        share_heads = H > 0: consecutive groups of H streams are the heads of one batch row and are scored as
+        one (a token's V over all heads is one vector), so they keep the same tokens."""
+        self.share_heads = share_heads
+        assert share_heads == 0 or (n_streams % share_heads == 0 and score_mode == 0)
         self.n_streams, self.d, self.cap = n_streams, head_dim, cap_rows
         self.score_mode = score_mode
         self.mass = np.zeros((n_streams, cap_rows), dtype=np.float32)
@@ -174,7 +179,14 @@ class OracleStreams:
         evict_pos = np.zeros((S, cap), dtype=np.int32)
         cand_pos = np.zeros((S, cap), dtype=np.int32)
         cand_score = np.zeros((S, cap), dtype=np.float32)
-        if self.score_mode == 1:
+        if self.share_heads:
+            failed = lib().adsa_oracle_layer_step_shared_batch(
+                C.byref(self.prm), S // self.share_heads, self.share_heads, d, cap, _p(self.n_live, C.c_int),
+                _p(self.pos, C.c_int), _p(self.k, C.c_float), _p(self.v, C.c_float), _p(q, C.c_float), _p(k_new, C.c_float),
+                _p(v_new, C.c_float), int(cur_pos), int(budget), _p(out, C.c_double),
+                _p(n_kept, C.c_int), _p(kept_pos, C.c_int), _p(n_evict, C.c_int), _p(evict_pos, C.c_int),
+                _p(n_cand, C.c_int), _p(cand_pos, C.c_int), _p(cand_score, C.c_float), int(n_threads))
+        elif self.score_mode == 1:
             failed = lib().adsa_oracle_layer_step_mass_batch(
                 C.byref(self.prm), S, d, cap, _p(self.n_live, C.c_int), _p(self.pos, C.c_int),
                 _p(self.k, C.c_float), _p(self.v, C.c_float), _p(self.mass, C.c_float), _p(q, C.c_float),

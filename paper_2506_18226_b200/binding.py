@@ -29,7 +29,7 @@ EXPORTS = [
 class AdsaConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "batch", "n_heads", "head_dim", "row_stride", "page_rows", "n_pages",
-        "max_rows_per_stream", "n_text", "grid_h", "grid_w", "n_prefix", "local_rows_back", "score_mode")] + \
+        "max_rows_per_stream", "n_text", "grid_h", "grid_w", "n_prefix", "local_rows_back", "score_mode", "score_share")] + \
         [("softmax_scale", C.c_float)]
 
 
@@ -138,7 +138,7 @@ class AdsaEngine:
 
     def __init__(self, *, n_layers, batch, n_heads, head_dim, n_text, grid_h, grid_w, max_rows_per_stream,
                  page_rows=32, n_pages=None, n_prefix=None, local_rows_back=1, softmax_scale=0.0, row_stride=None,
-                 device="cuda:0", allocate=True, score_mode=0):
+                 device="cuda:0", allocate=True, score_mode=0, score_share=0):
         self.lib = load()
         self.device = torch.device(device)
         row_stride = (head_dim + 7) // 8 * 8 if row_stride is None else row_stride
@@ -148,7 +148,7 @@ class AdsaEngine:
             n_pages = self.n_streams * self.max_pages
         self.cfg = AdsaConfig(n_layers, batch, n_heads, head_dim, row_stride, page_rows, n_pages,
                               max_rows_per_stream, n_text, grid_h, grid_w,
-                              n_text if n_prefix is None else n_prefix, local_rows_back, score_mode, softmax_scale)
+                              n_text if n_prefix is None else n_prefix, local_rows_back, score_mode, score_share, softmax_scale)
         self.S = batch * n_heads
         self.ctx = C.c_void_p(None)
         self._t = {}

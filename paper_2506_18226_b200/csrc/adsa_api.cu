@@ -70,6 +70,7 @@ int check_config(const adsa_config *c)
     if (c->n_text < 0 || c->grid_h < 1 || c->grid_w < 1) return ADSA_EINVAL;
     if (c->n_prefix < 0 || c->local_rows_back < 0) return ADSA_EINVAL;
     if (c->score_mode != 0 && c->score_mode != 1) return ADSA_EINVAL;
+    if (c->score_share != 0 && (c->score_share != 1 || c->score_mode != 0 || c->n_heads > 256)) return ADSA_EINVAL;
     if (!(c->softmax_scale >= 0.f) || isinf(c->softmax_scale)) return ADSA_EINVAL;
     if ((long long)c->n_layers * c->batch * c->n_heads > (1ll << 24)) return ADSA_EINVAL;
     if ((long long)c->n_pages * c->page_rows * c->row_stride > (1ll << 40)) return ADSA_EINVAL;
@@ -193,7 +194,7 @@ StagedChoice choose_staged(const adsa_ctx *ctx, int n_rows, bool fused)
     StagedChoice ch = {};
     const int m = ctx->kernel_mode;
     if (m == 0) return ch;
-    if (ctx->cfg.score_mode != 0) return ch;   // attention-mass pruning (the comparison method) runs on the four stand-alone kernels
+    if (ctx->cfg.score_mode != 0 || ctx->cfg.score_share != 0) return ch;   // the comparison method and the per-layer granularity run on the four stand-alone kernels
     if ((m == 1 || m == 4) && ctx->mma_ok) {
         ch.wp = plan_wstep(ctx->dev, fused, ctx->sm_count, ctx->max_stages, ctx->stream_warps);
         if (ctx->l2_ahead >= 0) ch.wp.l2_ahead = ctx->l2_ahead;
@@ -307,6 +308,8 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.logit = (float *)(w + ws.logit);
     d.ml = (float *)(w + ws.ml);
     d.score_mode = cfg->score_mode;
+    d.score_share = cfg->score_share;
+    d.n_heads = cfg->n_heads;
     d.status = (uint32_t *)(w + ws.status);
     d.d = cfg->head_dim;
     d.row_stride = cfg->row_stride;
@@ -584,7 +587,7 @@ static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_ro
     // sweeping, updating) instead of all starting and all draining together once per layer.  Taken when
     // every layer is between steps and in the same carried state; otherwise layer by layer.
     bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok &&
-                      ctx->cfg.score_mode == 0;
+                      ctx->cfg.score_mode == 0 && ctx->cfg.score_share == 0;
     if (one_launch) {
         const LayerState &L0 = ctx->layers[l0];
         for (int l = 0; l < NL && one_launch; ++l) {
@@ -851,6 +854,7 @@ namespace adsa {
 cudaError_t configure_kernels(const DevCtx &c)
 {
     cudaError_t e = configure_select_kernel(c);
+    if (e == cudaSuccess) e = configure_score_kernel(c);
     if (e == cudaSuccess) e = configure_update_kernel(c);
     if (e == cudaSuccess) e = configure_step_kernel(c);
     return e != cudaSuccess ? e : configure_pstep_kernel(c);

@@ -48,6 +48,8 @@ struct DevCtx {
     int partial_stride;     // floats per split partial: row_stride + 2 (m, l)
     uint32_t pr_magic;      // slot / page_rows == __umulhi(slot, pr_magic)
     int n_text, grid_w, n_prefix, rows_back;
+    int n_heads;            // heads per batch row (streams b * n_heads .. of a layer belong to batch row b)
+    int score_share;        // 1: Eq. 1-2 on a token's V over all heads of the layer (one score per batch row and token)
     int score_mode;         // 0: Eq. 1-3 (mean V-cosine similarity, keep the lowest); 1: attention mass, keep the highest
     float scale_log2e;      // softmax scale * log2(e)
 };

@@ -89,6 +89,7 @@ cudaError_t configure_wstep_kernel(const DevCtx &c);
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t configure_kernels(const DevCtx &c);
 cudaError_t configure_select_kernel(const DevCtx &c);
+cudaError_t configure_score_kernel(const DevCtx &c);
 cudaError_t configure_update_kernel(const DevCtx &c);
 
 }  // namespace adsa

@@ -118,6 +118,116 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 }
 
 // ---------------------------------------------------------------------------
+// Eq. 1-2 at the granularity of a layer: a token's V rows of all heads of a batch row are one vector of
+// n_heads * d elements, so u_j = v_j / |v_j| with |v_j|^2 summed over the heads, one score per (batch row,
+// token), written to every head's stream.  One block per batch row; the heads' caches must hold the same
+// positions slot by slot (they do when they are always stepped together; a difference raises
+// ADSA_DEV_BAD_POSITION).  Same row-sum identity as above, head after head.
+// Dynamic shared memory: 1/|v_j| by slot (0 = not a candidate), then s for every head.
+// ---------------------------------------------------------------------------
+template <int LPR>
+__global__ void __launch_bounds__(kSSThreads)
+score_shared_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
+{
+    constexpr int RPW = 32 / LPR;
+    extern __shared__ float sh_f[];
+    __shared__ float s_part[kSSWarps][256];
+    __shared__ int s_p;
+    float *invn = sh_f, *svec = sh_f + c.max_rows;
+    const int H = c.n_heads, b = blockIdx.x, local0 = b * H, sid0 = layer * c.S + local0;
+    const int n = c.n_live[sid0];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane % LPR, grp = lane / LPR;
+    const bool piece_ok = sub * 8 < c.row_stride;
+    if (threadIdx.x == 0) s_p = 0;
+    if (threadIdx.x < H && c.n_live[sid0 + threadIdx.x] != n) set_status(c, ADSA_DEV_BAD_POSITION);
+    __syncthreads();
+    // the tokens' norms over all heads, which of them are candidates, and whether the heads agree
+    for (int base = 0; base < n; base += kSSThreads) {
+        const int slot = base + threadIdx.x;
+        bool cand = false;
+        if (slot < n) {
+            const int ps = c.pos[(size_t)sid0 * c.max_rows + slot];
+            float ss = 0.f;
+            for (int h = 0; h < H; ++h) {
+                const size_t at = (size_t)(sid0 + h) * c.max_rows + slot;
+                const float nr = 1.0f / c.inv_norm[at];   // the head's |v| (1e-8 for an all-zero row)
+                ss = fmaf(nr, nr, ss);
+                if (c.pos[at] != ps) set_status(c, ADSA_DEV_BAD_POSITION);
+            }
+            const int reg = region_of(c, ps, cur_pos);
+            if (reg == kRegionInvalid) set_status(c, ADSA_DEV_BAD_POSITION);
+            cand = reg == kRegionPrevious;
+            invn[slot] = cand ? 1.0f / fmaxf(sqrtf(ss), kNormEps) : 0.f;
+        }
+        const unsigned bc = __ballot_sync(0xffffffffu, cand);
+        if (lane == 0 && bc) atomicAdd(&s_p, __popc(bc));
+    }
+    __syncthreads();
+    const int p = s_p;
+    // s^h = sum over the candidates of v_j^h / |v_j|, for every head
+    for (int h = 0; h < H; ++h) {
+        const int32_t *pt = c.page_table + (size_t)(sid0 + h) * c.max_pages;
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {
+            const float w = invn[slot];
+            if (w == 0.f || !piece_ok) continue;
+            float f[8];
+            unpack8(ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+        }
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+        }
+        if (grp == 0 && piece_ok) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_part[warp][sub * 8 + e] = acc[e];
+        }
+        __syncthreads();
+        if (threadIdx.x < c.row_stride) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kSSWarps; ++w) t += s_part[w][threadIdx.x];
+            svec[h * c.row_stride + threadIdx.x] = t;
+        }
+        __syncthreads();
+    }
+    // S_j = (u_j . s - u_j . u_j) / (p - 1), the dot products summed over the heads
+    for (int sb = warp * RPW; sb < n; sb += kSSWarps * RPW) {   // warp-uniform bounds: all lanes join the shuffles
+        const int slot = sb + grp;
+        const float w = slot < n ? invn[slot] : 0.f;
+        float dot = 0.f, self = 0.f;
+        if (w != 0.f && piece_ok) {
+            for (int h = 0; h < H; ++h) {
+                float f[8];
+                unpack8(ldg128(c.v_pool + row_offset(c, c.page_table + (size_t)(sid0 + h) * c.max_pages, slot) + sub * 8), f);
+                const float *sv = svec + h * c.row_stride + sub * 8;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], sv[e], dot); self = fmaf(f[e], f[e], self); }
+            }
+        }
+#pragma unroll
+        for (int o = 1; o < LPR; o <<= 1) {
+            dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            self += __shfl_xor_sync(0xffffffffu, self, o);
+        }
+        if (sub == 0 && slot < n) {
+            float S = CUDART_NAN_F;
+            if (w != 0.f) S = p > 1 ? (w * dot - w * w * self) / (float)(p - 1) + 0.0f : 0.0f;
+            for (int h = 0; h < H; ++h) {
+                c.scores[(size_t)(sid0 + h) * c.max_rows + slot] = S;
+                if (scores_out) scores_out[(size_t)(local0 + h) * c.max_rows + slot] = S;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Eq. 3 plus the always-kept regions: the threshold comes from block_select, this
 // kernel turns it into the keep mask, the retained / evicted lists and the counts.
 // ---------------------------------------------------------------------------
@@ -204,8 +314,32 @@ static int lanes_per_row(int row_stride)
     return pieces <= 4 ? 4 : pieces <= 8 ? 8 : pieces <= 16 ? 16 : 32;
 }
 
+static size_t score_shared_smem(const DevCtx &c) { return ((size_t)c.max_rows + (size_t)c.n_heads * c.row_stride) * sizeof(float); }
+
+cudaError_t configure_score_kernel(const DevCtx &c)
+{
+    if (!c.score_share || score_shared_smem(c) <= 48 * 1024) return cudaSuccess;
+    const int b = (int)score_shared_smem(c);
+    cudaError_t e = cudaFuncSetAttribute(score_shared_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_shared_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, b);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_shared_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, b);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_shared_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, b);
+    return e;
+}
+
 cudaError_t launch_score(const DevCtx &c, int layer, int cur_pos, float *scores_out, cudaStream_t st)
 {
+    if (c.score_share) {   // one block per batch row: a token's V over all heads is one vector
+        const int batch = c.S / c.n_heads;
+        const size_t sm = score_shared_smem(c);
+        switch (lanes_per_row(c.row_stride)) {
+        case 4: score_shared_kernel<4><<<batch, kSSThreads, sm, st>>>(c, layer, cur_pos, scores_out); break;
+        case 8: score_shared_kernel<8><<<batch, kSSThreads, sm, st>>>(c, layer, cur_pos, scores_out); break;
+        case 16: score_shared_kernel<16><<<batch, kSSThreads, sm, st>>>(c, layer, cur_pos, scores_out); break;
+        default: score_shared_kernel<32><<<batch, kSSThreads, sm, st>>>(c, layer, cur_pos, scores_out); break;
+        }
+        return cudaGetLastError();
+    }
     switch (lanes_per_row(c.row_stride)) {
     case 4: score_kernel<4><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;
     case 8: score_kernel<8><<<c.S, kSSThreads, 0, st>>>(c, layer, cur_pos, scores_out); break;

@@ -58,11 +58,13 @@ class LayerHarness:
         self.S, self.d = eng.S, cfg.head_dim
         # sample: the streams (indices within the layer) the oracle follows; None = all
         self.sample = list(range(self.S)) if sample is None else list(sample)
+        assert not cfg.score_share or sample is None, "head-shared selection: the oracle follows whole batch rows"
         self.mass_mode = cfg.score_mode == 1
         self.score_atol = MASS_ATOL if self.mass_mode else SCORE_ATOL
         self.tie_band = MASS_ATOL if self.mass_mode else TIE_BAND
         self.orc = orc.OracleStreams(len(self.sample), self.d, oracle_cap, cfg.n_text, cfg.grid_w, cfg.n_prefix,
-                                     cfg.local_rows_back, float(cfg.softmax_scale), score_variant, score_mode=cfg.score_mode)
+                                     cfg.local_rows_back, float(cfg.softmax_scale), score_variant, score_mode=cfg.score_mode,
+                                     share_heads=cfg.n_heads if cfg.score_share else 0)
         dev = eng.device
         R = cfg.max_rows_per_stream
         self.scores = torch.zeros((self.S, R), dtype=torch.float32, device=dev)

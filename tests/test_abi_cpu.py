@@ -21,7 +21,7 @@ def _declared():
 def _cfg(**kw):
     base = dict(n_layers=2, batch=2, n_heads=4, head_dim=64, row_stride=64, page_rows=16, n_pages=400,
                 max_rows_per_stream=188, n_text=120, grid_h=16, grid_w=16, n_prefix=120, local_rows_back=1,
-                score_mode=0, softmax_scale=0.0)
+                score_mode=0, score_share=0, softmax_scale=0.0)
     base.update(kw)
     return A.AdsaConfig(*[base[n] for n, _ in A.AdsaConfig._fields_])
 
@@ -45,7 +45,7 @@ def test_strerror_and_workspace_size():
 @pytest.mark.parametrize("bad", [
     dict(head_dim=4), dict(head_dim=300, row_stride=304), dict(row_stride=60), dict(row_stride=100, head_dim=100),
     dict(page_rows=1), dict(n_pages=0), dict(max_rows_per_stream=0), dict(grid_w=0), dict(n_prefix=-1),
-    dict(score_mode=3), dict(softmax_scale=-1.0), dict(n_layers=0),
+    dict(score_mode=3), dict(score_share=2), dict(score_share=1, score_mode=1), dict(softmax_scale=-1.0), dict(n_layers=0),
 ])
 def test_invalid_configurations_are_rejected(bad):
     out = C.c_size_t(0)

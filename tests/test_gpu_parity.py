@@ -43,11 +43,11 @@ def _apply_mode(eng, mode):
 
 
 def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=None, steps=None, n_prefix=None,
-                    rows_back=1, sample=None, chunk_rows=0, score_variant=0, mode="calls", score_mode=0):
+                    rows_back=1, sample=None, chunk_rows=0, score_variant=0, mode="calls", score_mode=0, score_share=0):
     H = _harness()
     cap = max(budget_fn(w.n_text + g) for g in range(w.n_cells))
     eng = H.engine_for(w, n_layers=n_layers_engine, page_rows=page_rows, capacity=cap, n_prefix=n_prefix,
-                       local_rows_back=rows_back, score_mode=score_mode)
+                       local_rows_back=rows_back, score_mode=score_mode, score_share=score_share)
     if chunk_rows:
         eng.set_attn_chunk_rows(chunk_rows)
     lh = H.LayerHarness(eng, 0, oracle_cap=w.l_max + 1, sample=sample, score_variant=score_variant,
@@ -350,6 +350,28 @@ def test_attention_mass_mode_update_needs_the_attention_first():
     with pytest.raises(A.AdsaError) as e:
         eng.kv_update(0, 120, kn, vn)
     assert e.value.status == A.binding.ESTATE
+
+
+# ---------------------------------------------------------------------------
+# granularity variant: one score per token over all heads of a layer (score_share 1)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("d,heads,page_rows,T0,gh,gw,beta", [
+    (64, 4, 16, 6, 7, 6, 0.5),
+    (100, 3, 5, 9, 5, 7, 0.5),
+    (32, 12, 8, 4, 6, 6, 0.4),
+])
+@pytest.mark.parametrize("mode", ["calls", "fused"])
+def test_head_shared_selection_full_trajectory(d, heads, page_rows, T0, gh, gw, beta, mode):
+    """Eq. 1-2 on a token's V over all heads: scores, kept and evicted sets (the same for every head of a
+    batch row), outputs and caches against the oracle; then a budget that moves (several rows at once)."""
+    w = Workload(f"shared-d{d}", 70 + d % 7, 1, 2, heads, d, T0, gh, gw, beta, 1.0)
+    C = max(2, w.capacity())
+    lh, eng = _run_trajectory(w, 0, 5, lambda cur: C, page_rows=page_rows, mode=mode, score_share=1)
+    assert lh.stats.steps == gh * gw and lh.stats.max_score_err <= 1e-6
+    pos = np.sort(eng._t["pos"][:, :C].cpu().numpy(), axis=1).reshape(w.batch, heads, C)
+    assert (pos == pos[:, :1]).all()                     # every head of a batch row holds the same tokens
+    lh, eng = _run_trajectory(w, 0, 6, lambda cur: C - (3 if (cur // 4) % 2 else 0), page_rows=page_rows, mode=mode, score_share=1)
+    assert lh.stats.steps == gh * gw
 
 
 # ---------------------------------------------------------------------------

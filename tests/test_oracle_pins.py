@@ -460,6 +460,97 @@ def test_a_key_that_draws_the_attention_survives_where_similarity_pruning_would_
         assert big <= set(st.rows(s)[0].tolist())
 
 
+# --------------------------------------------------------------------------
+# Granularity variant: one score per token over all heads of a layer
+# --------------------------------------------------------------------------
+def _run_shared_steps(T0, Hg, W, d, n_heads, budget, seed, share):
+    rng = np.random.default_rng(seed)
+    L = T0 + Hg * W
+    st = orc.OracleStreams(n_heads, d, L, T0, W, T0, share_heads=n_heads if share else 0)
+    hv = np.zeros((n_heads, L, d), np.float32)
+    hk = np.zeros((n_heads, L, d), np.float32)
+    hk[:, :T0], hv[:, :T0] = _randn(rng, n_heads, T0, d), _randn(rng, n_heads, T0, d)
+    st.append_rows(hk[:, :T0], hv[:, :T0], 0)
+    log = []
+    for g in range(Hg * W):
+        cur = T0 + g
+        q, kn, vn = _randn(rng, n_heads, d), _randn(rng, n_heads, d), _randn(rng, n_heads, d)
+        hk[:, cur], hv[:, cur] = kn, vn
+        log.append((cur, q, st.step(q, kn, vn, cur, budget)))
+    return st, hk, hv, log
+
+
+def test_shared_selection_scores_the_concatenated_value_rows():
+    """One score per token: Eq. 1-2 on the token's V rows of all heads laid end to end (taken from the full
+    history, which the step never sees); every head keeps the same tokens; each head's output is library
+    attention over its own rows at those tokens."""
+    T0, Hg, W, d, NH = 4, 6, 5, 8, 3
+    C = (T0 + Hg * W) // 2
+    st, hk, hv, log = _run_shared_steps(T0, Hg, W, d, NH, C, seed=41, share=True)
+    evictions = 0
+    for cur, q, res in log:
+        cp = res.cand_pos[0]
+        if len(cp):
+            cat = np.concatenate([hv[h, cp] for h in range(NH)], axis=1)
+            want = orc.score_definition(cat)
+            for h in range(NH):
+                assert np.array_equal(res.cand_pos[h], cp)
+                np.testing.assert_array_equal(res.cand_score[h], want)
+        for h in range(NH):
+            assert np.array_equal(res.kept_pos[h], res.kept_pos[0]) and np.array_equal(res.evict_pos[h], res.evict_pos[0])
+            idx = np.array(sorted(res.kept_pos[h].tolist()) + [cur])
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                torch.from_numpy(q[h].astype(np.float64))[None, None, None, :],
+                torch.from_numpy(hk[h, idx].astype(np.float64))[None, None],
+                torch.from_numpy(hv[h, idx].astype(np.float64))[None, None])[0, 0, 0].numpy()
+            np.testing.assert_allclose(res.out[h], ref, atol=1e-10)
+        evictions += len(res.evict_pos[0])
+    assert evictions > 5
+
+
+def test_shared_selection_with_one_head_is_the_per_stream_step():
+    a = _run_shared_steps(5, 5, 4, 8, 1, 12, seed=42, share=True)
+    b = _run_shared_steps(5, 5, 4, 8, 1, 12, seed=42, share=False)
+    for (cur, q, ra), (_, _, rb) in zip(a[3], b[3]):
+        assert np.array_equal(ra.kept_pos[0], rb.kept_pos[0]) and np.array_equal(ra.cand_score[0], rb.cand_score[0])
+        assert np.array_equal(ra.out, rb.out)
+
+
+def test_shared_selection_sees_redundancy_that_one_head_alone_misjudges():
+    """Tokens 1 and 5 have the same V in head 0 but orthogonal V in head 1; tokens 2 and 6 have the same V in
+    both heads.  Over both heads the pair (2, 6) is the most redundant (cosine 1 against 1/2) and, with room for
+    all but one, token 6 goes; head 0 on its own sees two equally redundant pairs and, by the position rule,
+    would drop token 6 as well only by luck of the order: with the pairs swapped it drops the wrong one."""
+    d, W = 8, 4
+    e = np.eye(16, d, dtype=np.float32)
+    def build(full_pair, half_pair):
+        v0 = np.stack([e[i % d] * 2 for i in range(8)])
+        v1 = np.stack([e[(i + 3) % d] * 2 for i in range(8)])
+        v0[:] = 0; v1[:] = 0
+        for i in range(8):
+            v0[i, i] = 2.0; v1[i, (i + 1) % 8] = 2.0
+        a, b = full_pair
+        v0[b], v1[b] = v0[a], v1[a]
+        a, b = half_pair
+        v0[b] = v0[a]
+        return np.stack([v0, v1])
+    rng = np.random.default_rng(43)
+    cur = 5 * W + 1
+    for full_pair, half_pair, want in (((2, 6), (1, 5), 6), ((1, 5), (2, 6), 5)):
+        v = build(full_pair, half_pair)
+        st = orc.OracleStreams(2, d, 16, 0, W, 0, share_heads=2)
+        for h in range(2):
+            st.load(h, np.arange(8), _randn(rng, 8, d), v[h])
+        res = st.step(_randn(rng, 2, d), _randn(rng, 2, d), _randn(rng, 2, d), cur, budget=8)
+        assert res.evict_pos[0].tolist() == [want] and res.evict_pos[1].tolist() == [want]
+    # head 0 alone: both pairs score the same, the highest position (6) goes whichever pair is the full one
+    v = build((1, 5), (2, 6))
+    st = orc.OracleStreams(1, d, 16, 0, W, 0)
+    st.load(0, np.arange(8), _randn(rng, 8, d), v[0])
+    res = st.step(_randn(rng, 1, d), _randn(rng, 1, d), _randn(rng, 1, d), cur, budget=8)
+    assert res.evict_pos[0].tolist() == [6]
+
+
 def _golden_rows():
     rows = []
     with open(GOLDEN) as f:
