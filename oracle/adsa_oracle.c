@@ -486,6 +486,44 @@ int adsa_oracle_layer_step_shared_batch(const adsa_oracle_params *prm, int n_row
     return failed;
 }
 
+/* -------------------------------------------------------------------------
+ * Dense causal attention over the rows of the condition (how the text tokens
+ * enter the cache before decoding starts; Section 4.2: the method is plain
+ * attention while the cache has room): out_i = attention of q_i over rows 0..i.
+ * ------------------------------------------------------------------------- */
+void adsa_oracle_causal_attend(const float *q, const float *k, const float *v, int n, int d, double scale, double *out)
+{
+    for (int i = 0; i < n; ++i)
+        adsa_oracle_attend(q + (size_t)i * d, k, v, i + 1, d, scale, out + (size_t)i * d, NULL);
+}
+
+/* -------------------------------------------------------------------------
+ * Two-dimensional rotary position embedding of q or k rows (Section 4.1 notes
+ * that RoPE sits on Q and K, which is why V is what gets compared).  The paper
+ * does not spell the embedding out; reading taken: elements are rotated in
+ * consecutive pairs (2i, 2i+1); the first d/4 pairs turn with the token's grid
+ * ROW, the next d/4 pairs with its grid COLUMN, pair i of either half by the
+ * angle index * base^(-i / (d/4)); a token of the text condition (pos < n_text)
+ * is not rotated.  d must be a multiple of 4.  x: [n][d], pos: [n].
+ * ------------------------------------------------------------------------- */
+void adsa_oracle_rope_2d(const float *x, const int *pos, int n, int d, int n_text, int grid_w, double base, double *out)
+{
+    const int quarter = d / 4;
+    for (int r = 0; r < n; ++r) {
+        const int cell = pos[r] - n_text;
+        for (int i = 0; i < d / 2; ++i) {
+            double angle = 0.0;
+            if (cell >= 0) {
+                const int index = i < quarter ? cell / grid_w : cell % grid_w;
+                angle = (double)index * pow(base, -(double)(i % quarter) / (double)quarter);
+            }
+            const double a = x[(size_t)r * d + 2 * i], b = x[(size_t)r * d + 2 * i + 1];
+            out[(size_t)r * d + 2 * i] = a * cos(angle) - b * sin(angle);
+            out[(size_t)r * d + 2 * i + 1] = a * sin(angle) + b * cos(angle);
+        }
+    }
+}
+
 /* The same step for many independent streams.  Arrays carry a leading stream
  * dimension with stride cap_rows (state, lists) or d (q, k_new, v_new, out).
  * Threads split the streams; nothing else is parallel.  Returns the number of

@@ -112,6 +112,27 @@ def attend(q, k, v, scale=None):
     return out, w
 
 
+def causal_attend(q, k, v, scale=None) -> np.ndarray:
+    """Dense causal attention: row i of q attends rows 0..i of k, v.  [n, d] each -> [n, d] float64."""
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    n, d = k.shape
+    out = np.zeros((n, d), dtype=np.float64)
+    sc = float(scale) if scale is not None else 1.0 / np.sqrt(d)
+    lib().adsa_oracle_causal_attend(_p(q, C.c_float), _p(k, C.c_float), _p(v, C.c_float), n, d, C.c_double(sc), _p(out, C.c_double))
+    return out
+
+
+def rope_2d(x, pos, n_text, grid_w, base=10000.0) -> np.ndarray:
+    """Two-dimensional rotary embedding of rows x [n, d] at context positions pos [n] -> [n, d] float64."""
+    x = _f32(x)
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    n, d = x.shape
+    assert d % 4 == 0
+    out = np.zeros((n, d), dtype=np.float64)
+    lib().adsa_oracle_rope_2d(_p(x, C.c_float), _p(pos, C.c_int), n, d, int(n_text), int(grid_w), C.c_double(base), _p(out, C.c_double))
+    return out
+
+
 @dataclass
 class StepResult:
     out: np.ndarray          # [streams, d] float64

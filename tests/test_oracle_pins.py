@@ -551,6 +551,55 @@ def test_shared_selection_sees_redundancy_that_one_head_alone_misjudges():
     assert res.evict_pos[0].tolist() == [6]
 
 
+# --------------------------------------------------------------------------
+# Prefill of the condition (dense causal attention) and 2-D rotary embedding
+# --------------------------------------------------------------------------
+def test_causal_attend_is_library_causal_attention():
+    rng = np.random.default_rng(51)
+    for n, d in [(1, 8), (17, 64), (120, 100)]:
+        q, k, v = _randn(rng, n, d), _randn(rng, n, d), _randn(rng, n, d)
+        out = orc.causal_attend(q, k, v)
+        t = lambda x: torch.from_numpy(x.astype(np.float64))[None, None]
+        ref = torch.nn.functional.scaled_dot_product_attention(t(q), t(k), t(v), is_causal=True)[0, 0].numpy()
+        np.testing.assert_allclose(out, ref, atol=1e-10)
+        np.testing.assert_allclose(out[0], v[0], atol=1e-12)              # the first row sees only itself
+
+
+def test_rope_2d_hand_values_and_invariants():
+    T0, W, d = 3, 5, 8                                   # two pairs per axis: angles index * 1 and index * base^(-1/2)
+    base = 10000.0
+    x = np.zeros((3, d), np.float32)
+    x[:, 0] = 1.0; x[:, 2] = 1.0; x[:, 4] = 1.0; x[:, 6] = 1.0     # every pair is (1, 0)
+    pos = np.array([1, T0 + 0, T0 + 2 * W + 3])          # a text token, cell (0, 0), cell (row 2, column 3)
+    out = orc.rope_2d(x, pos, T0, W, base)
+    np.testing.assert_allclose(out[0], x[0], atol=1e-15)             # text tokens are not rotated
+    np.testing.assert_allclose(out[1], x[1], atol=1e-15)             # neither is the grid's origin
+    th = base ** -0.5
+    want = [np.cos(2), np.sin(2), np.cos(2 * th), np.sin(2 * th), np.cos(3), np.sin(3), np.cos(3 * th), np.sin(3 * th)]
+    np.testing.assert_allclose(out[2], want, atol=1e-12)
+    # a rotation: pair norms are kept
+    rng = np.random.default_rng(52)
+    y = _randn(rng, 40, 16)
+    p = rng.integers(0, T0 + 7 * W, size=40)
+    r = orc.rope_2d(y, p, T0, W)
+    np.testing.assert_allclose((r.reshape(40, 8, 2) ** 2).sum(-1), (y.astype(np.float64).reshape(40, 8, 2) ** 2).sum(-1), rtol=1e-12)
+
+
+def test_rope_2d_makes_the_logit_depend_on_the_grid_offset_only():
+    """q.k after the embedding depends on the row and column distances of the two cells, not on where they
+    lie (the reason RoPE sits on Q and K): shifting both cells by the same rows and columns changes nothing."""
+    T0, W, d = 4, 9, 32
+    rng = np.random.default_rng(53)
+    q, k = _randn(rng, 1, d), _randn(rng, 1, d)
+    cell = lambda r, c: np.array([T0 + r * W + c])
+    ref = (orc.rope_2d(q, cell(3, 5), T0, W) @ orc.rope_2d(k, cell(1, 2), T0, W).T).item()
+    for dr, dc in [(1, 0), (0, 3), (4, 2), (-1, -2)]:
+        got = (orc.rope_2d(q, cell(3 + dr, 5 + dc), T0, W) @ orc.rope_2d(k, cell(1 + dr, 2 + dc), T0, W).T).item()
+        assert abs(got - ref) < 1e-9
+    other = (orc.rope_2d(q, cell(3, 5), T0, W) @ orc.rope_2d(k, cell(2, 2), T0, W).T).item()
+    assert abs(other - ref) > 1e-3
+
+
 def _golden_rows():
     rows = []
     with open(GOLDEN) as f:
