@@ -146,6 +146,24 @@ ADSA_API int adsa_reset(adsa_ctx *ctx, adsa_stream_t stream);
 ADSA_API int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, const int32_t *pos, int n_rows,
                                int first_pos, adsa_stream_t stream);
 
+/* The condition entering an EMPTY cache with its attention computed on the way (Section 4.2: while the cache
+ * has room the method is plain attention): for every stream of `layer`, row i of q attends rows 0 .. i of
+ * k, v (dense causal attention, fp32 softmax), and the n_rows rows of k, v are appended to the cache at
+ * positions first_pos .. first_pos+n_rows-1 exactly as adsa_prefill_rows does.  q, k, v: [device] bf16
+ * [batch][n_heads][n_rows][head_dim], 4-byte aligned (k and q already rotated, see adsa_rope_2d).
+ * out_bf16 / out_f32: [device] same shape; either may be NULL, not both.  ADSA_ESTATE if the layer's cache
+ * is not empty. */
+ADSA_API int adsa_prefill_attn(adsa_ctx *ctx, int layer, const void *q, const void *k, const void *v, int n_rows, int first_pos,
+                               void *out_bf16, float *out_f32, adsa_stream_t stream);
+
+/* Two-dimensional rotary position embedding of q or k rows, in place (Section 4.1: the embedding sits on Q and
+ * K, which is why the V rows are what Eq. 1-2 compare).  x: [device] bf16 [n_rows][head_dim], pos: [device] int32
+ * [n_rows] context positions.  Elements turn in consecutive pairs (2i, 2i+1): the first head_dim/4 pairs by the
+ * token's grid row, the next head_dim/4 by its grid column, pair i of either half by the angle
+ * index * base^(-i / (head_dim/4)); rows of the text condition (pos < n_text) are left as they are.
+ * head_dim must be a multiple of 4; base 0 => 10000.  fp32 arithmetic, bf16 result rounded to nearest even. */
+ADSA_API int adsa_rope_2d(adsa_ctx *ctx, void *x, const int32_t *pos, long long n_rows, float base, adsa_stream_t stream);
+
 /* Replace the cache of one stream by the given rows (tests, resynchronisation,
  * restoring a snapshot).  k, v: [device] bf16 [n_rows][head_dim]; pos: [device]
  * int32 [n_rows], distinct.  Pages are freed or taken as needed. */

@@ -20,7 +20,7 @@ DEV_POOL_EXHAUSTED, DEV_BAD_POSITION, DEV_ROW_OVERFLOW, DEV_RING_TIMEOUT, DEV_BA
 
 EXPORTS = [
     "adsa_workspace_bytes", "adsa_create", "adsa_destroy", "adsa_reset", "adsa_prefill_rows",
-    "adsa_set_stream_rows", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
+    "adsa_set_stream_rows", "adsa_prefill_attn", "adsa_rope_2d", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
     "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_stream_warps", "adsa_set_single_sweep",
     "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror", "adsa_decode_attn_static",
 ]
@@ -61,6 +61,8 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_reset": [vp, vp],
             "adsa_prefill_rows": [vp, i32, vp, vp, vp, i32, i32, vp],
             "adsa_set_stream_rows": [vp, i32, i32, i32, vp, vp, vp, i32, vp],
+            "adsa_prefill_attn": [vp, i32, vp, vp, vp, i32, i32, vp, vp, vp],
+            "adsa_rope_2d": [vp, vp, vp, C.c_longlong, C.c_float, vp],
             "adsa_score": [vp, i32, i32, vp, vp],
             "adsa_select": [vp, i32, i32, i32, vp, vp, vp, vp, vp],
             "adsa_sparse_decode_attn": [vp, i32, i32, vp, vp, vp, vp, vp, vp],
@@ -205,6 +207,15 @@ class AdsaEngine:
         """k, v: [batch, heads, n_rows, head_dim] bf16 on the device; pos: optional int32 [batch, heads, n_rows]."""
         n_rows = k.shape[-2]
         self._call("adsa_prefill_rows", layer, _ptr(k), _ptr(v), _ptr(pos), n_rows, first_pos, _stream())
+
+    def prefill_attn(self, layer, q, k, v, first_pos=0, out_bf16=None, out_f32=None):
+        """Dense causal attention over the given rows, which also enter the (empty) cache.  [batch, heads, n_rows, head_dim]."""
+        self._call("adsa_prefill_attn", layer, _ptr(q), _ptr(k), _ptr(v), k.shape[-2], first_pos, _ptr(out_bf16), _ptr(out_f32),
+                   _stream())
+
+    def rope_2d(self, x, pos, base=0.0):
+        """2-D rotary embedding in place.  x: [..., head_dim] bf16 (contiguous), pos: int32, one per row of x."""
+        self._call("adsa_rope_2d", _ptr(x), _ptr(pos), x.numel() // x.shape[-1], float(base), _stream())
 
     def set_stream_rows(self, layer, b, h, k, v, pos):
         n = 0 if pos is None else int(pos.shape[0])

@@ -395,6 +395,31 @@ int adsa_prefill_rows(adsa_ctx *ctx, int layer, const void *k, const void *v, co
     return cuda_fail(ctx, launch_append_rows(ctx->dev, layer, k, v, pos, n_rows, first_pos, (cudaStream_t)stream));
 }
 
+int adsa_prefill_attn(adsa_ctx *ctx, int layer, const void *q, const void *k, const void *v, int n_rows, int first_pos,
+                      void *out_bf16, float *out_f32, adsa_stream_t stream)
+{
+    int rc = check_layer(ctx, layer);
+    if (rc) return rc;
+    if (!q || !k || !v || (!out_bf16 && !out_f32) || n_rows < 1 || first_pos < 0) return ADSA_EINVAL;
+    if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v) & 3u) return ADSA_EINVAL;
+    LayerState &L = ctx->layers[layer];
+    if (L.phase != kIdle || L.rows_hi != 0) return ADSA_ESTATE;   // the rows attend each other only: the cache must be empty
+    rc = adsa_prefill_rows(ctx, layer, k, v, nullptr, n_rows, first_pos, stream);
+    if (rc) return rc;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_prefill_attn(ctx->dev, q, k, v, out_bf16, out_f32, n_rows, (cudaStream_t)stream));
+}
+
+int adsa_rope_2d(adsa_ctx *ctx, void *x, const int32_t *pos, long long n_rows, float base, adsa_stream_t stream)
+{
+    if (!ctx || !x || !pos || n_rows < 0 || !(base >= 0.f) || ((uintptr_t)x & 3u)) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    if (ctx->cfg.head_dim % 4 != 0) return ADSA_EINVAL;
+    if (n_rows == 0) return ADSA_OK;
+    ++ctx->launches;
+    return cuda_fail(ctx, launch_rope_2d(ctx->dev, x, pos, n_rows, base > 0.f ? base : 10000.f, (cudaStream_t)stream));
+}
+
 int adsa_set_stream_rows(adsa_ctx *ctx, int layer, int b, int h, const void *k, const void *v, const int32_t *pos,
                          int n_rows, adsa_stream_t stream)
 {

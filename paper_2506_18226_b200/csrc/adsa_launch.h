@@ -86,6 +86,11 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
                          int next_layer, int next_tiles, int n_run = 1);
 cudaError_t configure_wstep_kernel(const DevCtx &c);
 
+// Entering the condition: dense causal attention over n_rows rows per stream of a layer, and the 2-D rotary embedding.
+cudaError_t launch_prefill_attn(const DevCtx &c, const void *q, const void *k, const void *v, void *out_bf16, float *out_f32,
+                                int n_rows, cudaStream_t st);
+cudaError_t launch_rope_2d(const DevCtx &c, void *x, const int32_t *pos, long long n_rows, float base, cudaStream_t st);
+
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t configure_kernels(const DevCtx &c);
 cudaError_t configure_select_kernel(const DevCtx &c);
