@@ -91,14 +91,14 @@ def peaks():
     return 6650.0, "fallback"
 
 
-def dram_traffic(kind, workload, page_rows, launch):
+def dram_traffic(kind, workload, page_rows, launch, capacity_rows):
     """DRAM bytes (read + written) per layer-step from the ncu captures summarised under profiles/, or None
     when no capture matches the kernel configuration that was timed."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     try:
         with open(path) as f:
             for e in json.load(f)["entries"]:
-                if (e["kind"], e["workload"], e["page_rows"], e["launch"]) == (kind, workload, page_rows, launch):
+                if (e["kind"], e["workload"], e["page_rows"], e["launch"], e["capacity_rows"]) == (kind, workload, page_rows, launch, capacity_rows):
                     return e["dram_bytes_per_layer_step"]
     except (OSError, KeyError, ValueError):
         pass
@@ -418,7 +418,7 @@ def measure(w, args, dev, rank, world, local_rank, K, W, detail=True):
         res["roofline"] = _roofline("fused", f"fused layer-step (adsa_token_step, {launch_kind}: {per_launch} layer-step(s) per launch)",
                                     step_bytes, us_unit, per_launch, n_timed,
                                     dram_traffic("fused", args.workload if w.name.startswith(args.workload) else w.name[:4],
-                                                 st.page_rows, launch_kind))
+                                                 st.page_rows, launch_kind, C))
     if detail and rank == 0 and T0 + HW > C:
         res["detail"].update(full_cache_detail(st, args, M, step_bytes, attn_bytes))
     return res
@@ -447,7 +447,7 @@ def full_cache_detail(st, args, M, step_bytes, attn_bytes):
     launches = eng.launch_count() - n0
     out["roofline_layer_launch"] = _roofline("fused", "fused layer-step, one launch per layer (adsa_layer_step)", step_bytes,
                                              e0.elapsed_time(e1) * 1e3 / launches, 1, launches,
-                                             dram_traffic("fused", wname, st.page_rows, "layer-launch"))
+                                             dram_traffic("fused", wname, st.page_rows, "layer-launch", C))
     eng.set_token_launch(args.token_launch)
     # (2) the four calls
     st.load_late(HW - M)
@@ -476,7 +476,7 @@ def full_cache_detail(st, args, M, step_bytes, attn_bytes):
             call_us[name].append(ev[j].elapsed_time(ev[j + 1]) * 1e3 / L)
     assert eng.get_status()[0] == 0
     out["roofline_attn"] = _roofline("attn", "attention alone (adsa_sparse_decode_attn)", attn_bytes, attn_ms * 1e3 / (M * L), 1,
-                                     M * L, dram_traffic("attn", wname, st.page_rows, "layer-launch"))
+                                     M * L, dram_traffic("attn", wname, st.page_rows, "layer-launch", C))
     per_call = {n: float(np.median(v)) for n, v in call_us.items()}
     per_call["four_call_sequence"] = float(sum(per_call.values()))
     out["per_call_us_cache_full"] = per_call
