@@ -242,7 +242,9 @@ ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int bud
  * inputs are given at once, no layer has to wait for another: when the tensor-core
  * kernel serves the configuration and every layer is between steps, ONE launch walks
  * the streams of all layers (adsa_set_token_launch); otherwise the layers are
- * launched one after the other.  Results are those of adsa_layer_step layer by layer. */
+ * launched one after the other.  Results are those of adsa_layer_step layer by layer, up to the order in
+ * which partial sums are merged (it depends on how many warps share a stream, which the two ways may choose
+ * differently). */
 ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 

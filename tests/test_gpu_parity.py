@@ -248,6 +248,89 @@ def test_full_size_steps_that_change_the_code_path(cfg, pages, mode):
     assert _pages_in_use(eng) == S * -(-C // pr)
 
 
+@pytest.mark.parametrize("cfg,beta,n_layers,n_sample", [(4, 0.5, 4, 6), (3, 0.5, 6, 6), (5, 0.5, 2, 3)])
+def test_full_size_token_step_one_launch_for_all_layers(cfg, beta, n_layers, n_sample):
+    """adsa_token_step as the benchmark runs it: ONE launch of the tensor-core kernel for all layers (the
+    grouping the benchmark's launch uses: two warps per stream, as many streams per SM as fit), at the full
+    per-layer size of configs 3-5 with the benchmark's page size, from a seeded late state, over steps that
+    include the end of a grid row and the start of the next.  The oracle follows a sample of streams of every
+    layer: outputs, cache positions and payloads; and the same steps launched layer by layer agree to rounding
+    and leave the same caches."""
+    H = _harness()
+    from oracle import adsa_oracle as orc
+    from adsa_workloads import bf16_bits_to_f32, f32_to_bf16_bits
+    from dataclasses import replace
+    w = replace(get_workload(cfg, beta), n_layers=n_layers)
+    C, T0, W, S, d = w.capacity(), w.n_text, w.grid_w, w.streams_per_layer, w.head_dim
+    pr = _bench_page_rows(C)
+    g0 = (w.grid_h - 2) * W + W - 3                      # three cells before a row ends: cells W-3, W-2, W-1, then 0, 1
+    steps = 5
+    rng = np.random.default_rng(cfg)
+    sample = [sorted(rng.choice(S, size=n_sample, replace=False).tolist()) for _ in range(n_layers)]
+    engs = [H.engine_for(w, n_layers=n_layers, capacity=C, page_rows=pr) for _ in range(2)]
+    engs[1].set_token_launch(0)                          # the same steps, one launch per layer
+    ost = orc.OracleStreams(n_layers * n_sample, d, C + 4, T0, W, T0)
+    for l in range(n_layers):
+        pos, k, v = late_state(w, seed=100 * cfg + l, n_rows=C, cur_pos=T0 + g0)
+        for e in engs:
+            e.prefill_rows(l, H.dev_bf16(k.reshape(w.batch, w.n_heads, C, d)), H.dev_bf16(v.reshape(w.batch, w.n_heads, C, d)), 0,
+                           torch.from_numpy(pos.reshape(w.batch, w.n_heads, C)).to("cuda:0"))
+        for i, s_ in enumerate(sample[l]):
+            ost.load(l * n_sample + i, pos[s_], bf16_bits_to_f32(k[s_]), bf16_bits_to_f32(v[s_]))
+    shape = (n_layers, w.batch, w.n_heads, d)
+    outs = [torch.zeros(shape, dtype=torch.bfloat16, device="cuda:0") for _ in range(2)]
+    alive = np.ones(n_layers * n_sample, dtype=bool)     # streams still in step with the oracle (a tolerated tie ends a stream's comparison)
+    for t in range(steps):
+        per = [layer_step_qkv(w, 7, l, g0 + t) for l in range(n_layers)]
+        bits = [np.stack([x[i] for x in per]).reshape(shape) for i in range(3)]
+        dev = [H.dev_bf16(b) for b in bits]
+        before = engs[0].launch_count()
+        for e, o in zip(engs, outs):
+            e.token_step(T0 + g0 + t, C, dev[0], dev[1], dev[2], o)
+        if t > 0:
+            assert engs[0].launch_count() - before == 1          # scores are carried in: one launch for the whole stack
+        # (the two ways may give a stream a different number of warps, so partial sums merge in another order)
+        assert (outs[0].float() - outs[1].float()).abs().max().item() <= 4e-3, f"step {t}: one launch and per-layer launches differ"
+        pick = lambda b: np.concatenate([bf16_bits_to_f32(b).reshape(n_layers, S, d)[l, sample[l]] for l in range(n_layers)])
+        res = ost.step(pick(bits[0]), pick(bits[1]), pick(bits[2]), T0 + g0 + t, C)
+        got = outs[0].float().cpu().numpy().reshape(n_layers, S, d)
+        n_live = engs[0]._t["n_live"].cpu().numpy()
+        pos_now = engs[0]._t["pos"].cpu().numpy()
+        for l in range(n_layers):
+            for i, s_ in enumerate(sample[l]):
+                j = l * n_sample + i
+                if not alive[j]:
+                    continue
+                sid = l * S + s_
+                g_pos = set(pos_now[sid, :n_live[sid]].tolist())
+                o_pos = set(ost.rows(j)[0].tolist())
+                if g_pos != o_pos:                           # only a near-tie at the selection threshold may differ
+                    sc = dict(zip(res.cand_pos[j].tolist(), res.cand_score[j].tolist()))
+                    theta = max(sc[p_] for p_ in res.kept_pos[j].tolist() if p_ in sc)
+                    assert len(g_pos) == len(o_pos) and all(abs(sc[p_] - theta) <= 1e-6 for p_ in g_pos ^ o_pos), (t, l, s_)
+                    alive[j] = False
+                    continue
+                assert np.abs(got[l, s_] - res.out[j]).max() <= 2e-2, (t, l, s_)
+    assert alive.sum() >= alive.size - 2
+    for e in engs:
+        assert e.get_status()[0] == 0
+        assert (e._t["n_live"].cpu().numpy() == C).all()
+    same = np.sort(engs[0]._t["pos"].cpu().numpy(), axis=1) == np.sort(engs[1]._t["pos"].cpu().numpy(), axis=1)
+    assert same.all(axis=1).mean() >= 0.999              # (a near-tie may fall the other way with another summation order)
+    # payloads of the sampled streams, bit for bit
+    for l in range(n_layers):
+        for i, s_ in enumerate(sample[l]):
+            j = l * n_sample + i
+            if not alive[j]:
+                continue
+            pos, k, v = engs[0].read_stream(l * S + s_)
+            opos, ok, ov = ost.rows(j)
+            og, oo = np.argsort(pos.numpy()), np.argsort(opos)
+            assert np.array_equal(pos.numpy()[og], opos[oo])
+            assert np.array_equal(k.numpy().view(np.uint16)[og], f32_to_bf16_bits(ok)[oo])
+            assert np.array_equal(v.numpy().view(np.uint16)[og], f32_to_bf16_bits(ov)[oo])
+
+
 # ---------------------------------------------------------------------------
 # selection under structure: clusters, exact ties, equal and zero rows, any K
 # ---------------------------------------------------------------------------
