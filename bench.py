@@ -69,6 +69,7 @@ def parse_args(argv=None):
     ap.add_argument("--sweep-mode", type=int, default=2,
                     help="adsa_set_single_sweep: 0 two sweeps, 1 single sweep, 2 single sweep + carried evictee")
     ap.add_argument("--token-launch", type=int, default=1, help="adsa_set_token_launch: 1 one launch per token, 0 one launch per layer")
+    ap.add_argument("--host-chunks", type=int, default=0, help="adsa_set_host_chunks (0 = the library's default)")
     ap.add_argument("--next-tiles", type=int, default=-1, help="adsa_set_next_layer_hint (-1 = the library's default)")
     ap.add_argument("--ring-stages", type=int, default=0, help="cap on the persistent kernel's ring (0 = as many as fit)")
     ap.add_argument("--profiler-range", action="store_true",
@@ -202,6 +203,8 @@ class Stack:
         eng.set_staged(args.kernel_mode)
         eng.set_single_sweep(args.sweep_mode)
         eng.set_token_launch(args.token_launch)
+        if args.host_chunks:
+            eng.set_host_chunks(args.host_chunks)
         if args.next_tiles >= 0:
             eng.set_next_layer_hint(args.next_tiles)
         if args.ring_stages:

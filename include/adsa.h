@@ -249,8 +249,8 @@ ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const 
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 
 /* adsa_token_step with HOST tensors of the same shapes (pinned memory, or the
- * copies do not overlap anything).  Inputs and outputs travel in up to six
- * chunks of layers on two copy streams that the context creates on its first
+ * copies do not overlap anything).  Inputs and outputs travel in chunks of
+ * layers (four by default, adsa_set_host_chunks) on two copy streams that the context creates on its first
  * call here, so that later layers' inputs and earlier layers' outputs cross the
  * bus while the layers in between compute; the kernels run on `stream`.  When
  * the call returns every layer has run and the outputs are on the host.  Uses
@@ -299,6 +299,10 @@ ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
  * tiles per warp beyond the ring (0 = none, -1 = choose automatically, the default).  Results do not
  * depend on it. */
 ADSA_API int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles);
+
+/* adsa_token_step_host: in how many chunks of layers the tensors travel (2 .. 6; 0 = the default).  The first
+ * chunk is always a single layer, so that computing starts after a short copy. */
+ADSA_API int adsa_set_host_chunks(adsa_ctx *ctx, int chunks);
 
 /* adsa_token_step: 1 (default) = one launch serves every layer when it can, 0 = one launch per layer
  * (what a decoder whose layers feed each other has to do, through adsa_layer_step). */

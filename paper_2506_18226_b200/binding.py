@@ -21,7 +21,7 @@ DEV_POOL_EXHAUSTED, DEV_BAD_POSITION, DEV_ROW_OVERFLOW, DEV_RING_TIMEOUT, DEV_BA
 EXPORTS = [
     "adsa_workspace_bytes", "adsa_create", "adsa_destroy", "adsa_reset", "adsa_prefill_rows",
     "adsa_set_stream_rows", "adsa_prefill_attn", "adsa_rope_2d", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
-    "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_stream_warps", "adsa_set_single_sweep",
+    "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_host_chunks", "adsa_set_stream_warps", "adsa_set_single_sweep",
     "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror", "adsa_decode_attn_static",
 ]
 
@@ -78,6 +78,7 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_set_l2_lookahead": [vp, i32],
             "adsa_set_next_layer_hint": [vp, i32],
             "adsa_set_token_launch": [vp, i32],
+            "adsa_set_host_chunks": [vp, i32],
             "adsa_set_stream_warps": [vp, i32],
             "adsa_set_single_sweep": [vp, i32],
             "adsa_layer_rows_bound": [vp, i32, C.POINTER(i32)],
@@ -284,6 +285,9 @@ class AdsaEngine:
 
     def set_l2_lookahead(self, tiles):
         self._call("adsa_set_l2_lookahead", int(tiles))
+
+    def set_host_chunks(self, chunks):
+        self._call("adsa_set_host_chunks", int(chunks))
 
     def set_token_launch(self, mode):
         """token_step: 1 one launch for every layer (default), 0 one launch per layer."""
