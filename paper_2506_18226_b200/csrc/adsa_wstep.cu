@@ -75,6 +75,8 @@ namespace adsa {
 //   RS = 104, TR = 16   208-byte rows (head_dim 97 .. 104) written as they lie: a pitch of 208 bytes puts the eight
 //                       rows of an ldmatrix on eight different bank groups without any swizzle; a stage is half a
 //                       block (6.5 KB instead of 13 KB), so that shared memory still holds rings for ten warps.
+//   RS = 128, TR = 16   256-byte rows as two 128-byte halves, each a swizzled tile of its own (elements 0-63 of
+//                       every row, then elements 64-127), written by two tensor copies per pool; 8 KB per stage.
 // Rows are always dealt to the warps of a group in 32-row blocks (one word of every row mask).
 constexpr int kWTile = 32;                        // rows per block
 constexpr int kWMaxDepth = 8;                     // stages per warp
@@ -206,7 +208,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     constexpr int KS = (RS + 15) / 16;                 // 16-element steps over a row: k-steps of S = K.q and of the score product, M blocks of O^T
     constexpr int NJ = w_sets(RS);                     // a lane holds elements 64*j + 2*lane, + 1 of a row, j < NJ
     constexpr int NH = kWTile / TR, MB = TR / 16;      // stages per 32-row block, 16-row MMA blocks per stage
-    constexpr bool SWZ = RS == 64;                     // tiles written with the 128-byte swizzle
+    constexpr bool SWZ = RS % 64 == 0;                 // tiles written with the 128-byte swizzle, one sub-tile per 64 elements of a row
+    constexpr int NSEG = SWZ ? RS / 64 : 1;            // sub-tiles of a K (or V) tile
+    constexpr int PITCH = SWZ ? 128 : kWRowBytes;      // bytes from row to row inside a sub-tile
+    constexpr int SEGB = TR * 128;                     // bytes of a swizzled sub-tile
     constexpr bool RAGGED = RS % 16 != 0;              // the last 16-element step has only its first 8 elements
     constexpr int kWPart = w_part_floats(RS);
     extern __shared__ __align__(1024) unsigned char smem_all[];
@@ -258,20 +263,23 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     // Swizzled tiles: the rows a lane uses are (multiple of 8) + lr, so the swizzle term is (chunk ^ lr) << 4 and the
     // address is a per-lane base xor (b << 5).  Plain tiles: base + 32*b.  When the row ends in the middle of the last
     // step, the lanes whose chunk lies beyond it read 16 zero bytes instead.
-    const uint32_t v_off = SWZ ? (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + (((mi >> 1) ^ lr) << 4))
-                               : (uint32_t)((8 * (mi & 1) + lr) * kWRowBytes + ((mi >> 1) << 4));
-    const uint32_t vt_off = SWZ ? (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + (((mi & 1) ^ lr) << 4))
-                                : (uint32_t)((8 * (mi >> 1) + lr) * kWRowBytes + ((mi & 1) << 4));
+    const uint32_t v_off = SWZ ? (uint32_t)((8 * (mi & 1) + lr) * PITCH + (((mi >> 1) ^ lr) << 4))
+                               : (uint32_t)((8 * (mi & 1) + lr) * PITCH + ((mi >> 1) << 4));
+    const uint32_t vt_off = SWZ ? (uint32_t)((8 * (mi >> 1) + lr) * PITCH + (((mi & 1) ^ lr) << 4))
+                                : (uint32_t)((8 * (mi >> 1) + lr) * PITCH + ((mi & 1) << 4));
+    // (swizzled tiles: step b lies in sub-tile b / 4, at chunks 2 * (b % 4), + 1 of its 128-byte rows)
     auto a_addr = [&](uint32_t tile, int blk, int b) -> uint32_t {
         if (RAGGED && b == KS - 1 && (mi >> 1)) return zero_u32;
-        return tile + blk * 16 * kWRowBytes + (SWZ ? (v_off ^ (uint32_t)(b << 5)) : v_off + (uint32_t)(b << 5));
+        return tile + blk * 16 * PITCH + (SWZ ? (uint32_t)((b >> 2) * SEGB) + (v_off ^ (uint32_t)((b & 3) << 5)) : v_off + (uint32_t)(b << 5));
     };
     auto t_addr = [&](uint32_t tile, int blk, int b) -> uint32_t {
         if (RAGGED && b == KS - 1 && (mi & 1)) return zero_u32;
-        return tile + blk * 16 * kWRowBytes + (SWZ ? (vt_off ^ (uint32_t)(b << 5)) : vt_off + (uint32_t)(b << 5));
+        return tile + blk * 16 * PITCH + (SWZ ? (uint32_t)((b >> 2) * SEGB) + (vt_off ^ (uint32_t)((b & 3) << 5)) : vt_off + (uint32_t)(b << 5));
     };
     // byte offset of 16-byte chunk ch of row r inside a tile
-    auto chunk_off = [&](int r, int ch) -> uint32_t { return SWZ ? swz(r, ch) : (uint32_t)(r * kWRowBytes + (ch << 4)); };
+    auto chunk_off = [&](int r, int ch) -> uint32_t {
+        return SWZ ? (uint32_t)((ch >> 3) * SEGB) + swz(r, ch & 7) : (uint32_t)(r * kWRowBytes + (ch << 4));
+    };
     // one L2 hint per 128-byte line of a pool row
     auto hint_row = [&](const __nv_bfloat16 *row) {
 #pragma unroll
@@ -515,21 +523,27 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 // the common case: a whole tile inside one page is one box per pool; lane 0 copies K, lane 1 copies V
                 constexpr int kBox = TR == 32 ? 5 : 4;
                 const int y = pt_s[pg0] * c.page_rows + in0;
-                if (lane == 1 || (lane == 0 && pass == 0))
-                    tma_2d(lane ? vdst : kdst, lane ? &maps.v[kBox] : &maps.k[kBox], 0, y, bar);
+                if (lane == 1 || (lane == 0 && pass == 0)) {
+#pragma unroll
+                    for (int sg = 0; sg < NSEG; ++sg)
+                        tma_2d((lane ? vdst : kdst) + sg * SEGB, lane ? &maps.v[kBox] : &maps.k[kBox], 64 * sg, y, bar);
+                }
             } else if (lane == 0) {
                 int r = r0, pg = pg0, in = in0;
                 while (r < r1) {   // page pieces, each cut into boxes of 32, 16, 8, 4, 2 or 1 rows
                     int cnt = min(r1 - r, c.page_rows - in);
                     int y = pt_s[pg] * c.page_rows + in;
-                    uint32_t off = (uint32_t)(r - r0) * kWRowBytes;
+                    uint32_t off = (uint32_t)(r - r0) * PITCH;
                     r += cnt; in = 0; ++pg;
                     while (cnt > 0) {
                         int hb = 31 - __clz(cnt);
                         hb = hb > 5 ? 5 : hb;
-                        if (pass == 0) tma_2d(kdst + off, &maps.k[hb], 0, y, bar);
-                        tma_2d(vdst + off, &maps.v[hb], 0, y, bar);
-                        y += 1 << hb; off += (uint32_t)kWRowBytes << hb; cnt -= 1 << hb;
+#pragma unroll
+                        for (int sg = 0; sg < NSEG; ++sg) {
+                            if (pass == 0) tma_2d(kdst + sg * SEGB + off, &maps.k[hb], 64 * sg, y, bar);
+                            tma_2d(vdst + sg * SEGB + off, &maps.v[hb], 64 * sg, y, bar);
+                        }
+                        y += 1 << hb; off += (uint32_t)PITCH << hb; cnt -= 1 << hb;
                     }
                 }
             }
@@ -537,12 +551,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // Rows of a partial tile that the copy does not write must hold finite numbers (their weights
         // are zero, and 0 * NaN would not be): all lanes clear them before the tile is requested.
         auto clear_tail = [&](int u) {
-            constexpr int kChunks = kWRowBytes / 16;
+            constexpr int kChunks = PITCH / 16;      // 16-byte chunks of a row inside a sub-tile (the swizzle moves chunks within their row only)
             const int r0 = stage_row0(u);
             const int rows = max(0, min(n - r0, TR));
             if (rows < TR) {
                 uint4 *z = reinterpret_cast<uint4 *>(ring + i_stage * kWStageBytes);
-                for (int i = rows * kChunks + lane; i < TR * kChunks; i += 32) { z[i] = make_uint4(0u, 0u, 0u, 0u); z[kWTileBytes / 16 + i] = make_uint4(0u, 0u, 0u, 0u); }
+#pragma unroll
+                for (int sg = 0; sg < NSEG; ++sg)
+                    for (int i = rows * kChunks + lane; i < TR * kChunks; i += 32) {
+                        z[sg * (TR * kChunks) + i] = make_uint4(0u, 0u, 0u, 0u);
+                        z[kWTileBytes / 16 + sg * (TR * kChunks) + i] = make_uint4(0u, 0u, 0u, 0u);
+                    }
             }
         };
         // HBM is otherwise idle until the attention sweep starts (the ring holds `depth` stages and the
@@ -1335,8 +1354,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 }
 
 // ---- host side ------------------------------------------------------------
-// Row layouts the kernel is compiled for: 64-element rows (32-row stages) and 104-element rows (16-row stages).
-bool wstep_supported(const DevCtx &c) { return (c.row_stride == 64 || c.row_stride == 104) && c.d % 2 == 0; }
+// Row layouts the kernel is compiled for: 64-element rows (32-row stages), 104- and 128-element rows (16-row stages).
+bool wstep_supported(const DevCtx &c) { return (c.row_stride == 64 || c.row_stride == 104 || c.row_stride == 128) && c.d % 2 == 0; }
 static int wstep_stage_rows(const DevCtx &c) { return c.row_stride == 64 ? 32 : 16; }
 
 // Tensor maps of both pools for boxes of 1, 2, 4, .. 32 rows (128-byte swizzle for 128-byte rows, none
@@ -1360,11 +1379,11 @@ int build_wstep_maps(const DevCtx &c, WStepMaps *out)
     const cuuint32_t estr[2] = {1, 1};
     for (int pool = 0; pool < 2; ++pool) {
         for (int hb = 0; hb < 6; ++hb) {
-            const cuuint32_t box[2] = {(cuuint32_t)c.row_stride, 1u << hb};
+            const cuuint32_t box[2] = {(cuuint32_t)(c.row_stride == 104 ? 104 : 64), 1u << hb};   // swizzled tiles: 64 elements (128 bytes) wide
             CUtensorMap *m = pool == 0 ? &out->k[hb] : &out->v[hb];
             CUresult r = encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pool == 0 ? (void *)c.k_pool : (void *)c.v_pool,
                                 dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                c.row_stride == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                                c.row_stride == 104 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return -1;
         }
@@ -1386,6 +1405,10 @@ static wstep_fn wstep_variant(int row_stride, int warps, bool fused)
     if (row_stride == 104) {
         if (warps <= 8) return fused ? wstep_kernel<true, 8, 104, 16> : wstep_kernel<false, 8, 104, 16>;
         if (warps <= kWWideMaxWarps) return fused ? wstep_kernel<true, kWWideMaxWarps, 104, 16> : wstep_kernel<false, kWWideMaxWarps, 104, 16>;
+    }
+    if (row_stride == 128) {
+        if (warps <= 8) return fused ? wstep_kernel<true, 8, 128, 16> : wstep_kernel<false, 8, 128, 16>;
+        if (warps <= kWWideMaxWarps && !fused) return wstep_kernel<false, kWWideMaxWarps, 128, 16>;   // the fused step would spill at ten warps
     }
     return nullptr;
 }
@@ -1409,7 +1432,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
     WStepPlan p = {};
     if (!wstep_supported(c)) return p;
     const int rs = c.row_stride, tr = wstep_stage_rows(c), stage_bytes = w_stage_bytes(rs, tr);
-    const int max_warps = rs == 64 ? 16 : kWWideMaxWarps;   // the wide-row kernel needs more registers per thread
+    const int max_warps = rs == 64 ? 16 : (rs == 128 && fused) ? 8 : kWWideMaxWarps;   // the wide-row kernels need more registers per thread
     const int n_streams = c.S * (n_run < 1 ? 1 : n_run);   // streams one launch serves
     int groups = (n_streams + sm_count - 1) / sm_count;
     groups = groups < 1 ? 1 : groups > kScratchGroups ? kScratchGroups : groups;

@@ -72,6 +72,9 @@ def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=N
     (32, 3, 4, 4, 6, 0.6, 32),     # 4 lanes per row
     (100, 5, 9, 5, 7, 0.5, 0),     # non-power-of-two head_dim, padded row stride 104
     (128, 11, 6, 4, 4, 0.7, 0),    # 16 lanes per row
+    (128, 16, 40, 7, 6, 0.6, 0),   # 256-byte rows over several blocks, pages of exactly one 16-row stage
+    (128, 13, 45, 6, 7, 0.5, 0),   # 256-byte rows, pages that cut every stage into pieces
+    (122, 64, 33, 6, 6, 0.5, 0),   # head_dim just below 128: the padding of a 128-element row stays out of every sum
     (256, 4, 3, 3, 5, 0.5, 0),     # 32 lanes per row
     (8, 2, 2, 7, 3, 0.4, 0),       # smallest head_dim
 ])
@@ -248,7 +251,32 @@ def test_full_size_steps_that_change_the_code_path(cfg, pages, mode):
     assert _pages_in_use(eng) == S * -(-C // pr)
 
 
-@pytest.mark.parametrize("cfg,beta,n_layers,n_sample", [(4, 0.5, 4, 6), (3, 0.5, 6, 6), (5, 0.5, 2, 3)])
+def _wide_workload():
+    """Heads of 128 elements (the 256-byte row layout) on a 24 x 24 grid with enough streams that every SM
+    serves several of them."""
+    return Workload("wide-d128-24x24", 41, 3, 8, 32, 128, 120, 24, 24, 0.5, 1.0)
+
+
+@pytest.mark.parametrize("pages", ["bench", "paged"])
+@pytest.mark.parametrize("mode", ["calls", "fused", "two-sweep-fused", "cluster-fused"])
+def test_wide_rows_many_streams(pages, mode):
+    """128-element heads at a size that fills the device: the cache fills up on the last cell of a grid
+    row, the next row starts, the budget drops (general selection, survivors move) and is lifted again."""
+    w = _wide_workload()
+    C, W, T0 = w.capacity(), w.grid_w, w.n_text
+    pr = _bench_page_rows(C) if pages == "bench" else pick_page_rows(C, hi=64)
+    g0 = (w.grid_h - 3) * W + W - 3
+    eng, lh = _full_size_harness(w, C, pr, mode, 24, 411, C - 2, T0 + g0)
+    budgets = [C, C, C, C, C, C - 21, C - 21, C, C]
+    for t, budget in enumerate(budgets):
+        q, kn, vn = layer_step_qkv(w, 4, 0, g0 + t)
+        lh.step(q, kn, vn, T0 + g0 + t, budget)
+    assert (eng._t["n_live"].cpu().numpy() == C - 19).all()
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+    assert _pages_in_use(eng) == w.streams_per_layer * -(-(C - 19) // pr)
+
+
+@pytest.mark.parametrize("cfg,beta,n_layers,n_sample", [(4, 0.5, 4, 6), (3, 0.5, 6, 6), (5, 0.5, 2, 3), ("wide", 0.5, 4, 6)])
 def test_full_size_token_step_one_launch_for_all_layers(cfg, beta, n_layers, n_sample):
     """adsa_token_step as the benchmark runs it: ONE launch of the tensor-core kernel for all layers (the
     grouping the benchmark's launch uses: two warps per stream, as many streams per SM as fit), at the full
@@ -260,7 +288,8 @@ def test_full_size_token_step_one_launch_for_all_layers(cfg, beta, n_layers, n_s
     from oracle import adsa_oracle as orc
     from adsa_workloads import bf16_bits_to_f32, f32_to_bf16_bits
     from dataclasses import replace
-    w = replace(get_workload(cfg, beta), n_layers=n_layers)
+    w = replace(_wide_workload() if cfg == "wide" else get_workload(cfg, beta), n_layers=n_layers)
+    cfg = 6 if cfg == "wide" else cfg
     C, T0, W, S, d = w.capacity(), w.n_text, w.grid_w, w.streams_per_layer, w.head_dim
     pr = _bench_page_rows(C)
     g0 = (w.grid_h - 2) * W + W - 3                      # three cells before a row ends: cells W-3, W-2, W-1, then 0, 1
