@@ -92,13 +92,27 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def kernel_source_digest():
+    """SHA-256 over the sources of the timed kernel: counters taken from another version of them are not reported."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("adsa_wstep.cu", "adsa_dev.cuh", "adsa_select.cuh", "adsa_async.cuh"):
+        with open(os.path.join(ROOT, "paper_2506_18226_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def dram_traffic(kind, workload, page_rows, launch, capacity_rows):
     """DRAM bytes (read + written) per layer-step from the ncu captures summarised under profiles/, or None
-    when no capture matches the kernel configuration that was timed."""
+    when no capture matches the kernel configuration that was timed, or the kernel's sources have changed
+    since the captures were taken."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     try:
         with open(path) as f:
-            for e in json.load(f)["entries"]:
+            rec = json.load(f)
+            if rec.get("kernel_source_sha256") != kernel_source_digest():
+                return None
+            for e in rec["entries"]:
                 if (e["kind"], e["workload"], e["page_rows"], e["launch"], e["capacity_rows"]) == (kind, workload, page_rows, launch, capacity_rows):
                     return e["dram_bytes_per_layer_step"]
     except (OSError, KeyError, ValueError):
