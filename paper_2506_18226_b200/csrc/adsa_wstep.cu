@@ -214,6 +214,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     constexpr int SEGB = TR * 128;                     // bytes of a swizzled sub-tile
     constexpr bool RAGGED = RS % 16 != 0;              // the last 16-element step has only its first 8 elements
     constexpr int kWPart = w_part_floats(RS);
+    constexpr bool SPLIT = KS > 4;                     // two accumulation chains per K.q and V.s product
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = a.group_warps, D = a.depth;
@@ -512,6 +513,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     const __nv_bfloat16 *pool = lane ? c.v_pool : c.k_pool;
                     const uint32_t dst = lane ? vdst : kdst;
                     int r = r0, pg = pg0, in = in0;
+                    if (r1 > r0 && in0 + (r1 - r0) <= c.page_rows) {   // the common case: the stage lies inside one page
+                        bulk_g2s(dst, pool + ((size_t)pt_s[pg0] * c.page_rows + in0) * (size_t)RS, (uint32_t)(r1 - r0) * kWRowBytes, bar);
+                        r = r1;
+                    }
                     while (r < r1) {
                         const int cnt = min(r1 - r, c.page_rows - in);
                         bulk_g2s(dst + (uint32_t)(r - r0) * kWRowBytes, pool + ((size_t)pt_s[pg] * c.page_rows + in) * (size_t)RS,
@@ -567,9 +572,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // HBM is otherwise idle until the attention sweep starts (the ring holds `depth` stages and the
         // selection comes first), so the rows of the blocks after those are asked into L2 now, and one
         // block further with every block consumed: the sweep then finds them in L2.
-        auto l2_ask = [&](int u) {   // this warp's u-th block, a row per lane
-            const int row = (rk + u * G) * kWTile + lane;
-            if (u < mt && row < n) {
+        auto l2_ask = [&](int u) {   // this warp's u-th block: one hint per pool if a single page holds it, else a row per lane
+            const int b0 = (rk + u * G) * kWTile, row = b0 + lane;
+            if (u >= mt) return;
+            const int rows = min(n - b0, kWTile);
+            const int pg0 = (int)__umulhi((uint32_t)b0, c.pr_magic), in0 = b0 - pg0 * c.page_rows;
+            if (in0 + rows <= c.page_rows) {
+                if (lane < 2) {
+                    const __nv_bfloat16 *src = (lane ? c.v_pool : c.k_pool) + ((size_t)pt_s[pg0] * c.page_rows + in0) * (size_t)RS;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * kWRowBytes) : "memory");
+                }
+            } else if (row < n) {
                 const size_t off = c.max_pages == 1 ? ((size_t)pt_s[0] * c.page_rows + row) * (size_t)c.row_stride
                                                     : row_offset(c, pt_s, row);
                 hint_row(c.k_pool + off);
@@ -655,63 +668,61 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         auto score_mma = [&](uint32_t vb, float (&dt)[MB][4]) {
 #pragma unroll
             for (int mbk = 0; mbk < MB; ++mbk) {
+                float dt2[4];   // the odd k-steps: two short chains of MMAs instead of one long one
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     uint32_t af[4];
                     ldsm_x4(a_addr(vb, mbk, ks), af);
                     if (ks == 0) mma_bf16_z(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                    else if (SPLIT && ks == 1) mma_bf16_z(dt2, af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                    else if (SPLIT && (ks & 1)) mma_bf16(dt2, af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
                     else mma_bf16(dt[mbk], af[0], af[1], af[2], af[3], sb0[ks], sb1[ks]);
+                }
+                if (SPLIT) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dt[mbk][i] += dt2[i];
                 }
             }
         };
         // r0: the stream row of the tile's first row; cw: bit i = row r0 + i is to be scored
+        float *const scores_g = c.scores + (size_t)sid * c.max_rows;
         auto score_write = [&](const float (&dt)[MB][4], const unsigned char *vtile, int r0, uint32_t cw) {
-            float *scores = c.scores + (size_t)sid * c.max_rows;
-            int32_t *holes = reinterpret_cast<int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
-            // rows 16*mbk + 8*hh + g: columns 0, 1 of the product sit in lane t = 0, column 2 in t = 1
-            float sval[2 * MB], invv[2 * MB], dotv[2 * MB];
-            bool want[2 * MB];
-            const uint32_t cwg = t == 0 ? cw >> g : 0u;
+            // Rows 16*mbk + 8*hh + g of the product: columns 0, 1 sit in lane t = 0 of the row's group of four, column 2
+            // in lane t = 1 (whose second column is zero).  The three parts are added up across the pair and the sums
+            // are then handed round so that lane i holds row i of the stage: one row per lane from here on.
+            float dot = 0.f;
 #pragma unroll
-            for (int i = 0; i < 2 * MB; ++i) {
-                const int mbk = i >> 1, hh = i & 1;
-                const float lo = __shfl_down_sync(0xffffffffu, dt[mbk][2 * hh], 1);
-                const int row = r0 + 16 * mbk + 8 * hh + g;
-                want[i] = (cwg >> (16 * mbk + 8 * hh)) & 1u;
-                invv[i] = inv_s[row];   // past the last live row this reads whatever follows in shared memory: never wanted
-                dotv[i] = (dt[mbk][2 * hh] + dt[mbk][2 * hh + 1]) + lo;
-                sval[i] = (invv[i] * dotv[i] - 1.0f) * rden + 0.0f;
+            for (int mbk = 0; mbk < MB; ++mbk) {
+                float a = dt[mbk][0] + dt[mbk][1], b = dt[mbk][2] + dt[mbk][3];
+                a += __shfl_xor_sync(0xffffffffu, a, 1);
+                b += __shfl_xor_sync(0xffffffffu, b, 1);
+                const float va = __shfl_sync(0xffffffffu, a, 4 * (lane & 7)), vb = __shfl_sync(0xffffffffu, b, 4 * (lane & 7));
+                if (MB == 1 || (lane >> 4) == mbk) dot = (lane & 8) ? vb : va;
             }
+            const int row = r0 + lane;
+            if (!(lane < TR && ((cw >> lane) & 1u))) return;
+            const float inv = inv_s[row];
             // warp_rare (set when the row weights were made): one of this warp's scored rows has a clamped
             // norm, or rows move down in the update; otherwise every row is written where it stands
-            if (!warp_rare) {
-#pragma unroll
-                for (int i = 0; i < 2 * MB; ++i)
-                    if (want[i]) scores[r0 + 16 * (i >> 1) + 8 * (i & 1) + g] = sval[i];
-            } else {
-#pragma unroll
-                for (int i = 0; i < 2 * MB; ++i) {
-                    if (!want[i]) continue;
-                    const int mbk = i >> 1, hh = i & 1, row = r0 + 16 * mbk + 8 * hh + g;
-                    float s_out = sval[i];
-                    if (invv[i] >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
-                        float ss = 0.f;
-                        for (int ch = 0; ch < RS / 8; ++ch) {
-                            float f[8];
-                            unpack8(*reinterpret_cast<const uint4 *>(vtile + chunk_off(row - r0, ch)), f);
-                            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-                        }
-                        s_out = (invv[i] * dotv[i] - invv[i] * invv[i] * ss) * rden + 0.0f;
-                    }
-                    int dst = row;
-                    if (row >= n2) {   // a survivor: it moves into the hole of the same rank
-                        int lo_i = 0, hi_i = list_ns - 1;
-                        while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
-                        dst = holes[lo_i];
-                    }
-                    scores[dst] = s_out;
+            if (!warp_rare) { scores_g[row] = (inv * dot - 1.0f) * rden + 0.0f; return; }
+            float s_out = (inv * dot - 1.0f) * rden + 0.0f;
+            if (inv >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
+                float ss = 0.f;
+                for (int ch = 0; ch < RS / 8; ++ch) {
+                    float f[8];
+                    unpack8(*reinterpret_cast<const uint4 *>(vtile + chunk_off(lane, ch)), f);
+                    for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
                 }
+                s_out = (inv * dot - inv * inv * ss) * rden + 0.0f;
             }
+            int dst = row;
+            if (row >= n2) {   // a survivor: it moves into the hole of the same rank
+                const int32_t *holes = reinterpret_cast<const int32_t *>(sm_keys), *surv = holes + c.max_rows + 1;
+                int lo_i = 0, hi_i = list_ns - 1;
+                while (lo_i < hi_i) { int mid = (lo_i + hi_i) >> 1; if (surv[mid] < row) lo_i = mid + 1; else hi_i = mid; }
+                dst = holes[lo_i];
+            }
+            scores_g[dst] = s_out;
         };
 
         // ---- which rows are attended, and the weights of the rows the next step scores -------------
@@ -1049,16 +1060,21 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const uint32_t kw = (kmask[tl] >> (part_i * TR)) >> g;   // bits 0, 8 (, 16, 24): rows g, g + 8 (, g + 16, g + 24) of the stage are retained
             // S = K.q: A = 16 rows of K, B = q in every column, so every lane of a group of four holds the
             // logits of rows 16*mb + g (c0 = c1) and 16*mb + g + 8 (c2 = c3)
+            // (wide rows: even and odd k-steps accumulate apart, so that a product is two short chains of MMAs instead of one long one)
             float sc[MB][4];
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
+                float sc2[4];
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     uint32_t kf[4];
                     ldsm_x4(a_addr(kb, mb, ks), kf);
                     if (ks == 0) mma_bf16_z(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
+                    else if (SPLIT && ks == 1) mma_bf16_z(sc2, kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
+                    else if (SPLIT && (ks & 1)) mma_bf16(sc2, kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                     else mma_bf16(sc[mb], kf[0], kf[1], kf[2], kf[3], qa0[ks], qa2[ks]);
                 }
+                if (SPLIT) { sc[mb][0] += sc2[0]; sc[mb][2] += sc2[2]; }   // (columns 1 and 3 repeat 0 and 2)
             }
             peek_next(part_i + 1 < NH || tl + G < n_tiles || (FUSED && !single));
             float dts[MB][4];   // the score products of this tile, started before the softmax arithmetic
@@ -1075,12 +1091,16 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     mx = fmaxf(mx, x[mb][h]);
                 }
             }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-            const float m_new = fmaxf(m_run, mx);
-            const float corr = ex2(m_run - m_new);
-            m_run = m_new;
+            // the running maximum moves in few tiles of a stream: a vote tells whether the reduction over lanes is needed
+            float m_new = m_run, corr = 1.0f;
+            if (__any_sync(0xffffffffu, mx > m_run)) {
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                m_new = fmaxf(m_run, mx);
+                corr = ex2(m_run - m_new);
+                m_run = m_new;
+            }
             float psum = 0.f;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
@@ -1110,32 +1130,30 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 pb0[ks] = g == 0 ? h0 : g == 1 ? l0 : g <= 4 ? w0 : 0u;
                 pb2[ks] = g == 0 ? h2 : g == 1 ? l2 : g <= 4 ? w2 : 0u;
             }
-            // O^T_tile = V^T.B' from zero (A = V^T through transposing ldmatrix), then folded into the running sums
-            float ot[KS][4];
+            // The running sums follow the running maximum (roles 0, 1 carry softmax weights; the weight sums of the other
+            // roles are not rescaled).  The maximum is the same in every lane and moves in few tiles of a stream.
+            if (corr != 1.0f) {
+                const float corr_role = t == 0 ? corr : 1.0f;
 #pragma unroll
-            for (int md = 0; md < KS; ++md) {
-                uint32_t vf[4];
-                ldsm_x4_t(t_addr(vb, 0, md), vf);
-                mma_bf16_z(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[0], pb2[0]);
+                for (int md = 0; md < KS; ++md) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) o_run[md][i] *= corr_role;
+                }
             }
-            if constexpr (MB == 2) {
+            // O^T += V^T.B' (A = V^T through transposing ldmatrix), accumulated in the running sums themselves
+#pragma unroll
+            for (int mbk = 0; mbk < MB; ++mbk) {
 #pragma unroll
                 for (int md = 0; md < KS; ++md) {
                     uint32_t vf[4];
-                    ldsm_x4_t(t_addr(vb, 1, md), vf);
-                    mma_bf16(ot[md], vf[0], vf[1], vf[2], vf[3], pb0[MB - 1], pb2[MB - 1]);
+                    ldsm_x4_t(t_addr(vb, mbk, md), vf);
+                    mma_bf16(o_run[md], vf[0], vf[1], vf[2], vf[3], pb0[mbk], pb2[mbk]);
                 }
             }
             if constexpr (FUSED) {
                 if (single) score_write(dts, ring + stage * kWStageBytes + kWTileBytes, r0, n2 <= c.max_rows ? cmask[tl] >> (part_i * TR) : 0u);
             }
             release_and_refill();
-            const float corr_role = t == 0 ? corr : 1.0f;     // roles 0, 1 carry softmax weights; the weight sums are not rescaled
-#pragma unroll
-            for (int md = 0; md < KS; ++md) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) o_run[md][i] = fmaf(o_run[md][i], corr_role, ot[md][i]);
-            }
           }
         }
 
