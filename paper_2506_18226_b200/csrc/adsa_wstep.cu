@@ -606,6 +606,17 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         if constexpr (FUSED) {
             for (int u = (D + NH - 1) / NH; u < (D + NH - 1) / NH + a.l2_ahead; ++u) l2_ask(u);
         }
+        // The row the previous step named as this step's evictee (its note, when this step is a steady one with a
+        // full cache): its V row is asked for now, behind the first tiles.
+        const int carried_slot = try_fast && n == a.budget_rows && note.x == 1 && note.y >= 1 && note.w >= 1 && note.w <= n ? note.w - 1 : -1;
+        uint32_t ve[NJ];
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) ve[j] = 0u;
+        if (carried_slot >= 0) {
+            const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, carried_slot));
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
+        }
         // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
         // (the reads are complete once their results have been used, which in-order issue guarantees
         // for this thread and __syncwarp for the others; a fence is needed only after the generic-proxy
@@ -686,6 +697,15 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         };
         // r0: the stream row of the tile's first row; cw: bit i = row r0 + i is to be scored
         float *const scores_g = c.scores + (size_t)sid * c.max_rows;
+        // the highest score this lane has written, the slot it went to, and whether another of its rows had the same
+        // score: the next step's evictee if that step keeps all but one of these rows (Eq. 3 with K = p - 1)
+        float top_s = -INFINITY;
+        int top_slot = -1;
+        bool top_tie = false;
+        auto note_top = [&](float s_out, int dst) {
+            if (s_out > top_s) { top_s = s_out; top_slot = dst; top_tie = false; }
+            else if (s_out == top_s) top_tie = true;
+        };
         auto score_write = [&](const float (&dt)[MB][4], const unsigned char *vtile, int r0, uint32_t cw) {
             // Rows 16*mbk + 8*hh + g of the product: columns 0, 1 sit in lane t = 0 of the row's group of four, column 2
             // in lane t = 1 (whose second column is zero).  The three parts are added up across the pair and the sums
@@ -704,7 +724,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const float inv = inv_s[row];
             // warp_rare (set when the row weights were made): one of this warp's scored rows has a clamped
             // norm, or rows move down in the update; otherwise every row is written where it stands
-            if (!warp_rare) { scores_g[row] = (inv * dot - 1.0f) * rden + 0.0f; return; }
+            if (!warp_rare) {
+                const float s_out = (inv * dot - 1.0f) * rden + 0.0f;
+                scores_g[row] = s_out;
+                note_top(s_out, row);
+                return;
+            }
             float s_out = (inv * dot - 1.0f) * rden + 0.0f;
             if (inv >= 1.0f / kNormEps) {   // |v| was clamped: u.u is not 1, take it from the row
                 float ss = 0.f;
@@ -723,6 +748,18 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 dst = holes[lo_i];
             }
             scores_g[dst] = s_out;
+            note_top(s_out, dst);
+        };
+        // this warp's highest written score into its partial state: {score, slot or -1 if two rows share it}
+        auto publish_top = [&](float *w, int at) {
+            float v = top_s;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+            const bool mine = top_slot >= 0 && top_s == v;
+            const unsigned who = __ballot_sync(0xffffffffu, mine);
+            const bool tie = __any_sync(0xffffffffu, mine && top_tie) || __popc(who) > 1;
+            const int wslot = who ? __shfl_sync(0xffffffffu, top_slot, __ffs(who) - 1) : -1;
+            if (lane == 0) { w[at] = v; reinterpret_cast<int *>(w)[at + 1] = tie ? -1 : wslot; }
         };
 
         // ---- which rows are attended, and the weights of the rows the next step scores -------------
@@ -740,7 +777,11 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         // s' = s - u_e.  The sum of normalised rows is not summed again: s' is carried on (it is summed afresh
         // whenever the long way runs, at least once per grid row).
         bool fast = false;
-        if (try_fast && n == a.budget_rows && note.x == 1 && note.y >= 1) {   // the same decision in every warp of the group
+        if (carried_slot >= 0) {
+            // the previous step has named the row: the highest of the scores it wrote (one row alone had it)
+            fast = true;
+            evict_slot = carried_slot;
+        } else if (try_fast && n == a.budget_rows && note.x == 1 && note.y >= 1) {   // the same decision in every warp of the group
             const float *sc_g = c.scores + (size_t)sid * c.max_rows;
             float best = -INFINITY;
             int best_slot = -1;
@@ -788,8 +829,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             rden = p_next > 1 ? 1.0f / (float)(p_next - 1) : 0.0f;
             warp_clamped = (note.z & 1) != 0;   // known for the stream as a whole
             warp_rare = warp_clamped;
-            uint32_t ve[NJ];
-            {
+            if (carried_slot < 0) {
                 const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot));
 #pragma unroll
                 for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
@@ -1199,6 +1239,9 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 if (t == 1) { w[kSum + x0] = (o_run[md][0] + o_run[md][1]) + lo0; w[kSum + x1] = (o_run[md][2] + o_run[md][3]) + lo2; }
             }
             if (lane == 0) { w[kML] = m_run; w[kML + 1] = l_run; reinterpret_cast<int *>(w)[kML + 2] = warp_clamped ? 1 : 0; }
+            if constexpr (FUSED) {
+                if (single) publish_top(w, kML + 3);
+            }
         }
         group_sync();
         float sv0[NJ], sv1[NJ];   // s[64*j + 2*lane], s[64*j + 2*lane + 1]
@@ -1293,6 +1336,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                         release_and_refill();
                     }
                 }
+                publish_top(part + rk * kWPart, kML + 3);
             }
             // every warp's copies of this stream have landed before rows move or pages are freed (after a single
             // sweep the group has met since its last copy landed: at the merge of the partial states)
@@ -1317,8 +1361,18 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (rk == 0 && lane == 0) {
                 int clamped = 0;
                 for (int w = 0; w < G; ++w) clamped |= reinterpret_cast<const int *>(part + w * kWPart)[kML + 2];
+                // the highest of the scores just written and its slot (the new row's own score is not among them)
+                float gbest = -INFINITY;
+                int gslot = -1;
+                for (int w = 0; w < G; ++w) {
+                    const float wv = part[w * kWPart + kML + 3];
+                    const int ws = reinterpret_cast<const int *>(part + w * kWPart)[kML + 4];
+                    if (wv > gbest) { gbest = wv; gslot = ws; }
+                    else if (wv == gbest && wv > -INFINITY) gslot = -1;
+                }
+                if (new_cand) gslot = -1;
                 // rows that moved were scored at their new slots, but the mask above is by old slot: no note then
-                *reinterpret_cast<int4 *>(c.carry + (size_t)sid * 4) = make_int4(okay && ns == 0 ? 1 : 0, p_next, clamped, 0);
+                *reinterpret_cast<int4 *>(c.carry + (size_t)sid * 4) = make_int4(okay && ns == 0 ? 1 : 0, p_next, clamped, gslot + 1);
             }
 
             // ---- the update itself, by the first warp ---------------------------------------------------
