@@ -520,8 +520,9 @@ def end_to_end(st, args, K, W, world, prompts):
     per = int(np.prod(st.shape)) * 2
     return {"value": tokens / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 3 * per, "d2h_bytes_per_step": per,
             "steps": Ke, "ms_per_step": ms / Ke, "regions": len(regions),
-            "api": "adsa_token_step_host (pinned host q/k/v in, host output out, copies in chunks of layers under the "
-                   "compute, one sync per token)"}
+            "api": "adsa_token_step_host (q/k/v from pinned host memory by copy-engine copies in chunks of layers, queued beside "
+                   "ONE launch for all layers that waits for each layer's inputs to land; the output rows are written "
+                   "by the kernel into pinned host memory; one sync per token, wall clock around the calls)"}
 
 
 def compact(res):

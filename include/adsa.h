@@ -248,13 +248,18 @@ ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int bud
 ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 
-/* adsa_token_step with HOST tensors of the same shapes (pinned memory, or the
- * copies do not overlap anything).  Inputs and outputs travel in chunks of
- * layers (four by default, adsa_set_host_chunks) on two copy streams that the context creates on its first
- * call here, so that later layers' inputs and earlier layers' outputs cross the
- * bus while the layers in between compute; the kernels run on `stream`.  When
- * the call returns every layer has run and the outputs are on the host.  Uses
- * the staging part of the workspace; results are those of adsa_token_step. */
+/* adsa_token_step with HOST tensors of the same shapes.  The inputs cross the bus in chunks of layers on a copy
+ * stream that the context creates on its first call here, while earlier layers compute on `stream`:
+ *   - inputs in pinned host memory, and one launch of the tensor-core kernel can serve the whole stack (see
+ *     adsa_token_step): that launch is queued at once; every chunk of copies is followed by a small copy that marks
+ *     its layers as landed, and the kernel waits for a layer's mark (bounded: after a second or two it sets the
+ *     device status ADSA_DEV_COPY_TIMEOUT and reads what is there) before it reads that layer's q, k_new, v_new;
+ *   - otherwise, or after adsa_set_host_chunks(2 .. 6): every chunk of layers is a launch of its own, queued
+ *     behind its copies (pageable memory works here, but its copies overlap nothing).
+ * An output buffer in pinned, mapped host memory (cudaHostAlloc, cudaHostRegister) is written by the kernels
+ * directly; any other host buffer is filled by copies from a staging buffer.  When the call returns every layer
+ * has run and the outputs are on the host.  Uses the staging part of the workspace; results are those of
+ * adsa_token_step. */
 ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host,
                                   const void *k_new_host, const void *v_new_host, void *out_host,
                                   adsa_stream_t stream);
@@ -300,8 +305,9 @@ ADSA_API int adsa_set_ring_stages(adsa_ctx *ctx, int max_stages);
  * depend on it. */
 ADSA_API int adsa_set_l2_lookahead(adsa_ctx *ctx, int tiles);
 
-/* adsa_token_step_host: in how many chunks of layers the tensors travel (2 .. 6; 0 = the default).  The first
- * chunk is always a single layer, so that computing starts after a short copy. */
+/* adsa_token_step_host: 0 (default): one launch that waits for its inputs layer by layer when that is possible,
+ * else one launch per chunk with chunks that grow threefold from a single layer.  2 .. 6: always one launch per
+ * chunk: one layer, then chunks - 1 equal chunks. */
 ADSA_API int adsa_set_host_chunks(adsa_ctx *ctx, int chunks);
 
 /* adsa_token_step: 1 (default) = one launch serves every layer when it can, 0 = one launch per layer

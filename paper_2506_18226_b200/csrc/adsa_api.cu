@@ -31,7 +31,7 @@ struct LayerState {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, wscratch, logit, ml, status, staging, total;
+    size_t scores, keep_mask, counts, partials, tickets, svec, carry, cand_mask, wscratch, logit, ml, status, in_flags, staging, total;
 };
 
 int mask_words_of(const adsa_config &cfg) { return (cfg.max_rows_per_stream + 31) / 32; }
@@ -53,6 +53,7 @@ WorkspaceLayout layout_of(const adsa_config &cfg)
     w.logit = off;       off = align_up(off + (cfg.score_mode == 1 ? S * (size_t)cfg.n_layers * R * sizeof(float) : 0), 256);
     w.ml = off;          off = align_up(off + (cfg.score_mode == 1 ? S * (size_t)cfg.n_layers * 4 * sizeof(float) : 0), 256);
     w.status = off;      off = align_up(off + 4 * sizeof(uint32_t), 256);
+    w.in_flags = off;    off = align_up(off + (size_t)cfg.n_layers * sizeof(int32_t), 256);
     w.staging = off;     off = align_up(off + 4 * S * (size_t)cfg.n_layers * cfg.head_dim * sizeof(__nv_bfloat16), 256);
     w.total = off;
     return w;
@@ -118,6 +119,9 @@ struct adsa_ctx {
     // adsa_token_step_host moves its tensors in chunks of layers on two copy streams of its own, so that the
     // copies of later layers travel while earlier layers compute (created on first use, host-side objects only)
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    int *in_flags = nullptr;      // [n_layers] device words: adsa_token_step_host's inputs of a layer have landed
+    int *epoch_src = nullptr;     // [n_layers] pinned host words holding the current call's number, the source of those words
+    int host_epoch = 0;
     cudaEvent_t ev_start = nullptr;
     std::vector<cudaEvent_t> ev_in, ev_done;
 };
@@ -330,6 +334,7 @@ int adsa_create(const adsa_config *cfg, const adsa_buffers *buf, adsa_ctx **out)
     d.scale_log2e = scale * 1.4426950408889634f;
     size_t stage = (size_t)d.S * cfg->n_layers * cfg->head_dim;
     ctx->stage_q = (__nv_bfloat16 *)(w + ws.staging);
+    ctx->in_flags = (int *)(w + ws.in_flags);
     ctx->stage_k = ctx->stage_q + stage;
     ctx->stage_v = ctx->stage_k + stage;
     ctx->stage_o = ctx->stage_v + stage;
@@ -358,6 +363,7 @@ int adsa_destroy(adsa_ctx *ctx)
         for (cudaEvent_t e : ctx->ev_done) cudaEventDestroy(e);
         if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
         if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+        if (ctx->epoch_src) cudaFreeHost(ctx->epoch_src);
         if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     }
     delete ctx;
@@ -599,8 +605,27 @@ int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int budget_rows,
 }
 
 // One step of layers l0 .. l0 + NL - 1 (q, k_new, v_new, out_bf16 point at layer l0's tensors).
+// One launch for layers l0 .. l0 + NL - 1: the tensor-core kernel serves the configuration, every layer is between
+// steps and all are in the same carried state.
+static bool one_launch_possible(const adsa_ctx *ctx, int l0, int NL, int cur_pos, WStepPlan *plan)
+{
+    bool ok = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok &&
+              ctx->cfg.score_mode == 0 && ctx->cfg.score_share == 0;
+    const LayerState &L0 = ctx->layers[l0];
+    for (int l = 0; l < NL && ok; ++l) {
+        const LayerState &L = ctx->layers[l0 + l];
+        ok = L.phase == kIdle && (L.scores_pos == cur_pos) == (L0.scores_pos == cur_pos) && (L.svec_pos == cur_pos) == (L0.svec_pos == cur_pos);
+    }
+    if (!ok) return false;
+    WStepPlan wp = plan_wstep(ctx->dev, true, ctx->sm_count, ctx->max_stages, ctx->stream_warps, NL);
+    if (ctx->l2_ahead >= 0) wp.l2_ahead = ctx->l2_ahead;
+    if (plan) *plan = wp;
+    return wp.n_groups > 0;
+}
+
+// in_ready (optional, one launch only): per-layer words that say when a layer's inputs have landed (WStepArgs::in_ready)
 static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_rows, const void *q, const void *k_new,
-                       const void *v_new, void *out_bf16, adsa_stream_t stream)
+                       const void *v_new, void *out_bf16, adsa_stream_t stream, const int *in_ready = nullptr, int in_epoch = 0)
 {
     size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q, *kb = (const __nv_bfloat16 *)k_new,
@@ -612,23 +637,10 @@ static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_ro
     // The warps of a multiprocessor then sit in different phases of different streams (locating rows,
     // sweeping, updating) instead of all starting and all draining together once per layer.  Taken when
     // every layer is between steps and in the same carried state; otherwise layer by layer.
-    bool one_launch = ctx->token_launch == 1 && NL > 1 && (ctx->kernel_mode == 1 || ctx->kernel_mode == 4) && ctx->mma_ok &&
-                      ctx->cfg.score_mode == 0 && ctx->cfg.score_share == 0;
-    if (one_launch) {
-        const LayerState &L0 = ctx->layers[l0];
-        for (int l = 0; l < NL && one_launch; ++l) {
-            const LayerState &L = ctx->layers[l0 + l];
-            one_launch = L.phase == kIdle && (L.scores_pos == cur_pos) == (L0.scores_pos == cur_pos) &&
-                         (L.svec_pos == cur_pos) == (L0.svec_pos == cur_pos);
-        }
-    }
     WStepPlan wp = {};
-    if (one_launch) {
-        wp = plan_wstep(ctx->dev, true, ctx->sm_count, ctx->max_stages, ctx->stream_warps, NL);
-        if (ctx->l2_ahead >= 0) wp.l2_ahead = ctx->l2_ahead;
-        one_launch = wp.n_groups > 0;
-    }
+    const bool one_launch = one_launch_possible(ctx, l0, NL, cur_pos, &wp);
     if (!one_launch) {
+        if (in_ready) return ADSA_ESTATE;   // (the caller has checked: not reached)
         for (int l = 0; l < NL; ++l) {
             int rc = adsa_layer_step(ctx, l0 + l, cur_pos, budget_rows, qb + l * per_layer, kb + l * per_layer,
                                      vb + l * per_layer, ob + l * per_layer, stream);
@@ -667,7 +679,7 @@ static int step_layers(adsa_ctx *ctx, int l0, int NL, int cur_pos, int budget_ro
     const bool have_svec = ctx->layers[l0].svec_pos == cur_pos;
     ++ctx->launches;
     int rc = cuda_fail(ctx, launch_wstep(ctx->dev, wp, ctx->maps, true, l0, cur_pos, budget_rows, q, k_new, v_new, out_bf16, nullptr,
-                                         st, have_svec && ctx->sweep_mode >= 1, false, ctx->sweep_mode >= 2, -1, ctx->next_tiles, NL));
+                                         st, have_svec && ctx->sweep_mode >= 1, false, ctx->sweep_mode >= 2, -1, ctx->next_tiles, NL, in_ready, in_epoch));
     for (int l = 0; l < NL; ++l) {
         LayerState &L = ctx->layers[l0 + l];
         L.rows_hi = after[l];
@@ -699,19 +711,39 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
     if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     const int L = ctx->cfg.n_layers;
-    // chunk boundaries: a first chunk of one layer, so that computing starts after a short copy, then up to five
-    // equal ones (three by default: every chunk is one launch, and larger launches run closer to the copy rate)
+    // Chunk boundaries.  Every chunk is one launch, and larger launches run closer to the copy rate, so chunks are few;
+    // the first is one layer, so that computing starts after a short copy.  By default each chunk is about three
+    // times the one before it: a layer's inputs cross PCIe in about a quarter of the time the layer computes, so a
+    // chunk's copy ends while the chunk before it still runs.  adsa_set_host_chunks(n >= 2): one layer, then n - 1
+    // equal chunks.
     int bound[7], n_chunks = 0;
     bound[0] = 0;
     if (L <= 6) {
         for (int l = 1; l <= L; ++l) bound[l] = l;
         n_chunks = L;
-    } else {
+    } else if (ctx->host_chunks >= 2 && ctx->host_chunks <= 6) {
         bound[1] = 1;
-        const int parts = ctx->host_chunks >= 2 && ctx->host_chunks <= 6 ? ctx->host_chunks - 1 : 3;   // measured on the XL shape, image-tokens/s end to end: 2 chunks 17 943, 3: 19 235, 4: 19 633, 6: 18 303
-        const int rest = L - 1, per = (rest + parts - 1) / parts;
+        const int parts = ctx->host_chunks - 1, rest = L - 1, per = (rest + parts - 1) / parts;
         n_chunks = 1;
         for (int l = 1; l < L; l += per) { bound[n_chunks + 1] = l + per < L ? l + per : L; ++n_chunks; }
+    } else {
+        int size = 1, l = 0;
+        while (l < L) {
+            const int take = n_chunks == 5 || l + size + size / 2 >= L ? L - l : size;   // no small last chunk, six chunks at most
+            l += take;
+            bound[++n_chunks] = l;
+            size *= 3;
+        }
+    }
+    // An output buffer in pinned, mapped host memory is written by the kernels themselves (posted writes of whole
+    // rows); any other host memory gets its chunks by copies from a staging buffer.
+    __nv_bfloat16 *out_direct = nullptr;
+    {
+        cudaPointerAttributes attr = {};
+        if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+            out_direct = (__nv_bfloat16 *)attr.devicePointer;
+        else
+            cudaGetLastError();
     }
     cudaError_t e = cudaSuccess;
     if (!ctx->copy_in) {   // first use on this context
@@ -730,6 +762,61 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
     const size_t per_layer = (size_t)ctx->dev.S * ctx->cfg.head_dim;   // elements
     const char *qh = (const char *)q_host, *kh = (const char *)k_new_host, *vh = (const char *)v_new_host;
     char *oh = (char *)out_host;
+
+    // ---- one launch for the whole stack, started before its inputs are there ---------------------------------
+    // When the tensor-core kernel can take every layer in one launch and the inputs sit in pinned host memory, the
+    // launch is queued at once and the copies run beside it on the inbound stream, in small chunks of layers, each
+    // followed by a copy that writes this call's number into the chunk's per-layer words; the kernel waits for a
+    // layer's word (for a bounded time) before it reads that layer's q, k_new and v_new.  The copies are queued on
+    // their own stream and wait for nothing the kernel does, so they always proceed.
+    auto pinned = [](const void *p) {
+        cudaPointerAttributes attr = {};
+        if (cudaPointerGetAttributes(&attr, p) == cudaSuccess && attr.type == cudaMemoryTypeHost) return true;
+        cudaGetLastError();
+        return false;
+    };
+    if (ctx->host_chunks == 0 && L > 1 && pinned(q_host) && pinned(k_new_host) && pinned(v_new_host) &&
+        one_launch_possible(ctx, 0, L, cur_pos, nullptr)) {
+        if (!ctx->epoch_src) {
+            e = cudaHostAlloc((void **)&ctx->epoch_src, (size_t)L * sizeof(int), cudaHostAllocDefault);
+            if (e == cudaSuccess) e = cudaMemsetAsync(ctx->in_flags, 0, (size_t)L * sizeof(int), ctx->copy_in);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->copy_in);
+            if (e != cudaSuccess) { ctx->epoch_src = nullptr; return cuda_fail(ctx, e); }
+            ctx->host_epoch = 0;
+        }
+        const int epoch = ++ctx->host_epoch;   // (the previous call has drained its streams: the source words are free)
+        for (int l = 0; l < L; ++l) ctx->epoch_src[l] = epoch;
+        auto copy_layers = [&](int l0, int l1) -> cudaError_t {
+            const size_t off = (size_t)l0 * per_layer, bytes = (size_t)(l1 - l0) * per_layer * sizeof(__nv_bfloat16);
+            cudaError_t r = cudaMemcpyAsync(ctx->stage_q + off, qh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+            if (r == cudaSuccess) r = cudaMemcpyAsync(ctx->stage_k + off, kh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+            if (r == cudaSuccess) r = cudaMemcpyAsync(ctx->stage_v + off, vh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+            if (r == cudaSuccess)   // after the data, in stream order: the words that release these layers
+                r = cudaMemcpyAsync(ctx->in_flags + l0, ctx->epoch_src + l0, (size_t)(l1 - l0) * sizeof(int), cudaMemcpyHostToDevice, ctx->copy_in);
+            return r;
+        };
+        e = cudaEventRecord(ctx->ev_start, st);   // earlier work on the caller's stream may still read the staging buffers
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_in, ctx->ev_start, 0);
+        int done = 0, size = 1;
+        if (e == cudaSuccess) { e = copy_layers(0, 1); done = 1; }
+        int rc = ADSA_OK;
+        if (e == cudaSuccess)
+            rc = step_layers(ctx, 0, L, cur_pos, budget_rows, ctx->stage_q, ctx->stage_k, ctx->stage_v,
+                             out_direct ? out_direct : ctx->stage_o, stream, ctx->in_flags, epoch);
+        // The rest of the inputs, whatever the launch returned: a kernel that did start must find every word.
+        while (done < L && e == cudaSuccess) {
+            size *= 2;
+            const int take = done + size + size / 2 >= L ? L - done : size;
+            e = copy_layers(done, done + take);
+            done += take;
+        }
+        if (e == cudaSuccess && rc == ADSA_OK && !out_direct)
+            e = cudaMemcpyAsync(oh, ctx->stage_o, (size_t)L * per_layer * sizeof(__nv_bfloat16), cudaMemcpyDeviceToHost, st);
+        const cudaError_t s_in = cudaStreamSynchronize(ctx->copy_in), s_st = cudaStreamSynchronize(st);
+        if (rc != ADSA_OK) return rc;
+        if (e == cudaSuccess) e = s_in != cudaSuccess ? s_in : s_st;
+        return cuda_fail(ctx, e);
+    }
     auto copy_in_chunk = [&](int c) -> cudaError_t {   // inputs of chunk c, on the inbound copy stream
         const size_t off = (size_t)bound[c] * per_layer, bytes = (size_t)(bound[c + 1] - bound[c]) * per_layer * sizeof(__nv_bfloat16);
         cudaError_t r = cudaMemcpyAsync(ctx->stage_q + off, qh + off * 2, bytes, cudaMemcpyHostToDevice, ctx->copy_in);
@@ -750,11 +837,13 @@ int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void
         e = cudaStreamWaitEvent(st, ctx->ev_in[c], 0);
         if (e == cudaSuccess)   // the chunk's layers: one launch when the tensor-core kernel can take them together
             rc = step_layers(ctx, l0, l1 - l0, cur_pos, budget_rows, ctx->stage_q + l0 * per_layer, ctx->stage_k + l0 * per_layer,
-                             ctx->stage_v + l0 * per_layer, ctx->stage_o + l0 * per_layer, stream);
+                             ctx->stage_v + l0 * per_layer, (out_direct ? out_direct : ctx->stage_o) + l0 * per_layer, stream);
         if (e != cudaSuccess || rc != ADSA_OK) break;
-        e = cudaEventRecord(ctx->ev_done[c], st);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[c], 0);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(oh + off * 2, ctx->stage_o + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
+        if (!out_direct) {
+            e = cudaEventRecord(ctx->ev_done[c], st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[c], 0);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(oh + off * 2, ctx->stage_o + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
+        }
         if (e == cudaSuccess && c + 2 < n_chunks) e = copy_in_chunk(c + 2);
     }
     // One way out, whatever happened: nothing of this call may still be running on the private streams, or

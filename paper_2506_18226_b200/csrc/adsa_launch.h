@@ -83,7 +83,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                          float *out_f32, cudaStream_t st, bool have_svec, bool early_state, bool use_note,
-                         int next_layer, int next_tiles, int n_run = 1);
+                         int next_layer, int next_tiles, int n_run = 1, const int *in_ready = nullptr, int in_epoch = 0);
 cudaError_t configure_wstep_kernel(const DevCtx &c);
 
 // Entering the condition: dense causal attention over n_rows rows per stream of a layer, and the 2-D rotary embedding.

@@ -191,6 +191,8 @@ struct WStepArgs {
     __nv_bfloat16 *out_bf16;
     float *out_f32;
     unsigned long long *scratch; // [grid][n_groups][2 * max_rows + 4] words of 8 bytes: keys, compaction lists
+    const int *in_ready;         // null, or one word per layer of the context: layer l's q, k_new and v_new have landed (a copy
+    int in_epoch;                // engine is still writing them when the launch starts) once in_ready[l] - in_epoch >= 0
 };
 
 struct WSelPartial {      // what one warp of a group found in its share of the rows (32 bytes)
@@ -363,6 +365,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     };
     if (!a.early_state) dep_wait();
     int spin_limit = kCopySpinLimit;
+    int in_spin = kInputSpinLimit;   // polls of the inputs-have-landed word before giving up
     auto wait = [&](uint32_t bar, uint32_t parity) {
         if (!mbar_wait_sleepy(bar, parity, spin_limit)) {
             if (lane == 0) set_status(c, ADSA_DEV_COPY_TIMEOUT);
@@ -414,20 +417,35 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 #pragma unroll
         for (int j = 0; j < NJ; ++j) { qn[j] = 0u; kn[j] = 0u; vn[j] = 0u; }
         auto load_inputs = [&]() {
+            if (a.in_ready) {
+                // The caller's tensors may still be on their way (copies queued on another stream before this launch):
+                // wait, for a bounded time, for the word that the copy after them writes.  The loads below bypass L1.
+                const int *flag = a.in_ready + a.layer + local / c.S;
+                int v = 0;
+                for (int it = 0; it < in_spin; ++it) {
+                    asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                    if (v - a.in_epoch >= 0) break;
+                    __nanosleep(200);
+                }
+                if (v - a.in_epoch < 0) {   // gave up: flag it, read what is there, and do not wait as long again
+                    if (lane == 0) set_status(c, ADSA_DEV_COPY_TIMEOUT);
+                    in_spin = kCopySpinAfterTimeout;
+                }
+            }
             const uint32_t *q2 = reinterpret_cast<const uint32_t *>(a.q + (size_t)local * c.d);   // c.d is even
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 int e0 = 16 * ks + 2 * t, e1 = e0 + 8;
-                qa0[ks] = e0 < c.d ? q2[e0 >> 1] : 0u;
-                qa2[ks] = e1 < c.d ? q2[e1 >> 1] : 0u;
+                qa0[ks] = e0 < c.d ? __ldcg(q2 + (e0 >> 1)) : 0u;
+                qa2[ks] = e1 < c.d ? __ldcg(q2 + (e1 >> 1)) : 0u;
             }
             if (rk == 0) {
 #pragma unroll
                 for (int j = 0; j < NJ; ++j) {
                     if (64 * j + 2 * lane < c.d) {
-                        qn[j] = q2[32 * j + lane];
-                        kn[j] = reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d)[32 * j + lane];
-                        vn[j] = reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d)[32 * j + lane];
+                        qn[j] = __ldcg(q2 + 32 * j + lane);
+                        kn[j] = __ldcg(reinterpret_cast<const uint32_t *>(a.k_new + (size_t)local * c.d) + 32 * j + lane);
+                        vn[j] = __ldcg(reinterpret_cast<const uint32_t *>(a.v_new + (size_t)local * c.d) + 32 * j + lane);
                     }
                 }
             }
@@ -1546,9 +1564,10 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps &maps, bool fused, int layer, int cur_pos,
                          int budget_rows, const void *q, const void *k_new, const void *v_new, void *out_bf16,
                          float *out_f32, cudaStream_t st, bool have_svec, bool early_state, bool use_note, int next_layer, int next_tiles,
-                         int n_run)
+                         int n_run, const int *in_ready, int in_epoch)
 {
     WStepArgs a;
+    a.in_ready = in_ready; a.in_epoch = in_epoch;
     a.n_run = n_run < 1 ? 1 : n_run;
     a.next_layer = next_layer; a.next_tiles = next_tiles;
     a.have_svec = have_svec ? 1 : 0;

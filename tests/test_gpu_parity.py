@@ -655,10 +655,11 @@ def test_interleaved_layers_keep_their_own_selection():
     assert np.array_equal(np.sort(eng._t["pos"].cpu().numpy(), axis=1), np.sort(ref._t["pos"].cpu().numpy(), axis=1))
 
 
-@pytest.mark.parametrize("n_layers", [1, 4, 8])
-def test_token_step_host_matches_device_call(n_layers):
-    """adsa_token_step_host (inputs and outputs in pinned host memory, moved in chunks of layers while other
-    layers compute) gives bit for bit what adsa_token_step gives on device tensors, and leaves the same cache."""
+@pytest.mark.parametrize("n_layers,pinned_out,chunks", [(1, True, 0), (4, True, 0), (8, False, 0), (13, True, 0), (13, False, 3)])
+def test_token_step_host_matches_device_call(n_layers, pinned_out, chunks):
+    """adsa_token_step_host (inputs in pinned host memory, moved in chunks of layers while other layers compute;
+    the output either in pinned memory, which the kernels write themselves, or in pageable memory, which is
+    filled by copies) gives bit for bit what adsa_token_step gives on device tensors, and leaves the same cache."""
     H = _harness()
     w = Workload("host", 94, n_layers, 2, 2, 64, 16, 8, 7, 0.5, 1.0)
     C, L, T = w.capacity(), w.n_layers, w.n_cells
@@ -669,7 +670,10 @@ def test_token_step_host_matches_device_call(n_layers):
             e.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
     shape = (L, w.batch, w.n_heads, w.head_dim)
     out_d = torch.zeros(shape, dtype=torch.bfloat16, device="cuda:0")
-    out_h = torch.zeros(shape, dtype=torch.bfloat16).pin_memory()
+    out_h = torch.zeros(shape, dtype=torch.bfloat16)
+    if pinned_out:
+        out_h = out_h.pin_memory()
+    engs[1].set_host_chunks(chunks)
     for g in range(T):
         per = [layer_step_qkv(w, 6, l, g) for l in range(L)]
         bits = [np.stack([x[i] for x in per]).reshape(shape) for i in range(3)]
@@ -684,6 +688,41 @@ def test_token_step_host_matches_device_call(n_layers):
     assert torch.equal(engs[0]._t["n_live"].cpu(), engs[1]._t["n_live"].cpu())
     pos = [np.sort(e._t["pos"][:, :C].cpu().numpy(), axis=1) for e in engs]
     assert np.array_equal(pos[0], pos[1])
+
+
+def test_token_step_host_full_size_waits_for_its_inputs():
+    """At the per-layer size of config 4 with 12 layers, the inputs of the later layers are still crossing the bus
+    when the one launch that serves the whole stack is already running: it must wait for each layer's inputs.
+    Every step has new inputs and the staging buffers still hold the previous step's, so a layer read too early
+    shows up as a difference from the call on device tensors."""
+    H = _harness()
+    from dataclasses import replace
+    w = replace(get_workload(4), n_layers=12)
+    C, L, T0, d = w.capacity(), 12, w.n_text, w.head_dim
+    pr = _bench_page_rows(C)
+    g0 = w.n_cells - 6
+    engs = [H.engine_for(w, n_layers=L, capacity=C, page_rows=pr) for _ in range(2)]
+    for l in range(L):
+        pos, k, v = late_state(w, seed=300 + l, n_rows=C, cur_pos=T0 + g0)
+        for e in engs:
+            e.prefill_rows(l, H.dev_bf16(k.reshape(w.batch, w.n_heads, C, d)), H.dev_bf16(v.reshape(w.batch, w.n_heads, C, d)), 0,
+                           torch.from_numpy(pos.reshape(w.batch, w.n_heads, C)).to("cuda:0"))
+    shape = (L, w.batch, w.n_heads, d)
+    out_d = torch.zeros(shape, dtype=torch.bfloat16, device="cuda:0")
+    out_h = torch.zeros(shape, dtype=torch.bfloat16).pin_memory()
+    for t in range(6):
+        per = [layer_step_qkv(w, 8, l, g0 + t) for l in range(L)]
+        bits = [np.stack([x[i] for x in per]).reshape(shape) for i in range(3)]
+        dev = [H.dev_bf16(b) for b in bits]
+        host = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory() for b in bits]
+        engs[0].token_step(T0 + g0 + t, C, dev[0], dev[1], dev[2], out_d)
+        before = engs[1].launch_count()
+        engs[1].token_step_host(T0 + g0 + t, C, host[0], host[1], host[2], out_h)
+        if t > 0:
+            assert engs[1].launch_count() - before == 1
+        assert torch.equal(out_d.cpu(), out_h), f"step {t}"
+    for e in engs:
+        assert e.get_status()[0] == 0
 
 
 def test_error_paths_return_status_and_launch_nothing():
