@@ -134,6 +134,20 @@ def test_config1_full_trajectory(seed, mode):
     assert eng.pool_bytes_peak() <= w.streams_per_layer * -(-C // pr) * pr * w.row_stride * 4
 
 
+@pytest.mark.parametrize("setting,n_text,grid,budget", [
+    ("class-conditional", 1, 24, 384), ("class-conditional", 1, 24, 256),          # Sec. 5: context 576 cut to 384 and 256
+    ("text-conditional", 120, 32, 768), ("text-conditional", 120, 32, 640), ("text-conditional", 120, 32, 512),  # 1024 cut to 768, 640, 512
+])
+def test_context_budgets_of_the_experiments(setting, n_text, grid, budget):
+    """Whole generations at the context budgets of Sec. 5 (a class token or 120 text tokens, then a 24 x 24
+    or 32 x 32 grid), a few streams of 64-element heads, fused steps against the oracle at every step."""
+    w = Workload(setting, 70 + grid, 1, 1, 4, 64, n_text, grid, grid, budget / (n_text + grid * grid), 1.0)
+    lh, eng = _run_trajectory(w, 0, budget, lambda cur: budget, n_prefix=n_text, mode="fused")
+    assert lh.stats.steps == grid * grid
+    assert lh.stats.max_out_err <= 2e-2 and lh.mean_out_err() <= 2e-3
+    assert int(eng._t["n_live"].max().item()) == budget
+
+
 @pytest.mark.parametrize("mode", ["calls", "fused"])
 def test_config1_budget_as_fraction_of_current_context(mode):
     # the literal "50 % of the current context" schedule: budget grows with the context
