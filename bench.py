@@ -600,6 +600,17 @@ def run_ours(args, rank, world, local_rank):
             del r2
             torch.cuda.empty_cache()
         detail["all_configs"] = rows
+        # the headline workload once more with several pages per stream (the headline uses the largest divisor of the
+        # capacity up to 1024 rows, i.e. one page per stream where the capacity allows)
+        small = pick_page_rows(C, hi=64)
+        if small != res["kv_pool"]["page_rows"] and args.page_rows == 0:
+            a2 = copy.copy(args)
+            a2.page_rows, a2.profiler_range = small, False
+            r2 = measure(w, a2, dev, 0, 1, local_rank, min(20, w.n_cells), 5, detail=True)
+            r2["stack"] = None
+            detail["several_pages_per_stream"] = compact(r2)
+            del r2
+            torch.cuda.empty_cache()
     if not args.no_memory_sweep and world == 1:
         detail["memory_vs_batch"] = memory_vs_batch(args, dev)
 
