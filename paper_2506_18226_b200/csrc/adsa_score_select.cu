@@ -50,17 +50,39 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
     int cnt = 0;
-    for (int slot = warp * RPW + grp; slot < n; slot += kSSWarps * RPW) {   // no shuffles inside: lanes may leave early
-        int reg = region_of(c, pos[slot], cur_pos);
-        if (reg == kRegionInvalid && sub == 0) set_status(c, ADSA_DEV_BAD_POSITION);
-        if (reg != kRegionPrevious) continue;
-        if (sub == 0) ++cnt;
-        if (piece_ok) {
-            float f[8];
-            unpack8(ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8), f);
-            float inv = inv_norm[slot];
+    // U rows per lane group are requested before the first is used (positions, then rows and norms): a block holds
+    // U times as many bytes in flight; the rows are still added in ascending slot order.
+    constexpr int U = 4, kStep = kSSWarps * RPW;
+    for (int slot0 = warp * RPW + grp; slot0 < n; slot0 += U * kStep) {   // no shuffles inside: lanes may leave early
+        int ps[U];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = fmaf(inv, f[e], acc[e]);
+        for (int u = 0; u < U; ++u) ps[u] = slot0 + u * kStep < n ? pos[slot0 + u * kStep] : -1;
+        uint4 raw[U];
+        float inv[U];
+        bool prev[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int slot = slot0 + u * kStep;
+            const int reg = slot < n ? region_of(c, ps[u], cur_pos) : kRegionLocal;
+            if (reg == kRegionInvalid && sub == 0) set_status(c, ADSA_DEV_BAD_POSITION);
+            prev[u] = reg == kRegionPrevious;
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            inv[u] = 0.f;
+            if (prev[u] && piece_ok) {
+                raw[u] = ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8);
+                inv[u] = inv_norm[slot];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!prev[u]) continue;
+            if (sub == 0) ++cnt;
+            if (piece_ok) {
+                float f[8];
+                unpack8(raw[u], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(inv[u], f[e], acc[e]);
+            }
         }
     }
 #pragma unroll
@@ -88,31 +110,50 @@ score_kernel(DevCtx c, int layer, int cur_pos, float *scores_out)
 #pragma unroll
     for (int e = 0; e < 8; ++e) sv[e] = piece_ok ? s_vec[sub * 8 + e] : 0.f;
 
-    for (int sb = warp * RPW; sb < n; sb += kSSWarps * RPW) {   // warp-uniform bounds: all lanes join the shuffles
-        const int slot = sb + grp;
-        int reg = slot < n ? region_of(c, pos[slot], cur_pos) : kRegionInvalid;
-        float dot = 0.f, self = 0.f;
-        if (reg == kRegionPrevious && piece_ok) {
-            float f[8];
-            unpack8(ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8), f);
+    for (int sb0 = warp * RPW; sb0 < n; sb0 += U * kStep) {   // warp-uniform bounds: all lanes join the shuffles
+        int ps[U];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], sv[e], dot); self = fmaf(f[e], f[e], self); }
-        }
+        for (int u = 0; u < U; ++u) ps[u] = sb0 + u * kStep + grp < n ? pos[sb0 + u * kStep + grp] : -1;
+        uint4 raw[U];
+        float inv[U];
+        int regs[U];
 #pragma unroll
-        for (int o = 1; o < LPR; o <<= 1) {
-            dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            self += __shfl_xor_sync(0xffffffffu, self, o);
-        }
-        if (sub == 0 && slot < n) {
-            float S = CUDART_NAN_F;
-            if (reg == kRegionPrevious) {
-                float inv = inv_norm[slot];
-                // (p-1) S_i = u_i.s - u_i.u_i; dividing (not multiplying by a reciprocal) keeps the
-                // last bit where the definition puts it; "+ 0" folds -0 into +0 for the integer ordering
-                S = p > 1 ? (inv * dot - inv * inv * self) / (float)(p - 1) + 0.0f : 0.0f;
+        for (int u = 0; u < U; ++u) {
+            const int slot = sb0 + u * kStep + grp;
+            regs[u] = slot < n ? region_of(c, ps[u], cur_pos) : kRegionInvalid;
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            inv[u] = 0.f;
+            if (regs[u] == kRegionPrevious) {
+                if (piece_ok) raw[u] = ldg128(c.v_pool + row_offset(c, pt, slot) + sub * 8);
+                if (sub == 0) inv[u] = inv_norm[slot];
             }
-            scores[slot] = S;
-            if (scores_out) scores_out[slot] = S;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (sb0 + u * kStep >= n) break;   // (warp-uniform)
+            const int slot = sb0 + u * kStep + grp;
+            float dot = 0.f, self = 0.f;
+            if (regs[u] == kRegionPrevious && piece_ok) {
+                float f[8];
+                unpack8(raw[u], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], sv[e], dot); self = fmaf(f[e], f[e], self); }
+            }
+#pragma unroll
+            for (int o = 1; o < LPR; o <<= 1) {
+                dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                self += __shfl_xor_sync(0xffffffffu, self, o);
+            }
+            if (sub == 0 && slot < n) {
+                float S = CUDART_NAN_F;
+                if (regs[u] == kRegionPrevious) {
+                    // (p-1) S_i = u_i.s - u_i.u_i; dividing (not multiplying by a reciprocal) keeps the
+                    // last bit where the definition puts it; "+ 0" folds -0 into +0 for the integer ordering
+                    S = p > 1 ? (inv[u] * dot - inv[u] * inv[u] * self) / (float)(p - 1) + 0.0f : 0.0f;
+                }
+                scores[slot] = S;
+                if (scores_out) scores_out[slot] = S;
+            }
         }
     }
 }
