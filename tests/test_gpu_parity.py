@@ -398,6 +398,40 @@ def test_selection_on_structured_values(kind, mode):
         lh.step(q, kn, vn, cur, budget)
 
 
+@pytest.mark.parametrize("kind", ["duplicates", "equal"])
+@pytest.mark.parametrize("mode", ["fused", "two-sweep-fused", "calls"])
+def test_exact_ties_over_many_steps_follow_the_position_rule(kind, mode):
+    """A full cache whose V rows come in identical pairs (or are all identical), stepped many times with new rows
+    that repeat cached ones: at every step several candidates share the highest score exactly, so the row that
+    goes is decided by position (Eq. 3 with the tie rule), also on the steps where the fused kernel would
+    otherwise take the evictee the previous step noted.  Not one selection may differ from the oracle's."""
+    H = _harness()
+    T0, gh, gw, d = 4, 20, 16, 64
+    w = Workload("ties", 93, 1, 1, 6, d, T0, gh, gw, 0.5, 1.0)
+    n_rows = T0 + 250
+    g0 = 17 * gw + 3
+    cur0 = T0 + g0
+    eng = H.engine_for(w, capacity=n_rows, page_rows=32)
+    lh = H.LayerHarness(eng, 0, oracle_cap=n_rows + 2, fused=_apply_mode(eng, mode))
+    rng = np.random.default_rng(7)
+    recent = np.arange(cur0 - 2 * gw, cur0)                 # the cells of the local window and the row above are cached
+    older = np.arange(T0, cur0 - 2 * gw)
+    pos = np.stack([rng.permutation(np.concatenate([np.arange(T0), recent, np.sort(rng.choice(older, n_rows - T0 - recent.size, replace=False))]))
+                    for _ in range(6)]).astype(np.int32)
+    vals = np.stack([structured_values(kind, n_rows, d, seed=30 + s) for s in range(6)])
+    k = np.stack([structured_values("iid", n_rows, d, seed=40 + s) for s in range(6)]).reshape(1, 6, n_rows, d)
+    lh.prefill(k, vals.reshape(1, 6, n_rows, d), 0, pos)
+    for t in range(2 * gw + 5):                             # across two grid-row boundaries
+        q, kn, vn = layer_step_qkv(w, 3, 0, g0 + t)
+        vn = vn.copy().reshape(6, d)
+        if t % 3 != 2:                                      # two steps in three: the new row repeats a cached one
+            for s_ in range(6):
+                vn[s_] = vals[s_, (7 * t + s_) % n_rows]
+        lh.step(q, kn, vn.reshape(1, 6, d), cur0 + t, n_rows)
+    assert lh.stats.tolerated_divergences == 0
+    assert lh.stats.steps == 2 * gw + 5
+
+
 @pytest.mark.parametrize("mode", ["calls", "fused"])
 def test_repeat_runs_are_bit_identical(mode):
     outs = []
