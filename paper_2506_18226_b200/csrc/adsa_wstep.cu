@@ -215,6 +215,10 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     constexpr int PITCH = SWZ ? 128 : kWRowBytes;      // bytes from row to row inside a sub-tile
     constexpr int SEGB = TR * 128;                     // bytes of a swizzled sub-tile
     constexpr bool RAGGED = RS % 16 != 0;              // the last 16-element step has only its first 8 elements
+    // RS is the row width of the tiles in shared memory.  The swizzled layouts also serve narrower pool rows (any
+    // stride up to RS elements): the tensor copies fill what lies beyond a pool row with zeros.  The plain layout
+    // is the pool's rows as they lie (row stride = RS).
+    const int g_rs = SWZ ? c.row_stride : RS;          // elements per pool row
     constexpr int kWPart = w_part_floats(RS);
     constexpr bool SPLIT = KS > 4;                     // two accumulation chains per K.q and V.s product
     extern __shared__ __align__(1024) unsigned char smem_all[];
@@ -285,9 +289,11 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
     };
     // one L2 hint per 128-byte line of a pool row
     auto hint_row = [&](const __nv_bfloat16 *row) {
+        const int row_bytes = g_rs * 2;
 #pragma unroll
-        for (int o = 0; o < kWRowBytes; o += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + o));
-        if (kWRowBytes % 128 != 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + kWRowBytes - 16));
+        for (int o = 0; o < kWRowBytes; o += 128)
+            if (o < row_bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + o));
+        if (row_bytes % 128 != 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(row) + row_bytes - 16));
     };
     const RegionCut cut_now = region_cut(c, a.cur_pos), cut_next = region_cut(c, a.cur_pos + 1);
     // the local window does not move between this step and the next, and the new row stays inside it: the next
@@ -597,8 +603,8 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             const int pg0 = (int)__umulhi((uint32_t)b0, c.pr_magic), in0 = b0 - pg0 * c.page_rows;
             if (in0 + rows <= c.page_rows) {
                 if (lane < 2) {
-                    const __nv_bfloat16 *src = (lane ? c.v_pool : c.k_pool) + ((size_t)pt_s[pg0] * c.page_rows + in0) * (size_t)RS;
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * kWRowBytes) : "memory");
+                    const __nv_bfloat16 *src = (lane ? c.v_pool : c.k_pool) + ((size_t)pt_s[pg0] * c.page_rows + in0) * (size_t)g_rs;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * g_rs * 2) : "memory");
                 }
             } else if (row < n) {
                 const size_t off = c.max_pages == 1 ? ((size_t)pt_s[0] * c.page_rows + row) * (size_t)c.row_stride
@@ -633,7 +639,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
         if (carried_slot >= 0) {
             const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, carried_slot));
 #pragma unroll
-            for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
+            for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < g_rs ? vrow[32 * j + lane] : 0u;
         }
         // after a stage has been read (all lanes), lane 0 refills it with the tile `depth` ahead
         // (the reads are complete once their results have been used, which in-order issue guarantees
@@ -850,7 +856,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             if (carried_slot < 0) {
                 const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot));
 #pragma unroll
-                for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
+                for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < g_rs ? vrow[32 * j + lane] : 0u;
             }
             const uint32_t *cm_g = c.cand_mask + (size_t)sid * c.mask_words;
             for (int b = rk + lane * G; b < n_tiles; b += 32 * G) {   // one block per lane
@@ -957,7 +963,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                 if (single && evict_slot >= 0) {
                     const uint32_t *vrow = reinterpret_cast<const uint32_t *>(c.v_pool + row_offset(c, pt_s, evict_slot));
 #pragma unroll
-                    for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < RS ? vrow[32 * j + lane] : 0u;
+                    for (int j = 0; j < NJ; ++j) ve[j] = 64 * j + 2 * lane < g_rs ? vrow[32 * j + lane] : 0u;
                     inv_e = inv_s[evict_slot];
                 }
                 const bool drop_prev = K == 0 && p > 0;
@@ -1227,7 +1233,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     if (r0 + rows <= c.page_rows) {   // inside the first page: one bulk hint per pool
                         if (lane < 2) {
                             const __nv_bfloat16 *src = (lane ? c.v_pool : c.k_pool) + ((size_t)pg0 * c.page_rows + r0) * (size_t)c.row_stride;
-                            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * kWRowBytes) : "memory");
+                            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(rows * g_rs * 2) : "memory");
                         }
                     } else if (lane < rows) {         // a row per lane, located through the next stream's page table
                         const int row = r0 + lane;
@@ -1396,7 +1402,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
             // ---- the update itself, by the first warp ---------------------------------------------------
             if (okay && rk == 0) {
                 for (int i = 0; i < ns; ++i) {   // survivors move down: K and V rows in pieces of 16 bytes
-                    constexpr int kChunks = kWRowBytes / 16;
+                    const int kChunks = g_rs / 8;   // 16-byte pieces of a pool row
                     const int row = surv[i], dst = holes[i];
                     size_t so = row_offset(c, pt, row), go = row_offset(c, pt, dst);
                     if (lane < 2 * kChunks) {
@@ -1425,7 +1431,7 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
                     const size_t off = row_offset(c, pt_s, last_hole);
 #pragma unroll
                     for (int j = 0; j < NJ; ++j) {
-                        if (64 * j + 2 * lane < RS) {
+                        if (64 * j + 2 * lane < g_rs) {
                             *reinterpret_cast<uint32_t *>(c.k_pool + off + 64 * j + 2 * lane) = kn[j];
                             *reinterpret_cast<uint32_t *>(c.v_pool + off + 64 * j + 2 * lane) = vn[j];
                         }
@@ -1444,9 +1450,12 @@ wstep_kernel(DevCtx c, WStepArgs a, const __grid_constant__ WStepMaps maps)
 }
 
 // ---- host side ------------------------------------------------------------
-// Row layouts the kernel is compiled for: 64-element rows (32-row stages), 104- and 128-element rows (16-row stages).
-bool wstep_supported(const DevCtx &c) { return (c.row_stride == 64 || c.row_stride == 104 || c.row_stride == 128) && c.d % 2 == 0; }
-static int wstep_stage_rows(const DevCtx &c) { return c.row_stride == 64 ? 32 : 16; }
+// Tile layouts the kernel is compiled for: 64-element rows (32-row stages), 104- and 128-element rows (16-row stages).
+// A pool whose rows are narrower than 64 (or 128) elements is served by the 64- (or 128-) element layout: the tensor
+// copies read the pool's rows and fill the rest of a tile row with zeros.  104-element rows keep their own layout.
+bool wstep_supported(const DevCtx &c) { return c.row_stride >= 8 && c.row_stride <= 128 && c.row_stride % 8 == 0 && c.d % 2 == 0; }
+static int wstep_tile_rs(const DevCtx &c) { return c.row_stride == 104 ? 104 : c.row_stride <= 64 ? 64 : 128; }
+static int wstep_stage_rows(const DevCtx &c) { return wstep_tile_rs(c) == 64 ? 32 : 16; }
 
 // Tensor maps of both pools for boxes of 1, 2, 4, .. 32 rows (128-byte swizzle for 128-byte rows, none
 // otherwise).  The encoder is cuTensorMapEncodeTiled, looked up at run time so that the library links cudart only.
@@ -1508,7 +1517,7 @@ cudaError_t configure_wstep_kernel(const DevCtx &c)
     cudaError_t e = cudaSuccess;
     for (int warps : {8, 10, 12, 16})
         for (int fused = 0; fused < 2 && e == cudaSuccess; ++fused) {
-            wstep_fn f = wstep_variant(c.row_stride, warps, fused != 0);
+            wstep_fn f = wstep_variant(wstep_tile_rs(c), warps, fused != 0);
             if (f) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmemLimit);
         }
     return e;
@@ -1521,7 +1530,7 @@ WStepPlan plan_wstep(const DevCtx &c, bool fused, int sm_count, int max_depth, i
 {
     WStepPlan p = {};
     if (!wstep_supported(c)) return p;
-    const int rs = c.row_stride, tr = wstep_stage_rows(c), stage_bytes = w_stage_bytes(rs, tr);
+    const int rs = wstep_tile_rs(c), tr = wstep_stage_rows(c), stage_bytes = w_stage_bytes(rs, tr);
     const int max_warps = rs == 64 ? 16 : (rs == 128 && fused) ? 8 : kWWideMaxWarps;   // the wide-row kernels need more registers per thread
     const int n_streams = c.S * (n_run < 1 ? 1 : n_run);   // streams one launch serves
     int groups = (n_streams + sm_count - 1) / sm_count;
@@ -1580,7 +1589,7 @@ cudaError_t launch_wstep(const DevCtx &c, const WStepPlan &plan, const WStepMaps
     a.out_bf16 = (__nv_bfloat16 *)out_bf16; a.out_f32 = out_f32;
     a.scratch = c.wscratch;
     const int warps = plan.n_groups * plan.group_warps, threads = warps * 32;
-    wstep_fn kern = wstep_variant(c.row_stride, warps, fused);
+    wstep_fn kern = wstep_variant(wstep_tile_rs(c), warps, fused);
     if (!kern) return cudaErrorInvalidConfiguration;
     // launched so that its set-up overlaps the tail of the kernel before it in the stream (the kernel
     // itself waits for that kernel's completion before it reads or writes global memory)

@@ -75,6 +75,9 @@ def _run_trajectory(w, layer, seed, budget_fn, *, n_layers_engine=1, page_rows=N
     (128, 16, 40, 7, 6, 0.6, 0),   # 256-byte rows over several blocks, pages of exactly one 16-row stage
     (128, 13, 45, 6, 7, 0.5, 0),   # 256-byte rows, pages that cut every stage into pieces
     (122, 64, 33, 6, 6, 0.5, 0),   # head_dim just below 128: the padding of a 128-element row stays out of every sum
+    (48, 9, 20, 6, 7, 0.5, 0),     # 96-byte rows in 128-byte tiles: the copies fill the rest of a tile row with zeros
+    (72, 10, 30, 6, 6, 0.6, 0),    # 144-byte rows in the two-half layout (the second half holds 8 elements)
+    (120, 16, 35, 7, 5, 0.5, 0),   # 240-byte rows in the two-half layout
     (256, 4, 3, 3, 5, 0.5, 0),     # 32 lanes per row
     (8, 2, 2, 7, 3, 0.4, 0),       # smallest head_dim
 ])
@@ -84,6 +87,18 @@ def test_small_shapes_full_trajectory(d, page_rows, T0, gh, gw, beta, chunk, mod
     C = max(2, w.capacity())
     lh, eng = _run_trajectory(w, 0, 1, lambda cur: C, page_rows=page_rows, chunk_rows=chunk, mode=mode)
     assert lh.stats.steps == gh * gw and lh.stats.max_score_err <= 1e-6
+
+
+@pytest.mark.parametrize("d,served", [(8, True), (32, True), (48, True), (64, True), (72, True), (100, True), (120, True),
+                                      (128, True), (136, False), (256, False)])
+def test_which_head_dims_the_tensor_core_kernel_serves(d, served):
+    """Every row stride up to 128 elements runs on the tensor-core kernel (one warp group walks a whole stream in
+    32-row blocks: adsa_plan_attn reports one split of 32-row steps); wider rows fall back to the other kernels."""
+    H = _harness()
+    w = Workload(f"plan-d{d}", 60, 1, 1, 2, d, 8, 8, 8, 0.5, 1.0)
+    eng = H.engine_for(w, capacity=w.capacity(), page_rows=8)
+    splits, step_rows = eng.plan_attn(40)
+    assert ((splits, step_rows) == (1, 32)) == served
 
 
 @pytest.mark.parametrize("n_prefix_kind,rows_back", [("none", 1), ("text+5%", 1), ("text", 2), ("text", 0)])
