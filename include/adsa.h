@@ -269,8 +269,8 @@ ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, c
 ADSA_API int adsa_plan_attn(const adsa_ctx *ctx, int n_rows, int *n_splits, int *chunk_rows);
 
 /* Which kernels adsa_sparse_decode_attn and adsa_layer_step use.  Same results in every mode.
- *   1 (default) automatic: when pool rows are 64 elements wide, the warp-group kernel (a few warps
- *               own a stream, each with its own TMA tile ring; tensor-core arithmetic); else the
+ *   1 (default) automatic: when pool rows are at most 128 elements wide (and head_dim is even), the warp-group
+ *               kernel (a few warps own a stream, each with its own TMA tile ring; tensor-core arithmetic); else the
  *               persistent pipelined CUDA-core kernel (one CTA per SM, a producer warp feeding a
  *               ring of K/V tiles); if that does not fit shared memory, the cluster kernel; if a
  *               stream does not fit a cluster either, the streaming kernels

@@ -69,8 +69,9 @@
 
 namespace adsa {
 
-// The kernel is compiled for two row layouts (template parameters RS = elements per pool row, TR = rows per
-// ring stage):
+// The kernel is compiled for three tile layouts (template parameters RS = elements per tile row in shared memory,
+// TR = rows per ring stage).  The two swizzled ones also serve pools whose rows are narrower than the tile's: the
+// tensor copies read the pool's rows and fill the rest of a tile row with zeros.
 //   RS = 64,  TR = 32   128-byte rows written with the 128-byte swizzle; a stage is a whole 32-row block;
 //   RS = 104, TR = 16   208-byte rows (head_dim 97 .. 104) written as they lie: a pitch of 208 bytes puts the eight
 //                       rows of an ldmatrix on eight different bank groups without any swizzle; a stage is half a
