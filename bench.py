@@ -53,6 +53,7 @@ def parse_args(argv=None):
     ap.add_argument("--workload", default="cfg4", help="cfg1 .. cfg5: the headline workload of the JSON line")
     ap.add_argument("--beta", type=float, default=None)
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
+    ap.add_argument("--head-dim", type=int, default=0, help="override the head dimension (experiments with other row widths)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -81,7 +82,16 @@ def parse_args(argv=None):
 def _workload(args, name=None, beta=None):
     from dataclasses import replace
     w = get_workload(int((name or args.workload).replace("cfg", "")), beta if name else args.beta)
-    return w if args.layers is None or name else replace(w, n_layers=args.layers, name=f"{w.name}-{args.layers}layers")
+    if name:
+        return w
+    if args.head_dim:      # an experiment, not one of the benchmark configurations: the same stack with other heads
+        w = replace(w, head_dim=args.head_dim, name=f"{w.name}-headdim{args.head_dim}")
+    return w if args.layers is None else replace(w, n_layers=args.layers, name=f"{w.name}-{args.layers}layers")
+
+
+def _traffic_key(w):
+    """The workload name the ncu captures are filed under: "cfg4" ...; a head-dim experiment has none."""
+    return w.name if "headdim" in w.name else w.name[:4]
 
 
 def peaks():
@@ -428,8 +438,7 @@ def measure(w, args, dev, rank, world, local_rank, K, W, detail=True):
         per_launch = L if launch_kind == "token-launch" else 1
         res["roofline"] = _roofline("fused", f"fused layer-step (adsa_token_step, {launch_kind}: {per_launch} layer-step(s) per launch)",
                                     step_bytes, us_unit, per_launch, n_timed,
-                                    dram_traffic("fused", args.workload if w.name.startswith(args.workload) else w.name[:4],
-                                                 st.page_rows, launch_kind, C))
+                                    dram_traffic("fused", _traffic_key(w), st.page_rows, launch_kind, C))
     if detail and rank == 0 and T0 + HW > C:
         res["detail"].update(full_cache_detail(st, args, M, step_bytes, attn_bytes))
     return res
@@ -441,7 +450,7 @@ def full_cache_detail(st, args, M, step_bytes, attn_bytes):
     of the four calls.  The keep masks are per layer, so the grouped calls are a valid trajectory."""
     eng, L, C, T0, HW, dev = st.eng, st.L, st.C, st.T0, st.HW, st.dev
     out = {}
-    wname = st.w.name[:4]
+    wname = _traffic_key(st.w)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # (1) one launch per layer, as a decoder whose layers feed each other has to do
     eng.set_token_launch(0)                      # adsa_token_step now launches layer after layer, from C
