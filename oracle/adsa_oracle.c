@@ -524,6 +524,74 @@ void adsa_oracle_rope_2d(const float *x, const int *pos, int n, int d, int n_tex
     }
 }
 
+/* -------------------------------------------------------------------------
+ * The pieces of the host model around the attention (Section 5 integrates the
+ * method with LlamaGen; the paper defines none of these, they are the published
+ * operations of that decoder family).  Parity of a whole generated image is
+ * unpinned (no trained weights); each operation is pinned by its definition.
+ * ------------------------------------------------------------------------- */
+
+/* Root-mean-square normalisation: y_i = x_i / sqrt(mean_j x_j^2 + eps) * w_i.  x: [rows][dim], w: [dim]. */
+void adsa_oracle_rmsnorm(const float *x, const float *w, int rows, int dim, double eps, double *out)
+{
+    for (int r = 0; r < rows; ++r) {
+        double ss = 0.0;
+        for (int i = 0; i < dim; ++i) ss += (double)x[(size_t)r * dim + i] * (double)x[(size_t)r * dim + i];
+        const double inv = 1.0 / sqrt(ss / (double)dim + eps);
+        for (int i = 0; i < dim; ++i) out[(size_t)r * dim + i] = (double)x[(size_t)r * dim + i] * inv * (double)w[i];
+    }
+}
+
+/* The gated activation of the feed-forward block: out = silu(gate) * up, silu(g) = g / (1 + exp(-g)). */
+void adsa_oracle_swiglu(const float *gate, const float *up, long long n, double *out)
+{
+    for (long long i = 0; i < n; ++i) {
+        const double g = gate[i];
+        out[i] = g / (1.0 + exp(-g)) * (double)up[i];
+    }
+}
+
+/* Classifier-free guidance and sampling of the next image token for one image.
+ * logits_cond, logits_uncond: [vocab].  Steps: mixed = uncond + scale * (cond - uncond); keep the top_k largest
+ * mixed logits (equal logits at the threshold: the lower token id is kept); p_i proportional to
+ * exp((mixed_i - max) / temperature) over the kept tokens; the token is the first kept id, in ascending order of
+ * id, at which the running sum of p reaches u * (sum of p), u in [0, 1) given by the caller.
+ * mixed_out [vocab] (may be NULL) receives the mixed logits, cdf_out [vocab] (may be NULL) the running sum
+ * divided by the total at every id (unchanged across ids that are not kept).  Returns the token. */
+int adsa_oracle_cfg_sample(const float *logits_cond, const float *logits_uncond, int vocab, double scale, int top_k,
+                           double temperature, double u, double *mixed_out, double *cdf_out)
+{
+    double *mixed = (double *)malloc(sizeof(double) * (size_t)vocab);
+    char *kept = (char *)calloc((size_t)vocab, 1);
+    for (int i = 0; i < vocab; ++i) mixed[i] = (double)logits_uncond[i] + scale * ((double)logits_cond[i] - (double)logits_uncond[i]);
+    if (top_k < 1) top_k = 1;
+    if (top_k > vocab) top_k = vocab;
+    for (int n = 0; n < top_k; ++n) {            /* pick the largest not yet kept, lowest id first among equals */
+        int best = -1;
+        for (int i = 0; i < vocab; ++i)
+            if (!kept[i] && (best < 0 || mixed[i] > mixed[best])) best = i;
+        kept[best] = 1;
+    }
+    double mx = -INFINITY, total = 0.0;
+    for (int i = 0; i < vocab; ++i) if (kept[i] && mixed[i] > mx) mx = mixed[i];
+    for (int i = 0; i < vocab; ++i) if (kept[i]) total += exp((mixed[i] - mx) / temperature);
+    double run = 0.0;
+    int token = -1, last_kept = -1;
+    for (int i = 0; i < vocab; ++i) {
+        if (kept[i]) {
+            run += exp((mixed[i] - mx) / temperature);
+            last_kept = i;
+            if (token < 0 && run >= u * total) token = i;
+        }
+        if (cdf_out) cdf_out[i] = run / total;
+        if (mixed_out) mixed_out[i] = mixed[i];
+    }
+    if (token < 0) token = last_kept;            /* rounding at u close to 1 */
+    free(mixed);
+    free(kept);
+    return token;
+}
+
 /* The same step for many independent streams.  Arrays carry a leading stream
  * dimension with stride cap_rows (state, lists) or d (q, k_new, v_new, out).
  * Threads split the streams; nothing else is parallel.  Returns the number of

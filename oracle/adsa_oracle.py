@@ -133,6 +133,36 @@ def rope_2d(x, pos, n_text, grid_w, base=10000.0) -> np.ndarray:
     return out
 
 
+def rmsnorm(x, w, eps=1e-5) -> np.ndarray:
+    """Root-mean-square normalisation of every row of x [rows, dim] with weights w [dim] (float64 out)."""
+    x, w = _f32(x), _f32(w)
+    rows, dim = x.shape
+    out = np.empty((rows, dim), dtype=np.float64)
+    lib().adsa_oracle_rmsnorm(_p(x, C.c_float), _p(w, C.c_float), rows, dim, C.c_double(eps), _p(out, C.c_double))
+    return out
+
+
+def swiglu(gate, up) -> np.ndarray:
+    """silu(gate) * up, element by element (float64 out)."""
+    gate, up = _f32(gate), _f32(up)
+    out = np.empty(gate.shape, dtype=np.float64)
+    lib().adsa_oracle_swiglu(_p(gate, C.c_float), _p(up, C.c_float), C.c_longlong(gate.size), _p(out, C.c_double))
+    return out
+
+
+def cfg_sample(logits_cond, logits_uncond, scale, top_k, temperature, u):
+    """Classifier-free guidance, top-k filter and inverse-CDF sampling for one image.
+    Returns (token, mixed logits float64 [vocab], running share of the kept mass by token id float64 [vocab])."""
+    lc, lu = _f32(logits_cond), _f32(logits_uncond)
+    vocab = lc.shape[0]
+    mixed, cdf = np.empty(vocab, dtype=np.float64), np.empty(vocab, dtype=np.float64)
+    fn = lib().adsa_oracle_cfg_sample
+    fn.restype = C.c_int
+    tok = fn(_p(lc, C.c_float), _p(lu, C.c_float), vocab, C.c_double(scale), int(top_k), C.c_double(temperature),
+             C.c_double(u), _p(mixed, C.c_double), _p(cdf, C.c_double))
+    return int(tok), mixed, cdf
+
+
 @dataclass
 class StepResult:
     out: np.ndarray          # [streams, d] float64

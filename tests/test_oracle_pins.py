@@ -625,3 +625,84 @@ def test_cache_sizes_of_tables_1_and_2(table, H, W, dense, cache, printed):
         else:
             assert len(res.evict_pos[0]) == 1 and n_live[0] == cache             # then one eviction per step
     assert peak == cache
+
+
+# ---------------------------------------------------------------------------
+# the host model's operations around the attention (Section 5: the method is integrated with LlamaGen)
+# ---------------------------------------------------------------------------
+def test_rmsnorm_unit_mean_square_scale_invariance_and_torch():
+    import torch
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((5, 96)).astype(np.float32)
+    w = rng.standard_normal(96).astype(np.float32)
+    y = orc.rmsnorm(x, np.ones(96, np.float32), eps=0.0)
+    assert np.allclose((y ** 2).mean(axis=1), 1.0, atol=1e-12)                 # unit mean square without eps
+    assert np.allclose(orc.rmsnorm(4.0 * x, w, eps=0.0), orc.rmsnorm(x, w, eps=0.0), atol=1e-12)   # scale-free
+    want = torch.nn.functional.rms_norm(torch.from_numpy(x).double(), (96,), torch.from_numpy(w).double(), eps=1e-5)
+    assert np.allclose(orc.rmsnorm(x, w, eps=1e-5), want.numpy(), atol=1e-12)
+    # hand case: x = (3, 4), w = (1, 2): mean square 12.5, y = (3, 8) / sqrt(12.5)
+    y = orc.rmsnorm(np.array([[3.0, 4.0]], np.float32), np.array([1.0, 2.0], np.float32), eps=0.0)
+    assert np.allclose(y, np.array([[3.0, 8.0]]) / np.sqrt(12.5), atol=1e-14)
+    # eps matters for a zero row: the output is zero, not NaN
+    assert np.array_equal(orc.rmsnorm(np.zeros((1, 8), np.float32), np.ones(8, np.float32), eps=1e-5), np.zeros((1, 8)))
+
+
+def test_swiglu_hand_values_and_torch():
+    import torch
+    g = np.array([0.0, 1.0, -1.0, 20.0, -20.0], np.float32)
+    u = np.array([2.0, 2.0, 2.0, 0.5, 3.0], np.float32)
+    got = orc.swiglu(g, u)
+    assert got[0] == 0.0
+    assert np.isclose(got[1], 2.0 / (1.0 + np.exp(-1.0)), atol=1e-15)
+    assert np.isclose(got[1] - got[2], 2.0, atol=1e-15)                         # silu(g) - silu(-g) = g (both times up = 2)
+    assert np.isclose(got[3], 10.0, atol=1e-7) and abs(got[4]) < 1e-6             # silu -> identity / zero far out
+    rng = np.random.default_rng(12)
+    a, b = rng.standard_normal(200).astype(np.float32), rng.standard_normal(200).astype(np.float32)
+    want = torch.nn.functional.silu(torch.from_numpy(a).double()) * torch.from_numpy(b).double()
+    assert np.allclose(orc.swiglu(a, b), want.numpy(), atol=1e-14)
+
+
+def test_cfg_sample_mixing_top_k_and_inverse_cdf():
+    lc = np.array([1.0, 2.0, 3.0, 0.0, 3.0], np.float32)
+    lu = np.array([0.0, 1.0, 0.0, 4.0, 0.0], np.float32)
+    # scale 1 is the conditional logits, scale 0 the unconditional ones, scale 2 extrapolates
+    for scale, want in ((1.0, lc), (0.0, lu), (2.0, 2.0 * lc - lu)):
+        _, mixed, _ = orc.cfg_sample(lc, lu, scale, 5, 1.0, 0.0)
+        assert np.array_equal(mixed, want.astype(np.float64))
+    # top_k = 1 is the argmax, whatever u; equal maxima: the lower id
+    for u in (0.0, 0.3, 0.999999):
+        assert orc.cfg_sample(lc, lu, 1.0, 1, 1.0, u)[0] == 2
+    # top_k = 2 at scale 1 keeps ids 2 and 4 (both 3.0): each has half of the mass
+    tok, _, cdf = orc.cfg_sample(lc, lu, 1.0, 2, 1.0, 0.49)
+    assert tok == 2 and np.allclose(cdf, [0.0, 0.0, 0.5, 0.5, 1.0])
+    assert orc.cfg_sample(lc, lu, 1.0, 2, 1.0, 0.51)[0] == 4
+    # top_k = 3: the threshold value 2.0 is unique here; ids 1, 2, 4 with weights e^-1 : 1 : 1
+    tok, _, cdf = orc.cfg_sample(lc, lu, 1.0, 3, 1.0, 0.0)
+    z = np.exp(-1.0) + 2.0
+    assert tok == 1 and np.allclose(cdf, [0.0, np.exp(-1.0) / z, (np.exp(-1.0) + 1.0) / z, (np.exp(-1.0) + 1.0) / z, 1.0])
+    # a tie AT the threshold: logits (5, 1, 1, 1), top_k = 2 keeps id 0 and the lowest of the equal ids
+    tie = np.array([5.0, 1.0, 1.0, 1.0], np.float32)
+    _, _, cdf = orc.cfg_sample(tie, tie, 1.0, 2, 1.0, 0.0)
+    assert cdf[1] == 1.0 and cdf[0] < 1.0
+    # temperature: T -> 0 concentrates on the largest kept logit, a large T flattens the kept ones
+    assert orc.cfg_sample(lc, lu, 1.0, 3, 1e-3, 0.9)[0] in (2, 4)
+    _, _, cdf = orc.cfg_sample(lc, lu, 1.0, 3, 1e6, 0.0)
+    assert np.allclose(cdf[[1, 2, 4]], [1 / 3, 2 / 3, 1.0], atol=1e-5)
+
+
+def test_cfg_sample_frequencies_follow_the_softmax_of_the_kept_logits():
+    """Over a grid of u the share of each token equals its softmax probability among the kept tokens
+    (torch.softmax on torch.topk as the independent statement)."""
+    import torch
+    rng = np.random.default_rng(13)
+    lc, lu = rng.standard_normal(40).astype(np.float32), rng.standard_normal(40).astype(np.float32)
+    scale, k, T = 1.75, 7, 0.8
+    mixed = torch.from_numpy(lu).double() + scale * (torch.from_numpy(lc).double() - torch.from_numpy(lu).double())
+    top = torch.topk(mixed, k)
+    want = np.zeros(40)
+    want[top.indices.numpy()] = torch.softmax(top.values / T, 0).numpy()
+    n = 4000
+    counts = np.zeros(40)
+    for i in range(n):
+        counts[orc.cfg_sample(lc, lu, scale, k, T, (i + 0.5) / n)[0]] += 1
+    assert np.abs(counts / n - want).max() <= 1.0 / n + 1e-12
