@@ -364,6 +364,38 @@ ADSA_API int adsa_decode_attn_static(const void *q, const void *k, const void *v
                                      int row_stride, float softmax_scale, void *out_bf16, float *out_f32,
                                      adsa_stream_t stream);
 
+/* ---- the host model around the attention -------------------------------------------------------------------------
+ * Section 5 integrates the method with a LlamaGen decoder.  The paper defines none of that decoder's own operations;
+ * these three are its published element-wise and sampling steps, stateless calls on caller-owned buffers (no
+ * context, no workspace; the projections between them are plain GEMMs and are left to the caller's BLAS).  All
+ * pointers [device], 16-byte aligned where rows are read in 16-byte pieces; fp32 arithmetic; each call enqueues one
+ * kernel on `stream` and returns (ADSA_EINVAL for a null pointer, a misaligned buffer or a size outside the stated
+ * range, before anything is launched). */
+
+/* Root-mean-square normalisation, row by row: out[r][i] = x[r][i] / sqrt(mean_j x[r][j]^2 + eps) * w[i].
+ *   x, out  bf16 [rows][dim] (out may be x);  w  bf16 [dim];  dim a multiple of 8, >= 8;  eps >= 0 */
+ADSA_API int adsa_rmsnorm(const void *x, const void *w, void *out, long long rows, int dim, float eps,
+                          adsa_stream_t stream);
+
+/* The gated activation of the feed-forward block: out[r][i] = silu(gate[r][i]) * up[r][i], silu(g) = g / (1 + e^-g).
+ *   gate, up  bf16, rows of `hidden` elements ld_in elements apart (ld_in = hidden for two separate tensors,
+ *             2 * hidden with up = gate + hidden for one tensor that holds both halves side by side)
+ *   out       bf16 [rows][hidden];  hidden and ld_in multiples of 8 */
+ADSA_API int adsa_swiglu(const void *gate, const void *up, void *out, long long rows, int hidden, long long ld_in,
+                         adsa_stream_t stream);
+
+/* The next image token of every image from the logits of its conditional and unconditional rows:
+ *   mixed = uncond + scale * (cond - uncond)                       (classifier-free guidance)
+ *   keep the top_k largest mixed logits (equal logits at the threshold: the lower token ids)
+ *   p_i proportional to exp((mixed_i - max) / temperature) over the kept ids
+ *   token = the first kept id, in ascending order of id, at which the running sum of p reaches u * (sum of p)
+ * The random numbers are the caller's: uniforms [n_images] f32 in [0, 1).
+ *   logits  bf16 [2 * n_images][vocab]: the conditional rows of all images, then their unconditional rows
+ *   tokens  int32 [n_images];  1 <= top_k <= vocab <= 32768;  temperature > 0
+ * One block per image; sums are taken in fp32 in a fixed order, so a call is reproducible. */
+ADSA_API int adsa_cfg_sample(const void *logits, int n_images, int vocab, float scale, int top_k, float temperature,
+                             const float *uniforms, int32_t *tokens, adsa_stream_t stream);
+
 ADSA_API const char *adsa_strerror(int status);
 
 #ifdef __cplusplus

@@ -5,9 +5,12 @@ from .binding import (  # noqa: F401
     AdsaEngine,
     AdsaError,
     EXPORTS,
+    cfg_sample,
     decode_attn_static,
     load,
+    rmsnorm,
     strerror,
+    swiglu,
     workspace_bytes,
 )
 from .build import build_lib  # noqa: F401

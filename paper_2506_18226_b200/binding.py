@@ -23,6 +23,7 @@ EXPORTS = [
     "adsa_set_stream_rows", "adsa_prefill_attn", "adsa_rope_2d", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
     "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_host_chunks", "adsa_set_stream_warps", "adsa_set_single_sweep",
     "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror", "adsa_decode_attn_static",
+    "adsa_rmsnorm", "adsa_swiglu", "adsa_cfg_sample",
 ]
 
 
@@ -84,6 +85,9 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_layer_rows_bound": [vp, i32, C.POINTER(i32)],
             "adsa_get_status": [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_int32 * 4)],
             "adsa_decode_attn_static": [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp],
+            "adsa_rmsnorm": [vp, vp, vp, C.c_longlong, i32, C.c_float, vp],
+            "adsa_swiglu": [vp, vp, vp, C.c_longlong, i32, C.c_longlong, vp],
+            "adsa_cfg_sample": [vp, i32, i32, C.c_float, i32, C.c_float, vp, vp, vp],
         }
         for name, args in sig.items():
             fn = getattr(lib, name)
@@ -129,6 +133,41 @@ def decode_attn_static(q, k, v, n_rows, k_new, v_new, out_bf16=None, out_f32=Non
                                         _ptr(out_f32), _stream())
     if rc:
         raise AdsaError(rc, "adsa_decode_attn_static")
+
+
+def rmsnorm(x, w, out=None, eps=1e-5):
+    """adsa_rmsnorm: out[r] = x[r] / sqrt(mean(x[r]^2) + eps) * w, rows of bf16 [.., dim] (contiguous)."""
+    out = torch.empty_like(x) if out is None else out
+    rc = load().adsa_rmsnorm(_ptr(x), _ptr(w), _ptr(out), x.numel() // x.shape[-1], x.shape[-1], float(eps), _stream())
+    if rc:
+        raise AdsaError(rc, "adsa_rmsnorm")
+    return out
+
+
+def swiglu(gate, up, out=None):
+    """adsa_swiglu: silu(gate) * up.  gate, up: bf16 [rows, hidden], either two contiguous tensors or the two halves
+    of one contiguous [rows, 2 * hidden] tensor (views)."""
+    rows, hidden = gate.shape
+    ld = gate.stride(0)
+    if up.stride(0) != ld or gate.stride(1) != 1 or up.stride(1) != 1:
+        raise ValueError("gate and up must share a row pitch and be dense along the row")
+    out = torch.empty((rows, hidden), dtype=gate.dtype, device=gate.device) if out is None else out
+    rc = load().adsa_swiglu(_ptr(gate), _ptr(up), _ptr(out), rows, hidden, ld, _stream())
+    if rc:
+        raise AdsaError(rc, "adsa_swiglu")
+    return out
+
+
+def cfg_sample(logits, scale, top_k, temperature, uniforms, tokens=None):
+    """adsa_cfg_sample: the next image token of every image.  logits: bf16 [2 * n_images, vocab] (conditional rows,
+    then unconditional rows), uniforms: f32 [n_images] in [0, 1); returns int32 [n_images]."""
+    n_images, vocab = logits.shape[0] // 2, logits.shape[1]
+    tokens = torch.empty(n_images, dtype=torch.int32, device=logits.device) if tokens is None else tokens
+    rc = load().adsa_cfg_sample(_ptr(logits), n_images, vocab, float(scale), int(top_k), float(temperature), _ptr(uniforms),
+                                _ptr(tokens), _stream())
+    if rc:
+        raise AdsaError(rc, "adsa_cfg_sample")
+    return tokens
 
 
 class AdsaEngine:

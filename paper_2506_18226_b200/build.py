@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libadsa.so")
-SOURCES = ["adsa_api.cu", "adsa_pool.cu", "adsa_score_select.cu", "adsa_attn.cu", "adsa_step.cu", "adsa_pstep.cu", "adsa_wstep.cu", "adsa_prefill.cu", "adsa_attn_static.cu"]
+SOURCES = ["adsa_api.cu", "adsa_pool.cu", "adsa_score_select.cu", "adsa_attn.cu", "adsa_step.cu", "adsa_pstep.cu", "adsa_wstep.cu", "adsa_prefill.cu", "adsa_attn_static.cu", "adsa_shell.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -1,0 +1,168 @@
+"""The host model's operations around the attention (adsa_rmsnorm, adsa_swiglu, adsa_cfg_sample) against the oracle.
+
+Outputs in bf16 are compared within one rounding of the exact value (2^-8 relative: bf16 keeps 8 significant bits).
+The sampled token is an integer decided by floating-point sums, taken in fp32 on the GPU and in fp64 by the oracle;
+what is unique is compared exactly (the argmax, exact ties), and otherwise the token is checked to be a valid answer:
+it belongs to the kept set and the caller's uniform number falls in its share of the cumulative distribution, within
+the rounding of an fp32 sum.
+"""
+import numpy as np
+import pytest
+import torch
+
+from adsa_workloads import bf16_bits_to_f32, f32_to_bf16_bits
+
+pytestmark = pytest.mark.gpu
+
+BF16_RTOL = 2.0 ** -8 * 1.02
+CDF_EPS = 2e-5
+
+
+def _dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to("cuda:0").view(torch.bfloat16)
+
+
+def _bf16_normal(rng, shape, scale=1.0):
+    return f32_to_bf16_bits((scale * rng.standard_normal(shape)).astype(np.float32))
+
+
+def _host(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("rows,dim,eps", [(32, 1280, 1e-5), (7, 96, 1e-5), (1, 8, 0.0), (513, 1024, 1e-6), (3, 4096, 1e-5)])
+def test_rmsnorm_matches_the_oracle(rows, dim, eps):
+    import paper_2506_18226_b200 as A
+    from oracle import adsa_oracle as orc
+    rng = np.random.default_rng(rows + dim)
+    xb, wb = _bf16_normal(rng, (rows, dim), 3.0), _bf16_normal(rng, (dim,))
+    want = orc.rmsnorm(bf16_bits_to_f32(xb), bf16_bits_to_f32(wb), eps)
+    x = _dev(xb)
+    got = A.rmsnorm(x, _dev(wb), eps=eps)
+    torch.cuda.synchronize()
+    assert np.all(np.abs(_host(got) - want) <= BF16_RTOL * np.abs(want) + 1e-30)
+    A.rmsnorm(x, _dev(wb), out=x, eps=eps)                      # in place
+    torch.cuda.synchronize()
+    assert torch.equal(x, got)
+
+
+def test_rmsnorm_of_a_zero_row_is_zero():
+    import paper_2506_18226_b200 as A
+    x = torch.zeros((2, 64), dtype=torch.bfloat16, device="cuda:0")
+    w = torch.ones(64, dtype=torch.bfloat16, device="cuda:0")
+    assert torch.equal(A.rmsnorm(x, w, eps=1e-5), x)
+
+
+@pytest.mark.parametrize("rows,hidden,fused", [(32, 3584, False), (32, 3584, True), (5, 8, False), (129, 264, True)])
+def test_swiglu_matches_the_oracle(rows, hidden, fused):
+    import paper_2506_18226_b200 as A
+    from oracle import adsa_oracle as orc
+    rng = np.random.default_rng(rows * 7 + hidden)
+    both = _bf16_normal(rng, (rows, 2 * hidden), 2.5)
+    gate_f, up_f = bf16_bits_to_f32(both[:, :hidden]), bf16_bits_to_f32(both[:, hidden:])
+    want = orc.swiglu(np.ascontiguousarray(gate_f), np.ascontiguousarray(up_f))
+    if fused:                                                    # one tensor that holds both halves side by side
+        t = _dev(both)
+        got = A.swiglu(t[:, :hidden], t[:, hidden:])
+    else:
+        got = A.swiglu(_dev(np.ascontiguousarray(both[:, :hidden])), _dev(np.ascontiguousarray(both[:, hidden:])))
+    torch.cuda.synchronize()
+    assert np.all(np.abs(_host(got) - want) <= BF16_RTOL * np.abs(want) + 1e-30)
+
+
+def _check_tokens(logits_bits, n_images, scale, top_k, temperature, uniforms, tokens):
+    """Every token is a valid answer for its image (see the module docstring)."""
+    from oracle import adsa_oracle as orc
+    lf = bf16_bits_to_f32(logits_bits)
+    exact = 0
+    for b in range(n_images):
+        want, mixed, cdf = orc.cfg_sample(lf[b], lf[n_images + b], scale, top_k, temperature, float(uniforms[b]))
+        t = int(tokens[b])
+        exact += t == want
+        kth = np.sort(mixed)[-top_k]
+        assert mixed[t] >= kth - 1e-5 * max(1.0, abs(kth)), (b, t, want)              # kept (or tied with the last kept one)
+        before = cdf[t - 1] if t > 0 else 0.0
+        assert before - CDF_EPS <= uniforms[b] <= cdf[t] + CDF_EPS, (b, t, want, before, cdf[t], uniforms[b])
+    return exact
+
+
+@pytest.mark.parametrize("n_images,vocab,scale,top_k,temperature", [
+    (16, 16384, 7.5, 2000, 1.0),       # the codebook and the sampling defaults of the decoder family
+    (16, 16384, 1.75, 16384, 1.0),     # nothing filtered
+    (3, 1000, 4.0, 50, 0.7),
+    (5, 32768, 2.0, 300, 1.3),         # the largest vocabulary the kernel takes
+    (2, 37, 1.0, 5, 1.0),              # fewer ids than threads
+])
+def test_cfg_sample_tokens_are_valid_draws(n_images, vocab, scale, top_k, temperature):
+    import paper_2506_18226_b200 as A
+    rng = np.random.default_rng(vocab + top_k)
+    lb = _bf16_normal(rng, (2 * n_images, vocab), 2.0)
+    u = rng.random(n_images).astype(np.float32)
+    u[0] = 0.0                                                                        # the first kept id
+    toks = A.cfg_sample(_dev(lb), scale, top_k, temperature, torch.from_numpy(u).to("cuda:0"))
+    toks2 = A.cfg_sample(_dev(lb), scale, top_k, temperature, torch.from_numpy(u).to("cuda:0"))
+    torch.cuda.synchronize()
+    assert torch.equal(toks, toks2)                                                   # a call is reproducible
+    exact = _check_tokens(lb, n_images, scale, top_k, temperature, u, toks.cpu().numpy())
+    assert exact >= n_images - 1                                                      # and nearly always the oracle's own token
+
+
+def test_cfg_sample_top_1_is_the_argmax_with_the_lowest_id_among_equals():
+    import paper_2506_18226_b200 as A
+    from oracle import adsa_oracle as orc
+    rng = np.random.default_rng(3)
+    n, vocab = 8, 16384
+    lb = _bf16_normal(rng, (2 * n, vocab), 1.0)        # bf16 values repeat: equal maxima do occur
+    lf = bf16_bits_to_f32(lb)
+    lf[n:] = 0.0                                       # unconditional rows zero and scale 1: the mix is the conditional row, exactly
+    lf[1, 100] = lf[1, 9000] = lf[1].max() + 1.0       # a planted tie for the maximum
+    lb = f32_to_bf16_bits(lf)
+    u = rng.random(n).astype(np.float32)
+    toks = A.cfg_sample(_dev(lb), 1.0, 1, 1.0, torch.from_numpy(u).to("cuda:0")).cpu().numpy()
+    lf = bf16_bits_to_f32(lb)
+    for b in range(n):
+        assert toks[b] == int(np.argmax(lf[b])) == orc.cfg_sample(lf[b], lf[n + b], 1.0, 1, 1.0, float(u[b]))[0]
+    assert toks[1] == 100
+
+
+def test_cfg_sample_ties_at_the_threshold_keep_the_lower_ids():
+    """Logits 5 at id 7, 1 at ids 20, 300 and 9000, everything else -30: top_k = 3 keeps ids 7, 20 and 300.  The
+    shares are exp(0) : exp(-4) : exp(-4); a grid of u must return exactly those ids, in the oracle's proportions,
+    and never id 9000."""
+    import paper_2506_18226_b200 as A
+    from oracle import adsa_oracle as orc
+    vocab, n = 16384, 64
+    row = np.full(vocab, -30.0, np.float32)
+    row[7], row[20], row[300], row[9000] = 5.0, 1.0, 1.0, 1.0
+    lf = np.concatenate([np.tile(row, (n, 1)), np.zeros((n, vocab), np.float32)])
+    u = ((np.arange(n) + 0.5) / n).astype(np.float32)
+    toks = A.cfg_sample(_dev(f32_to_bf16_bits(lf)), 1.0, 3, 1.0, torch.from_numpy(u).to("cuda:0")).cpu().numpy()
+    want = np.array([orc.cfg_sample(lf[b], lf[n + b], 1.0, 3, 1.0, float(u[b]))[0] for b in range(n)])
+    assert set(toks.tolist()) <= {7, 20, 300}
+    assert np.array_equal(toks, want)
+
+
+def test_shell_calls_refuse_bad_arguments():
+    import paper_2506_18226_b200 as A
+    B = A.binding
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda:0")
+    w = torch.ones(64, dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(A.AdsaError) as e:
+        A.rmsnorm(x[:, :60], w[:60])                   # dim not a multiple of 8 (and rows no longer contiguous)
+    assert e.value.status == B.EINVAL
+    flat = torch.zeros(4 * 64 + 8, dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(A.AdsaError) as e:
+        A.rmsnorm(flat[4:4 + 256].view(4, 64), w)      # rows that do not start on a 16-byte boundary
+    assert e.value.status == B.EINVAL
+    lg = torch.zeros((4, 100), dtype=torch.bfloat16, device="cuda:0")
+    un = torch.zeros(2, dtype=torch.float32, device="cuda:0")
+    for bad in (dict(top_k=0), dict(top_k=101), dict(temperature=0.0)):
+        kw = dict(scale=1.0, top_k=10, temperature=1.0)
+        kw.update(bad)
+        with pytest.raises(A.AdsaError) as e:
+            A.cfg_sample(lg, kw["scale"], kw["top_k"], kw["temperature"], un)
+        assert e.value.status == B.EINVAL
+    big = torch.zeros((2, 40000), dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(A.AdsaError) as e:
+        A.cfg_sample(big, 1.0, 10, 1.0, un[:1])        # vocabulary above 32768
+    assert e.value.status == B.EINVAL
