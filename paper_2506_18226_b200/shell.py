@@ -1,0 +1,173 @@
+"""A LlamaGen-shaped decoder around the ADSA attention, with random weights (Section 5 integrates the method with
+LlamaGen; trained weights are not available, so this shell has the decoder's shapes and data flow and nothing of
+its quality).
+
+What runs where: the attention, the KV cache, the rotary embedding, the normalisations, the gated activation and
+the sampling are libadsa calls; the projections, the residual additions and the embedding look-up are torch
+(cuBLAS GEMMs: plain library contractions); the token ids go to a pinned host buffer as they are drawn, one
+asynchronous copy per step (Section 4.2: generated ids are kept on the host until the image is decoded).
+
+One block: x -> RMSNorm -> q, k, v projections -> 2-D RoPE on q and k -> ADSA layer-step -> output projection
+(+ residual) -> RMSNorm -> gate/up projection -> silu(gate) * up -> down projection (+ residual).  Classifier-free
+guidance doubles the batch: rows [0, n_images) are conditional, rows [n_images, 2 n_images) unconditional; both
+halves are fed the same sampled ids.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+from . import binding as B
+
+
+@dataclass(frozen=True)
+class ShellConfig:
+    n_layers: int
+    dim: int
+    n_heads: int
+    ffn_hidden: int
+    vocab: int = 16384
+    n_text: int = 120
+    grid_h: int = 32
+    grid_w: int = 32
+    n_images: int = 16
+    budget_fraction: float = 0.5
+    cfg_scale: float = 7.5
+    top_k: int = 2000
+    temperature: float = 1.0
+    norm_eps: float = 1e-5
+
+    @property
+    def head_dim(self) -> int:
+        return self.dim // self.n_heads
+
+    @property
+    def batch(self) -> int:
+        return 2 * self.n_images
+
+    @property
+    def capacity(self) -> int:
+        return int(self.budget_fraction * (self.n_text + self.grid_h * self.grid_w) + 1e-9)
+
+
+# the three decoder sizes the benchmark configurations are shaped after (hidden sizes: 2/3 * 4 * dim rounded up to 256)
+SHAPES = {
+    "B": dict(n_layers=12, dim=768, n_heads=12, ffn_hidden=2048),
+    "L": dict(n_layers=24, dim=1024, n_heads=16, ffn_hidden=2816),
+    "XL": dict(n_layers=36, dim=1280, n_heads=20, ffn_hidden=3584),
+}
+
+
+class LlamaGenShell:
+    def __init__(self, cfg: ShellConfig, seed: int = 0, device: str = "cuda:0"):
+        self.cfg, self.dev = cfg, torch.device(device)
+        g = torch.Generator(device=self.dev).manual_seed(seed)
+        bf = dict(dtype=torch.bfloat16, device=self.dev)
+
+        def w(*shape):
+            return (0.02 * torch.randn(*shape, generator=g, device=self.dev)).to(torch.bfloat16)
+
+        L, D, Hd, V = cfg.n_layers, cfg.dim, cfg.ffn_hidden, cfg.vocab
+        self.tok_emb = w(V, D)
+        self.wq, self.wk, self.wv, self.wo = w(L, D, D), w(L, D, D), w(L, D, D), w(L, D, D)
+        self.w13 = w(L, 2 * Hd, D)          # gate and up projections side by side
+        self.w2 = w(L, D, Hd)
+        self.norm1 = torch.ones(L, D, **bf)
+        self.norm2 = torch.ones(L, D, **bf)
+        self.norm_f = torch.ones(D, **bf)
+        self.head = w(V, D)
+        C = cfg.capacity
+        from adsa_workloads import pick_page_rows
+        self.eng = B.AdsaEngine(n_layers=L, batch=cfg.batch, n_heads=cfg.n_heads, head_dim=cfg.head_dim, n_text=cfg.n_text,
+                                grid_h=cfg.grid_h, grid_w=cfg.grid_w, max_rows_per_stream=max(C, cfg.n_text) + 1,
+                                page_rows=pick_page_rows(C, hi=1024), device=device)
+        self.budget = max(C, cfg.n_text + 1)
+        Bt, H, d = cfg.batch, cfg.n_heads, cfg.head_dim
+        self.q, self.k, self.v, self.o = (torch.empty(Bt, H, d, **bf) for _ in range(4))
+        self.h = torch.empty(Bt, D, **bf)
+        self.gu = torch.empty(Bt, 2 * Hd, **bf)
+        self.act = torch.empty(Bt, Hd, **bf)
+        self.logits = torch.empty(Bt, V, **bf)
+        self.pos = torch.zeros(Bt * H, dtype=torch.int32, device=self.dev)
+        self.tokens = torch.zeros(cfg.n_images, dtype=torch.int32, device=self.dev)
+        self.ids_host = torch.zeros(cfg.grid_h * cfg.grid_w, cfg.n_images, dtype=torch.int32).pin_memory()
+        # the random numbers of the whole generation, drawn once (the sampling call takes them as an input)
+        self.uniforms = torch.rand(cfg.grid_h * cfg.grid_w, cfg.n_images, generator=g, device=self.dev, dtype=torch.float32)
+        self.kernel_calls = 0               # libadsa calls made (each is at least one kernel of the library)
+
+    # -- one block on a [rows, dim] activation; `attend` does the attention for this layer ------------------------
+    def _block(self, layer, x, attend):
+        c = self.cfg
+        step = x.shape[0] == c.batch                                       # a decode step reuses its buffers
+        h = B.rmsnorm(x, self.norm1[layer], out=self.h if step else None, eps=c.norm_eps)
+        attn = attend(layer, h)                                            # [rows, dim]
+        x.addmm_(attn, self.wo[layer].t())
+        h = B.rmsnorm(x, self.norm2[layer], out=self.h if step else None, eps=c.norm_eps)
+        gu = torch.mm(h, self.w13[layer].t(), out=self.gu) if step else h @ self.w13[layer].t()
+        act = B.swiglu(gu[:, :c.ffn_hidden], gu[:, c.ffn_hidden:], out=self.act if step else None)
+        x.addmm_(act, self.w2[layer].t())
+        self.kernel_calls += 3
+        return x
+
+    def prefill(self, text_emb):
+        """The condition: text_emb [batch, n_text, dim] bf16 (rows of the unconditional half are the caller's null
+        condition).  Fills the caches through dense causal attention and returns the first image tokens."""
+        c = self.cfg
+        Bt, T, H, d = c.batch, c.n_text, c.n_heads, c.head_dim
+        self.eng.reset()
+        x = text_emb.reshape(Bt * T, c.dim).clone()
+        pos = torch.arange(T, dtype=torch.int32, device=self.dev).repeat(Bt * H)            # condition rows are not rotated
+        out = torch.empty(Bt, H, T, d, dtype=torch.bfloat16, device=self.dev)
+
+        def attend(layer, h):
+            q, k, v = ((h @ wm[layer].t()).view(Bt, T, H, d).transpose(1, 2).contiguous() for wm in (self.wq, self.wk, self.wv))
+            self.eng.rope_2d(q, pos)
+            self.eng.rope_2d(k, pos)
+            self.eng.prefill_attn(layer, q, k, v, 0, out)
+            self.kernel_calls += 3
+            return out.transpose(1, 2).reshape(Bt * T, c.dim)
+
+        for layer in range(c.n_layers):
+            x = self._block(layer, x, attend)
+        return self._sample(x.view(Bt, T, c.dim)[:, -1].contiguous(), 0)
+
+    def decode_step(self, cell):
+        """The image token of grid cell `cell` (>= 1) from the token of cell - 1: one pass through every layer."""
+        c = self.cfg
+        cur = c.n_text + cell - 1                                          # position of the token that is fed in
+        emb = self.tok_emb[self.tokens.long()]
+        x = torch.cat([emb, emb], dim=0)                                   # conditional and unconditional rows
+        self.pos.fill_(cur)
+
+        def attend(layer, h):
+            torch.mm(h, self.wq[layer].t(), out=self.q.view(c.batch, c.dim))
+            torch.mm(h, self.wk[layer].t(), out=self.k.view(c.batch, c.dim))
+            torch.mm(h, self.wv[layer].t(), out=self.v.view(c.batch, c.dim))
+            self.eng.rope_2d(self.q, self.pos)
+            self.eng.rope_2d(self.k, self.pos)
+            self.eng.layer_step(layer, cur, self.budget, self.q, self.k, self.v, self.o)
+            self.kernel_calls += 3
+            return self.o.view(c.batch, c.dim)
+
+        for layer in range(c.n_layers):
+            x = self._block(layer, x, attend)
+        return self._sample(x, cell)
+
+    def _sample(self, x_last, cell):
+        c = self.cfg
+        h = B.rmsnorm(x_last, self.norm_f, eps=c.norm_eps)
+        torch.mm(h, self.head.t(), out=self.logits)
+        B.cfg_sample(self.logits, c.cfg_scale, min(c.top_k, c.vocab), c.temperature, self.uniforms[cell], tokens=self.tokens)
+        self.ids_host[cell].copy_(self.tokens, non_blocking=True)          # ids leave the GPU as they are drawn
+        self.kernel_calls += 2
+        return self.tokens
+
+    def generate(self, text_emb, n_cells=None):
+        """Prefill and decode `n_cells` grid cells (default: the whole grid); returns the ids on the host, [cells, n_images]."""
+        n = self.cfg.grid_h * self.cfg.grid_w if n_cells is None else n_cells
+        self.prefill(text_emb)
+        for cell in range(1, n):
+            self.decode_step(cell)
+        torch.cuda.synchronize(self.dev)
+        return self.ids_host[:n]

@@ -166,3 +166,25 @@ def test_shell_calls_refuse_bad_arguments():
     with pytest.raises(A.AdsaError) as e:
         A.cfg_sample(big, 1.0, 10, 1.0, un[:1])        # vocabulary above 32768
     assert e.value.status == B.EINVAL
+
+
+def test_model_shell_generates_an_image_worth_of_tokens():
+    """The LlamaGen-shaped shell (random weights) end to end on a small shape: the condition is prefilled through
+    dense causal attention, every grid cell is decoded through all layers with the cache at half the context, ids
+    arrive on the host; the same seed gives the same ids, the caches end at the budget, no status bit is set."""
+    from paper_2506_18226_b200.shell import LlamaGenShell, ShellConfig
+    cfg = ShellConfig(n_layers=2, dim=128, n_heads=2, ffn_hidden=256, vocab=512, n_text=8, grid_h=6, grid_w=6, n_images=2,
+                      top_k=50)
+    runs = []
+    for _ in range(2):
+        sh = LlamaGenShell(cfg, seed=5)
+        g = torch.Generator(device="cuda:0").manual_seed(9)
+        text = torch.randn(cfg.batch, cfg.n_text, cfg.dim, generator=g, device="cuda:0").to(torch.bfloat16)
+        ids = sh.generate(text).clone()
+        assert ids.shape == (36, 2) and int(ids.min()) >= 0 and int(ids.max()) < cfg.vocab
+        assert sh.eng.get_status()[0] == 0
+        n_live = sh.eng._t["n_live"].cpu().numpy()
+        assert (n_live == min(sh.budget, cfg.n_text + 35)).all()      # 35 tokens were fed in after the condition
+        runs.append(ids)
+    assert torch.equal(runs[0], runs[1])
+    assert len(set(runs[0].flatten().tolist())) > 4                    # not a constant sequence
