@@ -54,6 +54,8 @@ def parse_args(argv=None):
     ap.add_argument("--beta", type=float, default=None)
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
     ap.add_argument("--head-dim", type=int, default=0, help="override the head dimension (experiments with other row widths)")
+    ap.add_argument("--shell", default="", choices=["", "B", "L", "XL"],
+                    help="also time whole generations of the LlamaGen-shaped model shell of this size (detail.model_shell)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -577,6 +579,35 @@ def memory_vs_batch(args, dev):
     return rows
 
 
+def model_shell(args, dev):
+    """Whole generations through the LlamaGen-shaped shell (random weights): the condition is prefilled, every grid
+    cell is decoded through all layers (torch GEMMs around libadsa's kernels, one ADSA layer-step launch per layer,
+    because every layer's q/k/v depend on the layer before), ids go to the host as they are drawn."""
+    from paper_2506_18226_b200.shell import SHAPES, LlamaGenShell, ShellConfig
+    grid = {"B": 16, "L": 24, "XL": 32}[args.shell]
+    n_images = {"B": 1, "L": 8, "XL": 16}[args.shell]
+    cfg = ShellConfig(grid_h=grid, grid_w=grid, n_images=n_images, **SHAPES[args.shell])
+    sh = LlamaGenShell(cfg, seed=args.seed, device=str(dev))
+    g = torch.Generator(device=dev).manual_seed(args.seed + 1)
+    text = torch.randn(cfg.batch, cfg.n_text, cfg.dim, generator=g, device=dev).to(torch.bfloat16)
+    sh.generate(text, n_cells=min(64, grid * grid))          # warm-up: kernels loaded, cuBLAS handles made
+    times = []
+    for _ in range(2):
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        ids = sh.generate(text)
+        times.append(time.perf_counter() - t0)
+    t = min(times)
+    cells = grid * grid
+    weights = sum(x.numel() for x in (sh.wq, sh.wk, sh.wv, sh.wo, sh.w13, sh.w2, sh.head, sh.tok_emb)) * 2
+    return {"shape": args.shell, "layers": cfg.n_layers, "dim": cfg.dim, "heads": cfg.n_heads, "ffn_hidden": cfg.ffn_hidden,
+            "vocab": cfg.vocab, "n_images": n_images, "batch_rows": cfg.batch, "grid": [grid, grid], "capacity_rows": cfg.capacity,
+            "image_tokens_per_s": n_images * cells / t, "ms_per_token": t / cells * 1e3, "seconds_per_generation": t,
+            "weights_bytes": weights, "ids_on_host": int(ids.numel()), "data": "random weights, random condition embeddings",
+            "timing": "wall clock around prefill + every decode step + the final synchronisation, best of 2",
+            "status": int(sh.eng.get_status()[0])}
+
+
 def run_ours(args, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -622,6 +653,8 @@ def run_ours(args, rank, world, local_rank):
             torch.cuda.empty_cache()
     if not args.no_memory_sweep and world == 1:
         detail["memory_vs_batch"] = memory_vs_batch(args, dev)
+    if args.shell and world == 1:
+        detail["model_shell"] = model_shell(args, dev)
 
     ms, tokens = res["ms"], res["tokens"]
     line = {

@@ -84,12 +84,15 @@ class LlamaGenShell:
                                 page_rows=pick_page_rows(C, hi=1024), device=device)
         self.budget = max(C, cfg.n_text + 1)
         Bt, H, d = cfg.batch, cfg.n_heads, cfg.head_dim
-        self.q, self.k, self.v, self.o = (torch.empty(Bt, H, d, **bf) for _ in range(4))
+        self.qkv = torch.empty(3, Bt, H, d, **bf)    # q, k, v of a decode step, each dense [batch, heads, head_dim]
+        self.q, self.k, self.v = self.qkv[0], self.qkv[1], self.qkv[2]
+        self.o = torch.empty(Bt, H, d, **bf)
+        self.wqkv_t = torch.stack([self.wq, self.wk, self.wv], dim=1).transpose(2, 3).contiguous()   # [L, 3, dim(in), dim(out)]
         self.h = torch.empty(Bt, D, **bf)
         self.gu = torch.empty(Bt, 2 * Hd, **bf)
         self.act = torch.empty(Bt, Hd, **bf)
         self.logits = torch.empty(Bt, V, **bf)
-        self.pos = torch.zeros(Bt * H, dtype=torch.int32, device=self.dev)
+        self.pos = torch.zeros(2 * Bt * H, dtype=torch.int32, device=self.dev)   # one per row of q and of k
         self.tokens = torch.zeros(cfg.n_images, dtype=torch.int32, device=self.dev)
         self.ids_host = torch.zeros(cfg.grid_h * cfg.grid_w, cfg.n_images, dtype=torch.int32).pin_memory()
         # the random numbers of the whole generation, drawn once (the sampling call takes them as an input)
@@ -141,13 +144,10 @@ class LlamaGenShell:
         self.pos.fill_(cur)
 
         def attend(layer, h):
-            torch.mm(h, self.wq[layer].t(), out=self.q.view(c.batch, c.dim))
-            torch.mm(h, self.wk[layer].t(), out=self.k.view(c.batch, c.dim))
-            torch.mm(h, self.wv[layer].t(), out=self.v.view(c.batch, c.dim))
-            self.eng.rope_2d(self.q, self.pos)
-            self.eng.rope_2d(self.k, self.pos)
+            torch.bmm(h.unsqueeze(0).expand(3, -1, -1), self.wqkv_t[layer], out=self.qkv.view(3, c.batch, c.dim))   # one batched GEMM
+            self.eng.rope_2d(self.qkv[:2], self.pos)                       # q and k in one call
             self.eng.layer_step(layer, cur, self.budget, self.q, self.k, self.v, self.o)
-            self.kernel_calls += 3
+            self.kernel_calls += 2
             return self.o.view(c.batch, c.dim)
 
         for layer in range(c.n_layers):
