@@ -599,13 +599,42 @@ def model_shell(args, dev):
         times.append(time.perf_counter() - t0)
     t = min(times)
     cells = grid * grid
+    # the three stateless kernels on their own, at sizes larger than L2 (CUDA events, 20 launches each)
+    import paper_2506_18226_b200 as A
+    hbm, _ = peaks()
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / 20 * 1e3     # us
+
+    rows = 65536
+    x = torch.randn(rows, cfg.dim, device=dev).to(torch.bfloat16)
+    y = torch.empty_like(x)
+    us_norm = timed(lambda: A.rmsnorm(x, sh.norm_f, out=y, eps=cfg.norm_eps))
+    gu = torch.randn(rows, 2 * cfg.ffn_hidden, device=dev).to(torch.bfloat16)
+    act = torch.empty(rows, cfg.ffn_hidden, dtype=torch.bfloat16, device=dev)
+    us_act = timed(lambda: A.swiglu(gu[:, :cfg.ffn_hidden], gu[:, cfg.ffn_hidden:], out=act))
+    us_sample = timed(lambda: A.cfg_sample(sh.logits, cfg.cfg_scale, min(cfg.top_k, cfg.vocab), cfg.temperature, sh.uniforms[0],
+                                           tokens=sh.tokens))
+    b_norm, b_act = 2 * x.numel() * 2, 3 * act.numel() * 2
+    ops = {"rmsnorm": {"rows": rows, "dim": cfg.dim, "us": us_norm, "gbs": b_norm / us_norm * 1e-3, "frac_of_measured_copy": b_norm / us_norm * 1e-3 / hbm},
+           "swiglu": {"rows": rows, "hidden": cfg.ffn_hidden, "us": us_act, "gbs": b_act / us_act * 1e-3, "frac_of_measured_copy": b_act / us_act * 1e-3 / hbm},
+           "cfg_sample": {"n_images": n_images, "vocab": cfg.vocab, "top_k": min(cfg.top_k, cfg.vocab), "us": us_sample}}
+    del x, y, gu, act
     weights = sum(x.numel() for x in (sh.wq, sh.wk, sh.wv, sh.wo, sh.w13, sh.w2, sh.head, sh.tok_emb)) * 2
     return {"shape": args.shell, "layers": cfg.n_layers, "dim": cfg.dim, "heads": cfg.n_heads, "ffn_hidden": cfg.ffn_hidden,
             "vocab": cfg.vocab, "n_images": n_images, "batch_rows": cfg.batch, "grid": [grid, grid], "capacity_rows": cfg.capacity,
             "image_tokens_per_s": n_images * cells / t, "ms_per_token": t / cells * 1e3, "seconds_per_generation": t,
             "weights_bytes": weights, "ids_on_host": int(ids.numel()), "data": "random weights, random condition embeddings",
             "timing": "wall clock around prefill + every decode step + the final synchronisation, best of 2",
-            "status": int(sh.eng.get_status()[0])}
+            "kernels_alone": ops, "status": int(sh.eng.get_status()[0])}
 
 
 def run_ours(args, rank, world, local_rank):

@@ -248,7 +248,7 @@ int adsa_swiglu(const void *gate, const void *up, void *out, long long rows, int
     if (rows == 0) return ADSA_OK;
     const long long pieces = rows * (hidden / 8);
     long long blocks = (pieces + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > 148 * 128) blocks = 148 * 128;
     adsa::swiglu_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16 *)gate, (const __nv_bfloat16 *)up,
                                                                               (__nv_bfloat16 *)out, rows, hidden, ld_in);
     return cudaGetLastError() == cudaSuccess ? ADSA_OK : ADSA_ECUDA;
