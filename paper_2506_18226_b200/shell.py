@@ -60,8 +60,9 @@ SHAPES = {
 
 
 class LlamaGenShell:
-    def __init__(self, cfg: ShellConfig, seed: int = 0, device: str = "cuda:0"):
+    def __init__(self, cfg: ShellConfig, seed: int = 0, device: str = "cuda:0", use_graphs: bool = True):
         self.cfg, self.dev = cfg, torch.device(device)
+        self.use_graphs, self.graphs = use_graphs, None
         g = torch.Generator(device=self.dev).manual_seed(seed)
         bf = dict(dtype=torch.bfloat16, device=self.dev)
 
@@ -98,6 +99,8 @@ class LlamaGenShell:
         # the random numbers of the whole generation, drawn once (the sampling call takes them as an input)
         self.uniforms = torch.rand(cfg.grid_h * cfg.grid_w, cfg.n_images, generator=g, device=self.dev, dtype=torch.float32)
         self.kernel_calls = 0               # libadsa calls made (each is at least one kernel of the library)
+        self.x = torch.empty(Bt, D, **bf)   # the residual stream of a decode step
+        self.u = torch.zeros(cfg.n_images, dtype=torch.float32, device=self.dev)   # this step's uniform numbers
 
     # -- one block on a [rows, dim] activation; `attend` does the attention for this layer ------------------------
     def _block(self, layer, x, attend):
@@ -135,10 +138,80 @@ class LlamaGenShell:
             x = self._block(layer, x, attend)
         return self._sample(x.view(Bt, T, c.dim)[:, -1].contiguous(), 0)
 
+    # -- a decode step as CUDA graphs around the attention launches ---------------------------------------------------
+    # Everything between two attention launches works on fixed buffers with fixed arguments, so it is captured once:
+    # graph 0 = embedding look-up and the first block's part before the attention; graph l + 1 = block l's part after
+    # the attention and block l + 1's part before it (the last one ends with the LM head and the sampling).  The
+    # attention launches stay outside: their arguments (position, budget, carried state) change every step.
+    def _pre(self, layer):
+        c = self.cfg
+        B.rmsnorm(self.x, self.norm1[layer], out=self.h, eps=c.norm_eps)
+        torch.bmm(self.h.unsqueeze(0).expand(3, -1, -1), self.wqkv_t[layer], out=self.qkv.view(3, c.batch, c.dim))
+        self.eng.rope_2d(self.qkv[:2], self.pos)
+
+    def _post(self, layer):
+        c = self.cfg
+        self.x.addmm_(self.o.view(c.batch, c.dim), self.wo[layer].t())
+        B.rmsnorm(self.x, self.norm2[layer], out=self.h, eps=c.norm_eps)
+        torch.mm(self.h, self.w13[layer].t(), out=self.gu)
+        B.swiglu(self.gu[:, :c.ffn_hidden], self.gu[:, c.ffn_hidden:], out=self.act)
+        self.x.addmm_(self.act, self.w2[layer].t())
+
+    def _first(self):
+        n = self.cfg.n_images
+        torch.index_select(self.tok_emb, 0, self.tokens, out=self.x[:n])
+        self.x[n:].copy_(self.x[:n])                                       # conditional and unconditional rows
+        self._pre(0)
+
+    def _last(self):
+        c = self.cfg
+        B.rmsnorm(self.x, self.norm_f, out=self.h, eps=c.norm_eps)
+        torch.mm(self.h, self.head.t(), out=self.logits)
+        B.cfg_sample(self.logits, c.cfg_scale, min(c.top_k, c.vocab), c.temperature, self.u, tokens=self.tokens)
+
+    def _segments(self):
+        L = self.cfg.n_layers
+        segs = [self._first]
+        for layer in range(L):
+            nxt = (lambda l=layer: (self._post(l), self._pre(l + 1))) if layer + 1 < L else (lambda l=layer: (self._post(l), self._last()))
+            segs.append(nxt)
+        return segs
+
+    def _capture(self):
+        segs = self._segments()
+        side = torch.cuda.Stream(device=self.dev)
+        side.wait_stream(torch.cuda.current_stream(self.dev))
+        with torch.cuda.stream(side):                                      # once eagerly: libraries make their handles and workspaces
+            for seg in segs:
+                seg()
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        torch.cuda.synchronize(self.dev)
+        graphs = []
+        for seg in segs:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                seg()
+            graphs.append(g)
+        self.graphs = graphs
+
     def decode_step(self, cell):
         """The image token of grid cell `cell` (>= 1) from the token of cell - 1: one pass through every layer."""
         c = self.cfg
         cur = c.n_text + cell - 1                                          # position of the token that is fed in
+        if self.use_graphs:
+            if self.graphs is None:
+                saved = self.tokens.clone()
+                self._capture()                                            # (the capture's trial run overwrote the ids)
+                self.tokens.copy_(saved)
+            self.pos.fill_(cur)
+            self.u.copy_(self.uniforms[cell])
+            self.graphs[0].replay()
+            for layer in range(c.n_layers):
+                self.eng.layer_step(layer, cur, self.budget, self.q, self.k, self.v, self.o)
+                self.graphs[layer + 1].replay()
+            self.ids_host[cell].copy_(self.tokens, non_blocking=True)
+            self.kernel_calls += 5 * c.n_layers + 3
+            return self.tokens
         emb = self.tok_emb[self.tokens.long()]
         x = torch.cat([emb, emb], dim=0)                                   # conditional and unconditional rows
         self.pos.fill_(cur)

@@ -188,3 +188,14 @@ def test_model_shell_generates_an_image_worth_of_tokens():
         runs.append(ids)
     assert torch.equal(runs[0], runs[1])
     assert len(set(runs[0].flatten().tolist())) > 4                    # not a constant sequence
+
+
+def test_model_shell_graphs_and_eager_steps_draw_the_same_ids():
+    """The decode step replayed from CUDA graphs around the attention launches gives the ids of the eager step."""
+    from paper_2506_18226_b200.shell import LlamaGenShell, ShellConfig
+    cfg = ShellConfig(n_layers=3, dim=128, n_heads=2, ffn_hidden=256, vocab=512, n_text=8, grid_h=6, grid_w=6, n_images=2,
+                      top_k=50)
+    g = torch.Generator(device="cuda:0").manual_seed(4)
+    text = torch.randn(cfg.batch, cfg.n_text, cfg.dim, generator=g, device="cuda:0").to(torch.bfloat16)
+    ids = [LlamaGenShell(cfg, seed=2, use_graphs=flag).generate(text).clone() for flag in (True, False)]
+    assert torch.equal(ids[0], ids[1])
