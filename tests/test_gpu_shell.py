@@ -199,3 +199,76 @@ def test_model_shell_graphs_and_eager_steps_draw_the_same_ids():
     text = torch.randn(cfg.batch, cfg.n_text, cfg.dim, generator=g, device="cuda:0").to(torch.bfloat16)
     ids = [LlamaGenShell(cfg, seed=2, use_graphs=flag).generate(text).clone() for flag in (True, False)]
     assert torch.equal(ids[0], ids[1])
+
+
+def test_model_shell_logits_follow_a_float64_replica():
+    """The whole data flow of the shell against a replica assembled from the oracle's functions and float64 matrix
+    products, rounding to bf16 where the shell stores bf16 (so that what is compared is the wiring, not the storage
+    type): the logits after the condition and after each of three decode steps.  The budget covers the whole context
+    here, so the attention is dense causal attention (Sec. 4.2: identical to the baseline while the cache is not
+    full) and no selection can flip.  The replica is fed the ids the shell drew."""
+    from oracle import adsa_oracle as orc
+    from paper_2506_18226_b200.shell import LlamaGenShell, ShellConfig
+    cfg = ShellConfig(n_layers=2, dim=128, n_heads=2, ffn_hidden=256, vocab=512, n_text=6, grid_h=4, grid_w=4, n_images=2,
+                      top_k=40, budget_fraction=1.0)
+    sh = LlamaGenShell(cfg, seed=11, use_graphs=False)
+    gen = torch.Generator(device="cuda:0").manual_seed(12)
+    text = torch.randn(cfg.batch, cfg.n_text, cfg.dim, generator=gen, device="cuda:0").to(torch.bfloat16)
+    Bt, T, H, d, D, L = cfg.batch, cfg.n_text, cfg.n_heads, cfg.head_dim, cfg.dim, cfg.n_layers
+
+    def f64(t):
+        return t.float().cpu().numpy().astype(np.float64)
+
+    def r(a):                                                   # round to bf16, as every stored activation is
+        return bf16_bits_to_f32(f32_to_bf16_bits(np.asarray(a, dtype=np.float32))).astype(np.float64)
+
+    W = {n: f64(getattr(sh, n)) for n in ("tok_emb", "wq", "wk", "wv", "wo", "w13", "w2", "norm1", "norm2", "norm_f", "head")}
+    Kc = [[[np.zeros((0, d)) for _ in range(H)] for _ in range(Bt)] for _ in range(L)]      # the replica's caches
+    Vc = [[[np.zeros((0, d)) for _ in range(H)] for _ in range(Bt)] for _ in range(L)]
+
+    def block(l, x, positions, causal):
+        h = r(orc.rmsnorm(x, W["norm1"][l], cfg.norm_eps))
+        q, k, v = (r(h @ W[n][l].T).reshape(Bt, -1, H, d) for n in ("wq", "wk", "wv"))
+        n_new = q.shape[1]
+        attn = np.zeros((Bt, n_new, H, d))
+        for b in range(Bt):
+            for hh in range(H):
+                qr = r(orc.rope_2d(q[b, :, hh], positions, cfg.n_text, cfg.grid_w))
+                kr = r(orc.rope_2d(k[b, :, hh], positions, cfg.n_text, cfg.grid_w))
+                Kall = np.concatenate([Kc[l][b][hh], kr]); Vall = np.concatenate([Vc[l][b][hh], v[b, :, hh]])
+                if causal:
+                    attn[b, :, hh] = orc.causal_attend(qr, kr, v[b, :, hh])
+                else:
+                    attn[b, 0, hh] = orc.attend(qr[0], Kall, Vall)[0]
+                Kc[l][b][hh], Vc[l][b][hh] = Kall, Vall
+        attn = r(attn).reshape(Bt * n_new, D)
+        x = r(x + attn @ W["wo"][l].T)
+        h = r(orc.rmsnorm(x, W["norm2"][l], cfg.norm_eps))
+        gu = r(h @ W["w13"][l].T)
+        act = r(orc.swiglu(np.ascontiguousarray(gu[:, :cfg.ffn_hidden]), np.ascontiguousarray(gu[:, cfg.ffn_hidden:])))
+        return r(x + act @ W["w2"][l].T)
+
+    def logits_of(x_last):
+        return r(r(orc.rmsnorm(x_last, W["norm_f"], cfg.norm_eps)) @ W["head"].T)
+
+    def close(got, want):
+        err = np.linalg.norm(got - want) / np.linalg.norm(want)
+        cos = float((got * want).sum() / (np.linalg.norm(got) * np.linalg.norm(want)))
+        assert err <= 5e-2 and cos >= 0.998, (err, cos)
+
+    # the condition
+    sh.prefill(text)
+    x = f64(text).reshape(Bt * T, D)
+    for l in range(L):
+        x = block(l, x, np.arange(T, dtype=np.int32), causal=True)
+    close(f64(sh.logits), logits_of(x.reshape(Bt, T, D)[:, -1]))
+    # three decode steps, fed the ids the shell drew
+    for cell in range(1, 4):
+        ids = sh.tokens.cpu().numpy()
+        sh.decode_step(cell)
+        emb = W["tok_emb"][ids]
+        x = np.concatenate([emb, emb])
+        for l in range(L):
+            x = block(l, x, np.array([cfg.n_text + cell - 1], dtype=np.int32), causal=False)
+        close(f64(sh.logits), logits_of(x))
+    assert sh.eng.get_status()[0] == 0
