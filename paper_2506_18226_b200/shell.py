@@ -79,10 +79,11 @@ class LlamaGenShell:
         self.norm_f = torch.ones(D, **bf)
         self.head = w(V, D)
         C = cfg.capacity
-        from adsa_workloads import pick_page_rows
+        # rows per pool page: the largest divisor of the capacity up to 1024 rows, so that a full stream fills whole pages
+        page_rows = next((pr for pr in range(min(C, 1024), 15, -1) if C % pr == 0), 32)
         self.eng = B.AdsaEngine(n_layers=L, batch=cfg.batch, n_heads=cfg.n_heads, head_dim=cfg.head_dim, n_text=cfg.n_text,
                                 grid_h=cfg.grid_h, grid_w=cfg.grid_w, max_rows_per_stream=max(C, cfg.n_text) + 1,
-                                page_rows=pick_page_rows(C, hi=1024), device=device)
+                                page_rows=page_rows, device=device)
         self.budget = max(C, cfg.n_text + 1)
         Bt, H, d = cfg.batch, cfg.n_heads, cfg.head_dim
         self.qkv = torch.empty(3, Bt, H, d, **bf)    # q, k, v of a decode step, each dense [batch, heads, head_dim]
