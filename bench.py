@@ -599,6 +599,9 @@ def model_shell(args, dev):
         times.append(time.perf_counter() - t0)
     t = min(times)
     cells = grid * grid
+    status = int(sh.eng.get_status()[0])
+    weights = sum(x.numel() for x in (sh.wq, sh.wk, sh.wv, sh.wo, sh.w13, sh.w2, sh.head, sh.tok_emb)) * 2
+    n_ids = int(ids.numel())
     # the three stateless kernels on their own, at sizes larger than L2 (CUDA events, 20 launches each)
     import paper_2506_18226_b200 as A
     hbm, _ = peaks()
@@ -628,13 +631,29 @@ def model_shell(args, dev):
            "swiglu": {"rows": rows, "hidden": cfg.ffn_hidden, "us": us_act, "gbs": b_act / us_act * 1e-3, "frac_of_measured_copy": b_act / us_act * 1e-3 / hbm},
            "cfg_sample": {"n_images": n_images, "vocab": cfg.vocab, "top_k": min(cfg.top_k, cfg.vocab), "us": us_sample}}
     del x, y, gu, act
-    weights = sum(x.numel() for x in (sh.wq, sh.wk, sh.wv, sh.wo, sh.w13, sh.w2, sh.head, sh.tok_emb)) * 2
+    # Device memory the shell holds (weights, KV pool with its metadata, workspace, activations) against the number of
+    # images, with the cache at the budget and with a cache for the whole context: allocated bytes, not a formula
+    # (Sec. 5, "GPU Memory-efficient Image Generation", Fig. 8).
+    del sh
+    torch.cuda.empty_cache()
+    mem = []
+    for n_img in (1, 2, 4, 8, 16, 32):
+        row = {"n_images": n_img, "batch_rows": 2 * n_img}
+        for key, frac in (("adsa_bytes", cfg.budget_fraction), ("dense_bytes", 1.0)):
+            base = torch.cuda.memory_allocated(dev)
+            tmp = LlamaGenShell(ShellConfig(grid_h=grid, grid_w=grid, n_images=n_img, budget_fraction=frac, **SHAPES[args.shell]),
+                                seed=args.seed, device=str(dev))
+            row[key] = torch.cuda.memory_allocated(dev) - base
+            del tmp
+            torch.cuda.empty_cache()
+        row["ratio"] = row["adsa_bytes"] / row["dense_bytes"]
+        mem.append(row)
     return {"shape": args.shell, "layers": cfg.n_layers, "dim": cfg.dim, "heads": cfg.n_heads, "ffn_hidden": cfg.ffn_hidden,
             "vocab": cfg.vocab, "n_images": n_images, "batch_rows": cfg.batch, "grid": [grid, grid], "capacity_rows": cfg.capacity,
             "image_tokens_per_s": n_images * cells / t, "ms_per_token": t / cells * 1e3, "seconds_per_generation": t,
-            "weights_bytes": weights, "ids_on_host": int(ids.numel()), "data": "random weights, random condition embeddings",
+            "weights_bytes": weights, "ids_on_host": n_ids, "data": "random weights, random condition embeddings",
             "timing": "wall clock around prefill + every decode step + the final synchronisation, best of 2",
-            "kernels_alone": ops, "status": int(sh.eng.get_status()[0])}
+            "kernels_alone": ops, "memory_vs_images_allocated": mem, "status": status}
 
 
 def run_ours(args, rank, world, local_rank):

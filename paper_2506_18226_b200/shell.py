@@ -71,25 +71,24 @@ class LlamaGenShell:
 
         L, D, Hd, V = cfg.n_layers, cfg.dim, cfg.ffn_hidden, cfg.vocab
         self.tok_emb = w(V, D)
-        self.wq, self.wk, self.wv, self.wo = w(L, D, D), w(L, D, D), w(L, D, D), w(L, D, D)
+        self.wqkv_t = w(L, 3, D, D)         # q, k, v projections, stored transposed: [layer][which][in][out]
+        self.wo = w(L, D, D)
         self.w13 = w(L, 2 * Hd, D)          # gate and up projections side by side
         self.w2 = w(L, D, Hd)
         self.norm1 = torch.ones(L, D, **bf)
         self.norm2 = torch.ones(L, D, **bf)
         self.norm_f = torch.ones(D, **bf)
         self.head = w(V, D)
-        C = cfg.capacity
+        C = self.budget = max(cfg.capacity, cfg.n_text + 1)   # rows a stream may hold (a row is evicted before one is inserted)
         # rows per pool page: the largest divisor of the capacity up to 1024 rows, so that a full stream fills whole pages
         page_rows = next((pr for pr in range(min(C, 1024), 15, -1) if C % pr == 0), 32)
         self.eng = B.AdsaEngine(n_layers=L, batch=cfg.batch, n_heads=cfg.n_heads, head_dim=cfg.head_dim, n_text=cfg.n_text,
-                                grid_h=cfg.grid_h, grid_w=cfg.grid_w, max_rows_per_stream=max(C, cfg.n_text) + 1,
+                                grid_h=cfg.grid_h, grid_w=cfg.grid_w, max_rows_per_stream=C,
                                 page_rows=page_rows, device=device)
-        self.budget = max(C, cfg.n_text + 1)
         Bt, H, d = cfg.batch, cfg.n_heads, cfg.head_dim
         self.qkv = torch.empty(3, Bt, H, d, **bf)    # q, k, v of a decode step, each dense [batch, heads, head_dim]
         self.q, self.k, self.v = self.qkv[0], self.qkv[1], self.qkv[2]
         self.o = torch.empty(Bt, H, d, **bf)
-        self.wqkv_t = torch.stack([self.wq, self.wk, self.wv], dim=1).transpose(2, 3).contiguous()   # [L, 3, dim(in), dim(out)]
         self.h = torch.empty(Bt, D, **bf)
         self.gu = torch.empty(Bt, 2 * Hd, **bf)
         self.act = torch.empty(Bt, Hd, **bf)
@@ -102,6 +101,11 @@ class LlamaGenShell:
         self.kernel_calls = 0               # libadsa calls made (each is at least one kernel of the library)
         self.x = torch.empty(Bt, D, **bf)   # the residual stream of a decode step
         self.u = torch.zeros(cfg.n_images, dtype=torch.float32, device=self.dev)   # this step's uniform numbers
+
+    # the projections in the usual [out][in] orientation (views)
+    wq = property(lambda self: self.wqkv_t[:, 0].transpose(1, 2))
+    wk = property(lambda self: self.wqkv_t[:, 1].transpose(1, 2))
+    wv = property(lambda self: self.wqkv_t[:, 2].transpose(1, 2))
 
     # -- one block on a [rows, dim] activation; `attend` does the attention for this layer ------------------------
     def _block(self, layer, x, attend):
@@ -128,7 +132,7 @@ class LlamaGenShell:
         out = torch.empty(Bt, H, T, d, dtype=torch.bfloat16, device=self.dev)
 
         def attend(layer, h):
-            q, k, v = ((h @ wm[layer].t()).view(Bt, T, H, d).transpose(1, 2).contiguous() for wm in (self.wq, self.wk, self.wv))
+            q, k, v = ((h @ self.wqkv_t[layer, i]).view(Bt, T, H, d).transpose(1, 2).contiguous() for i in range(3))
             self.eng.rope_2d(q, pos)
             self.eng.rope_2d(k, pos)
             self.eng.prefill_attn(layer, q, k, v, 0, out)
