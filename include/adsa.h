@@ -248,12 +248,26 @@ ADSA_API int adsa_layer_step_host(adsa_ctx *ctx, int layer, int cur_pos, int bud
 ADSA_API int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
                              const void *v_new, void *out_bf16, adsa_stream_t stream);
 
+/* adsa_token_step whose inputs may still be on their way when it is called: layer l's q, k_new and v_new are read
+ * only once ready[l] - epoch >= 0 (wrap-around comparison), where ready is an int32 [n_layers] array in device
+ * memory that the caller's own copies or kernels write AFTER the layer's tensors, in an order the device sees
+ * (the same stream as those copies, or a release at system scope).  Whatever writes the words must not wait for
+ * this call's kernel.  A stream waits for its layer's word for about a second; then it sets the device status
+ * ADSA_DEV_COPY_TIMEOUT, reads what is there and goes on (later waits of that warp are a millisecond), so the
+ * kernel always ends and the context stays usable (adsa_get_status; adsa_reset clears the state).  Needs the one
+ * launch for all layers that adsa_token_step describes: ADSA_ESTATE when the tensor-core kernel cannot serve the
+ * configuration in one launch or the layers are not all between steps in the same carried state.
+ * This is how adsa_token_step_host overlaps its copies with the kernel. */
+ADSA_API int adsa_token_step_gated(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new,
+                                   const void *v_new, void *out_bf16, const int32_t *ready, int32_t epoch,
+                                   adsa_stream_t stream);
+
 /* adsa_token_step with HOST tensors of the same shapes.  The inputs cross the bus in chunks of layers on a copy
  * stream that the context creates on its first call here, while earlier layers compute on `stream`:
  *   - inputs in pinned host memory, and one launch of the tensor-core kernel can serve the whole stack (see
  *     adsa_token_step): that launch is queued at once; every chunk of copies is followed by a small copy that marks
- *     its layers as landed, and the kernel waits for a layer's mark (bounded: after a second or two it sets the
- *     device status ADSA_DEV_COPY_TIMEOUT and reads what is there) before it reads that layer's q, k_new, v_new;
+ *     its layers as landed, and the kernel waits for a layer's mark (adsa_token_step_gated: bounded, with the
+ *     device status ADSA_DEV_COPY_TIMEOUT when a wait runs out) before it reads that layer's q, k_new, v_new;
  *   - otherwise, or after adsa_set_host_chunks(2 .. 6): every chunk of layers is a launch of its own, queued
  *     behind its copies (pageable memory works here, but its copies overlap nothing).
  * An output buffer in pinned, mapped host memory (cudaHostAlloc, cudaHostRegister) is written by the kernels

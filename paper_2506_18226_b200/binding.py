@@ -21,7 +21,7 @@ DEV_POOL_EXHAUSTED, DEV_BAD_POSITION, DEV_ROW_OVERFLOW, DEV_RING_TIMEOUT, DEV_BA
 EXPORTS = [
     "adsa_workspace_bytes", "adsa_create", "adsa_destroy", "adsa_reset", "adsa_prefill_rows",
     "adsa_set_stream_rows", "adsa_prefill_attn", "adsa_rope_2d", "adsa_score", "adsa_select", "adsa_sparse_decode_attn", "adsa_kv_update",
-    "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_host_chunks", "adsa_set_stream_warps", "adsa_set_single_sweep",
+    "adsa_layer_step", "adsa_layer_step_host", "adsa_token_step", "adsa_token_step_gated", "adsa_token_step_host", "adsa_plan_attn", "adsa_set_attn_chunk_rows", "adsa_set_staged", "adsa_set_ring_stages", "adsa_set_l2_lookahead", "adsa_set_next_layer_hint", "adsa_set_token_launch", "adsa_set_host_chunks", "adsa_set_stream_warps", "adsa_set_single_sweep",
     "adsa_layer_rows_bound", "adsa_get_status", "adsa_launch_count", "adsa_strerror", "adsa_decode_attn_static",
     "adsa_rmsnorm", "adsa_swiglu", "adsa_cfg_sample",
 ]
@@ -72,6 +72,7 @@ def load(rebuild: bool = False) -> C.CDLL:
             "adsa_layer_step_host": [vp, i32, i32, i32, vp, vp, vp, vp, vp],
             "adsa_token_step": [vp, i32, i32, vp, vp, vp, vp, vp],
             "adsa_token_step_host": [vp, i32, i32, vp, vp, vp, vp, vp],
+            "adsa_token_step_gated": [vp, i32, i32, vp, vp, vp, vp, vp, i32, vp],
             "adsa_plan_attn": [vp, i32, C.POINTER(i32), C.POINTER(i32)],
             "adsa_set_attn_chunk_rows": [vp, i32],
             "adsa_set_staged": [vp, i32],
@@ -291,6 +292,11 @@ class AdsaEngine:
         """All layers of one token; tensors are [n_layers, batch, heads, head_dim] bf16 on the device."""
         self._call("adsa_token_step", cur_pos, budget_rows, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out_bf16),
                    _stream())
+
+    def token_step_gated(self, cur_pos, budget_rows, q, k_new, v_new, out_bf16, ready, epoch):
+        """token_step that reads layer l's inputs only once ready[l] - epoch >= 0 (ready: int32 [n_layers] on the device)."""
+        self._call("adsa_token_step_gated", cur_pos, budget_rows, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out_bf16),
+                   _ptr(ready), int(epoch), _stream())
 
     def token_step_host(self, cur_pos, budget_rows, q, k_new, v_new, out):
         """token_step with HOST tensors (pinned for asynchronous copies).  Synchronises the stream."""

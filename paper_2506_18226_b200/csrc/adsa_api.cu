@@ -702,6 +702,16 @@ int adsa_token_step(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, 
     return step_layers(ctx, 0, ctx->cfg.n_layers, cur_pos, budget_rows, q, k_new, v_new, out_bf16, stream);
 }
 
+int adsa_token_step_gated(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q, const void *k_new, const void *v_new,
+                          void *out_bf16, const int32_t *ready, int32_t epoch, adsa_stream_t stream)
+{
+    if (!ctx || !q || !k_new || !v_new || !out_bf16 || !ready) return ADSA_EINVAL;
+    if (ctx->cuda_error) return ADSA_ECUDA;
+    if (cur_pos < 0 || budget_rows < 1) return ADSA_EINVAL;
+    if (!one_launch_possible(ctx, 0, ctx->cfg.n_layers, cur_pos, nullptr)) return ADSA_ESTATE;
+    return step_layers(ctx, 0, ctx->cfg.n_layers, cur_pos, budget_rows, q, k_new, v_new, out_bf16, stream, ready, epoch);
+}
+
 int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host, const void *k_new_host,
                          const void *v_new_host, void *out_host, adsa_stream_t stream)
 {

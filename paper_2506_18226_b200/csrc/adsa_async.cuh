@@ -8,7 +8,7 @@ namespace adsa {
 
 constexpr int kCopySpinLimit = 1 << 20;          // polls of one mbarrier before a block gives up on it
 constexpr int kCopySpinAfterTimeout = 1 << 10;   // once a wait has run out, later waits of that thread are short
-constexpr int kInputSpinLimit = 1 << 21;         // polls (a load and a 200 ns sleep each) of an inputs-have-landed word: a second or two
+constexpr int kInputSpinLimit = 1 << 19;         // polls (a load and a 200 ns sleep each) of an inputs-have-landed word: about a second
 
 // ---- PTX wrappers ---------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }

@@ -788,6 +788,60 @@ def test_token_step_host_full_size_waits_for_its_inputs():
         assert e.get_status()[0] == 0
 
 
+def test_gated_token_step_waits_for_its_words_and_gives_up_after_a_bounded_time():
+    """adsa_token_step_gated reads a layer's inputs only after the layer's word says they have landed.  With the
+    words set it equals adsa_token_step bit for bit.  With words that nothing ever sets the kernel does not hang:
+    every wait runs out after a bounded time, the device status reports ADSA_DEV_COPY_TIMEOUT, the call returns,
+    and after a reset the context works as before."""
+    import time
+    import paper_2506_18226_b200 as A
+    H = _harness()
+    w = Workload("gated", 95, 3, 2, 4, 64, 12, 8, 8, 0.5, 1.0)
+    C, L = w.capacity(), w.n_layers
+    shape = (L, w.batch, w.n_heads, w.head_dim)
+
+    def fresh():
+        e = H.engine_for(w, capacity=C, page_rows=16)
+        for l in range(L):
+            k, v = prefix_kv(w, 6, l)
+            e.prefill_rows(l, H.dev_bf16(k), H.dev_bf16(v), 0)
+        return e
+
+    def inputs(g):
+        per = [layer_step_qkv(w, 6, l, g) for l in range(L)]
+        return [H.dev_bf16(np.stack([x[i] for x in per]).reshape(shape)) for i in range(3)]
+
+    ref, eng = fresh(), fresh()
+    ready = torch.zeros(L, dtype=torch.int32, device="cuda:0")
+    out_r, out_g = (torch.zeros(shape, dtype=torch.bfloat16, device="cuda:0") for _ in range(2))
+    for g in range(6):                                        # words written before the call: no waiting at all
+        q, k, v = inputs(g)
+        ready.fill_(g + 1)
+        ref.token_step(w.n_text + g, C, q, k, v, out_r)
+        eng.token_step_gated(w.n_text + g, C, q, k, v, out_g, ready, g + 1)
+        assert torch.equal(out_r, out_g)
+    assert eng.get_status()[0] == 0
+    # words that stay behind: the step ends by itself and says so
+    q, k, v = inputs(6)
+    t0 = time.perf_counter()
+    eng.token_step_gated(w.n_text + 6, C, q, k, v, out_g, ready, 1000)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert eng.get_status()[0] & A.binding.DEV_COPY_TIMEOUT
+    assert 0.05 < waited < 20.0
+    # the context is usable again after a reset
+    eng.reset()
+    for l in range(L):
+        kk, vv = prefix_kv(w, 6, l)
+        eng.prefill_rows(l, H.dev_bf16(kk), H.dev_bf16(vv), 0)
+    ref2 = fresh()
+    q, k, v = inputs(0)
+    ready.fill_(5)
+    ref2.token_step(w.n_text, C, q, k, v, out_r)
+    eng.token_step_gated(w.n_text, C, q, k, v, out_g, ready, 5)
+    assert torch.equal(out_r, out_g) and eng.get_status()[0] == 0
+
+
 def test_error_paths_return_status_and_launch_nothing():
     import paper_2506_18226_b200 as A
     H = _harness()
