@@ -636,6 +636,16 @@ def model_shell(args, dev):
     # (Sec. 5, "GPU Memory-efficient Image Generation", Fig. 8).
     del sh
     torch.cuda.empty_cache()
+    # the same generation with a cache for the whole context (nothing is ever evicted: dense attention)
+    dense = LlamaGenShell(ShellConfig(grid_h=grid, grid_w=grid, n_images=n_images, budget_fraction=1.0, **SHAPES[args.shell]),
+                          seed=args.seed, device=str(dev))
+    dense.generate(text, n_cells=min(64, grid * grid))
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    dense.generate(text)
+    t_dense = time.perf_counter() - t0
+    del dense
+    torch.cuda.empty_cache()
     mem = []
     for n_img in (1, 2, 4, 8, 16, 32):
         row = {"n_images": n_img, "batch_rows": 2 * n_img}
@@ -651,6 +661,8 @@ def model_shell(args, dev):
     return {"shape": args.shell, "layers": cfg.n_layers, "dim": cfg.dim, "heads": cfg.n_heads, "ffn_hidden": cfg.ffn_hidden,
             "vocab": cfg.vocab, "n_images": n_images, "batch_rows": cfg.batch, "grid": [grid, grid], "capacity_rows": cfg.capacity,
             "image_tokens_per_s": n_images * cells / t, "ms_per_token": t / cells * 1e3, "seconds_per_generation": t,
+            "whole_context_cache": {"ms_per_token": t_dense / cells * 1e3, "image_tokens_per_s": n_images * cells / t_dense,
+                                    "time_ratio_adsa_over_dense": t / t_dense},
             "weights_bytes": weights, "ids_on_host": n_ids, "data": "random weights, random condition embeddings",
             "timing": "wall clock around prefill + every decode step + the final synchronisation, best of 2",
             "kernels_alone": ops, "memory_vs_images_allocated": mem, "status": status}
