@@ -272,8 +272,9 @@ ADSA_API int adsa_token_step_gated(adsa_ctx *ctx, int cur_pos, int budget_rows, 
  *     behind its copies (pageable memory works here, but its copies overlap nothing).
  * An output buffer in pinned, mapped host memory (cudaHostAlloc, cudaHostRegister) is written by the kernels
  * directly; any other host buffer is filled by copies from a staging buffer.  When the call returns every layer
- * has run and the outputs are on the host.  Uses the staging part of the workspace; results are those of
- * adsa_token_step. */
+ * has run and the outputs are on the host.  Uses the staging part of the workspace (and, on its first call, creates
+ * two streams, a few events and n_layers words of pinned host memory that live as long as the context); results
+ * are those of adsa_token_step. */
 ADSA_API int adsa_token_step_host(adsa_ctx *ctx, int cur_pos, int budget_rows, const void *q_host,
                                   const void *k_new_host, const void *v_new_host, void *out_host,
                                   adsa_stream_t stream);
